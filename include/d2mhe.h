@@ -1,0 +1,205 @@
+/*
+ * d2mhe.h - C ABI of the B200 (sm_100a) library for the private gradient update
+ * of D2-MHE: multiparty BFV over R_q = Z_q[X]/(X^N+1) in residue-number-system
+ * form, every party simulated as a batch dimension on one GPU.
+ *
+ * Citations name the passage of the paper (arXiv 2207.04604) that defines the
+ * operation: "Sec. 3.2 item k" is the k-th algorithm of the BFV summary,
+ * "Sec. 4.2 item k" the k-th multiparty function, "Algorithm 2" the
+ * privacy-preserving D-PSGD loop.
+ *
+ * Conventions
+ *  - Polynomials are row-major uint64 arrays [..., L, N] (N contiguous), limb l
+ *    holding the residues mod q_l in [0, q_l), in the COEFFICIENT domain.
+ *  - Unless a parameter says "host", every data pointer is a DEVICE pointer,
+ *    16-byte aligned, sized exactly as annotated, owned by the caller.
+ *  - Hot calls are asynchronous on the context's stream, allocate nothing and
+ *    do not synchronise.  The library allocates only in d2mhe_create.
+ *  - Every function returns a d2mhe_status (0 = success, < 0 = error) and
+ *    never aborts.  Arguments visible on the host are validated before any
+ *    launch; a failed validation launches nothing.  Asynchronous CUDA errors
+ *    and the device range flag are reported by d2mhe_sync.
+ *  - One context per host thread.  Randomness is counter based
+ *    (Philox4x32-10 keyed by `seed`), so every output is a deterministic
+ *    function of (params, seed, inputs, stream indices).
+ */
+#ifndef D2MHE_H
+#define D2MHE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct d2mhe_ctx d2mhe_ctx; /* opaque: tables, secret shares, collective key */
+typedef int32_t d2mhe_status;
+
+enum {
+  D2MHE_OK = 0,
+  D2MHE_ERR_INVALID_ARG = -1, /* NULL / misaligned pointer, zero count, bad struct_size */
+  D2MHE_ERR_BAD_PARAMS = -2,  /* moduli not prime / not 1 mod 2N / repeated / too wide  */
+  D2MHE_ERR_STATE = -3,       /* call order: keygen -> collective_pk -> encrypt ...      */
+  D2MHE_ERR_WORKSPACE = -4,   /* caller-provided workspace too small                     */
+  D2MHE_ERR_CUDA = -5,        /* a CUDA runtime call failed                              */
+  D2MHE_ERR_RANGE = -6,       /* index out of range, or a value outside (-t/2, t/2)      */
+  D2MHE_ERR_UNSUPPORTED = -7  /* operation not available for these parameters            */
+};
+
+typedef struct {
+  uint32_t struct_size;   /* = sizeof(d2mhe_params)                                      */
+  uint32_t log2_n;        /* ring degree N = 2^log2_n, 3 <= log2_n <= 16.  The protocol
+                             calls need log2_n <= 14; 15 and 16 serve the transform and
+                             multiply-add entry points only.                            */
+  uint32_t num_limbs;     /* L, 1..24                                                    */
+  uint32_t num_parties;   /* K, 1..65535                                                 */
+  const uint64_t* moduli; /* HOST array of L distinct primes, q_l = 1 mod 2N, q_l < 2^61 */
+  uint64_t plain_modulus; /* t: prime < 2^30, coprime to every q_l.  Packing
+                             (encode/decode) additionally needs t = 1 mod 2N.            */
+  uint64_t seed;          /* Philox key                                                  */
+  uint32_t gauss_bound;   /* B of the error distribution; must be 19 (sigma = 3.2)       */
+  uint32_t flags;         /* reserved, must be 0                                         */
+  int32_t device;         /* CUDA device ordinal                                         */
+} d2mhe_params;
+
+/* Validates params, builds all tables on `device`.  *out is NULL on failure. */
+d2mhe_status d2mhe_create(const d2mhe_params* params, d2mhe_ctx** out);
+void d2mhe_destroy(d2mhe_ctx* ctx);
+/* Stream (a cudaStream_t passed as void*) on which later calls are enqueued; NULL = default. */
+d2mhe_status d2mhe_set_stream(d2mhe_ctx* ctx, void* cuda_stream);
+/* Waits for the stream; returns the first asynchronous error or D2MHE_ERR_RANGE if
+ * d2mhe_encode saw a value outside [-(t-1)/2, (t-1)/2] since the last sync (flag is cleared). */
+d2mhe_status d2mhe_sync(d2mhe_ctx* ctx);
+const char* d2mhe_strerror(d2mhe_status status);
+
+/*
+ * MBFV.SecKeyGen (Sec. 4.2 item 1; BFV.SecKeyGen, Sec. 3.2 item 1): each listed
+ * party k draws s_k uniformly from R_3 (coefficients in {-1,0,1}).  The shares stay
+ * inside the context (transform domain); s = sum s_k is never formed.
+ * parties: HOST array of n_parties distinct indices < K.
+ */
+d2mhe_status d2mhe_keygen_share(d2mhe_ctx* ctx, const uint32_t* parties, uint32_t n_parties);
+
+/*
+ * MBFV.PubKeyGen (Sec. 4.2 item 2): common p_1 uniform on R_q; each listed party
+ * samples e_k from chi and forms p_{0,k} = -(p_1 s_k + e_k); pk = ([sum_k p_{0,k}]_q, p_1).
+ * All listed parties must have key shares.  The party set of the last call is the set
+ * of share holders that d2mhe_combine_decrypt expects.
+ * pk_shares_dev: optional out [n_parties, L, N] (may be NULL).
+ * pk_dev:        optional out [2, L, N] = (p_0, p_1) (may be NULL).
+ */
+d2mhe_status d2mhe_collective_pk(d2mhe_ctx* ctx, const uint32_t* parties, uint32_t n_parties,
+                                 uint64_t* pk_shares_dev, uint64_t* pk_dev);
+
+/*
+ * Packing (Sec. 6, SIMD slots): values int32 [n_cts, N] (caller zero-pads), each in
+ * [-(t-1)/2, (t-1)/2] -> plaintext polynomials uint32 [n_cts, N] in [0,t) with
+ * m(psi_t^(2j+1)) = value_j mod t, psi_t = g^((t-1)/2N) for the smallest primitive
+ * root g of t.  d2mhe_decode is the inverse, returning centred values.
+ * In-place use (values == plain storage) is allowed.
+ */
+d2mhe_status d2mhe_encode(d2mhe_ctx* ctx, const int32_t* values_dev, uint32_t n_cts,
+                          uint32_t* plain_dev);
+d2mhe_status d2mhe_decode(d2mhe_ctx* ctx, const uint32_t* plain_dev, uint32_t n_cts,
+                          int32_t* values_dev);
+
+/*
+ * BFV.Encrypt under the collective key (Sec. 3.2 item 3; Algorithm 2 lines 6, 11):
+ * ct = (Lambda m + u p_0 + e_0, u p_1 + e_1), Lambda = floor(q/t), u from R_3,
+ * e_0, e_1 from chi.  The randomness of unit (parties[a], c) is the stream
+ * (party = parties[a], ciphertext index = ct_first + c).
+ * plain_dev: [n_parties, n_cts, N] uint32 in [0,t);  ct_dev: out [n_parties, n_cts, 2, L, N].
+ */
+d2mhe_status d2mhe_encrypt(d2mhe_ctx* ctx, const uint32_t* parties, uint32_t n_parties,
+                           uint32_t ct_first, uint32_t n_cts, const uint32_t* plain_dev,
+                           uint64_t* ct_dev);
+
+/*
+ * BFV.Add over neighbour lists (Sec. 3.2 item 4; Algorithm 2 line 6 with unit weights):
+ * agg[i, c] = sum_{r in list(i)} ct[r, c] mod q, both components.
+ * ct_dev: [n_rows, n_cts, 2, L, N].  nbr_offsets (HOST, n_out+1 entries, non-decreasing,
+ * nbr_offsets[0] = 0) and nbr_rows (HOST, nbr_offsets[n_out] entries, each < n_rows) are
+ * the lists in CSR form; they are validated on the host.  An empty list gives zero.
+ * agg_dev: out [n_out, n_cts, 2, L, N]; must not overlap ct_dev.
+ * Limits: n_out <= 65536 and nbr_offsets[n_out] <= 1048576.
+ */
+d2mhe_status d2mhe_aggregate(d2mhe_ctx* ctx, const uint64_t* ct_dev, uint32_t n_rows,
+                             uint32_t n_cts, const uint32_t* nbr_offsets,
+                             const uint32_t* nbr_rows, uint32_t n_out, uint64_t* agg_dev);
+
+/*
+ * Decryption shares (Sec. 4.2 item 3, Eq. 2 with mu_k = 0; equally Eq. 4 with M_k = 0):
+ * shares[i, a, c] = s_k c_1 + e, k = parties[a], c_1 the second component of agg[i, c],
+ * e from chi on the stream (party k, recipient recipients[i], ciphertext index ct_first + c).
+ * agg_dev: [n_rec, n_cts, 2, L, N];  shares_dev: out [n_rec, n_parties, n_cts, L, N].
+ * recipients, parties: HOST arrays of indices < K.
+ */
+d2mhe_status d2mhe_partial_decrypt(d2mhe_ctx* ctx, const uint64_t* agg_dev,
+                                   const uint32_t* recipients, uint32_t n_rec,
+                                   const uint32_t* parties, uint32_t n_parties,
+                                   uint32_t ct_first, uint32_t n_cts, uint64_t* shares_dev);
+
+/*
+ * Combine and decrypt (Sec. 4.2 item 3: c_0 + sum_k h_k; Sec. 3.2 item 5:
+ * x = [ round(t/q [.]_q) ]_t, computed exactly in RNS by a mixed-radix conversion).
+ * n_shares must equal the size of the party set of the last d2mhe_collective_pk.
+ * agg_dev: [n_rec, n_cts, 2, L, N] (only c_0 is read);
+ * shares_dev: [n_rec, n_shares, n_cts, L, N];  plain_dev: out [n_rec, n_cts, N] in [0,t).
+ */
+d2mhe_status d2mhe_combine_decrypt(d2mhe_ctx* ctx, const uint64_t* agg_dev,
+                                   const uint64_t* shares_dev, uint32_t n_rec,
+                                   uint32_t n_shares, uint32_t n_cts, uint32_t* plain_dev);
+
+/*
+ * Batched negacyclic number-theoretic transform of [batch, L, N], in place.
+ * Forward: position p of limb l receives a(psi_l^(2 brv(p) + 1)), brv = reversal of
+ * the log2_n-bit index, psi_l the root reported by d2mhe_get_root.  Inverse undoes it.
+ * These are the ring isomorphism behind every product of Sec. 3.2 / 4.2.
+ */
+d2mhe_status d2mhe_ntt_forward(d2mhe_ctx* ctx, uint64_t* polys_dev, uint32_t batch);
+d2mhe_status d2mhe_ntt_inverse(d2mhe_ctx* ctx, uint64_t* polys_dev, uint32_t batch);
+/* d = a (.) b + c residue by residue on [batch, L, N] (the RNS multiply-add inside
+ * u p_0 + e_0 and s_k c_1 + e_k).  d may alias a, b or c. */
+d2mhe_status d2mhe_poly_muladd(d2mhe_ctx* ctx, const uint64_t* a_dev, const uint64_t* b_dev,
+                               const uint64_t* c_dev, uint64_t* d_dev, uint32_t batch);
+
+/*
+ * One whole private gradient update for ciphertext indices ct_first .. ct_first+n_cts-1
+ * of all K parties (Algorithm 2 lines 6-9 and 11 without the model update): encode,
+ * encrypt, neighbour sums, shares from every share holder, combine, decode.  Ciphertext
+ * indices are processed in chunks so that all protocol messages of a chunk
+ * (ciphertexts, aggregates, shares) live in the caller's workspace.
+ *   values:  int32 [K, n_cts, N]   in
+ *   sums:    int32 [K, n_cts, N]   out: sums[i] = sum over list(i) of the values
+ *   nbr_offsets / nbr_rows: HOST CSR lists over parties, K lists.
+ *   workspace_dev / workspace_bytes: device scratch, at least
+ *   d2mhe_round_workspace_bytes(ctx, 1); larger workspaces allow larger chunks.
+ * d2mhe_round_device takes device values/sums.  d2mhe_round_host takes HOST values/sums
+ * (pinned memory recommended), copies them in and out on the context's stream and
+ * returns after the stream has drained.
+ */
+size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* ctx, uint32_t chunk_cts);
+d2mhe_status d2mhe_round_device(d2mhe_ctx* ctx, const int32_t* values_dev, uint32_t ct_first,
+                                uint32_t n_cts, const uint32_t* nbr_offsets,
+                                const uint32_t* nbr_rows, int32_t* sums_dev,
+                                void* workspace_dev, size_t workspace_bytes);
+d2mhe_status d2mhe_round_host(d2mhe_ctx* ctx, const int32_t* values_host, uint32_t ct_first,
+                              uint32_t n_cts, const uint32_t* nbr_offsets,
+                              const uint32_t* nbr_rows, int32_t* sums_host,
+                              void* workspace_dev, size_t workspace_bytes);
+
+/* Test hooks. */
+/* s_k as int8 [N] on the HOST (needs a key share for `party`). */
+d2mhe_status d2mhe_debug_export_secret(d2mhe_ctx* ctx, uint32_t party, int8_t* s_host);
+/* The primitive 2N-th root of unity used for limb `limb`. */
+d2mhe_status d2mhe_get_root(const d2mhe_ctx* ctx, uint32_t limb, uint64_t* psi);
+/* psi_t, the slot root (D2MHE_ERR_UNSUPPORTED if t != 1 mod 2N). */
+d2mhe_status d2mhe_get_plain_root(const d2mhe_ctx* ctx, uint64_t* psi_t);
+/* Number of kernels this context has launched since creation. */
+uint64_t d2mhe_launch_count(const d2mhe_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* D2MHE_H */

@@ -1,0 +1,355 @@
+// Device-side building blocks: 64-bit modular arithmetic, the Philox4x32-10 sampler,
+// and the shared-memory negacyclic NTT engine used by every kernel.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+typedef unsigned long long u64;
+typedef unsigned int u32;
+
+// ---------------------------------------------------------------------------
+// Per-limb constants (one entry per RNS prime q_l), resident in global memory.
+// ---------------------------------------------------------------------------
+struct LimbTab {
+  u64 p;             // q_l
+  u64 twop;          // 2 q_l
+  u64 pinv;          // q_l^-1 mod 2^64 (Montgomery)
+  u64 one_sh;        // floor(2^64 / q_l): Shoup companion of 1, reduces any 64-bit value
+  u64 ninv, ninv_sh; // N^-1 mod q_l with Shoup companion
+  u64 mont_ninv, mont_ninv_sh;  // N^-1 * 2^64 mod q_l: x -> x * N^-1 in Montgomery form
+  u64 delta, delta_sh;          // floor(q/t) mod q_l
+  u64 tmod, tmod_sh;            // t mod q_l
+  u64 half;                     // (q-1)/2 mod q_l
+  u64 cq;                       // ceil(2^61 / q_l) * q_l: keeps Garner differences non-negative
+  u64 mask;                     // 2^bitlen(q_l) - 1, for the rejection sampler
+  u64 rmod, rmod_sh;            // 2^64 mod q_l: leaves Montgomery form
+  const ulonglong2* W;          // [N] forward twiddles psi^brv(i) as {w, floor(w 2^64 / q_l)}
+  const ulonglong2* IW;         // [N] their inverses
+};
+
+// ---------------------------------------------------------------------------
+// Modular arithmetic on [0, 2^64)
+// ---------------------------------------------------------------------------
+
+// x*w mod p in [0, 2p) for any 64-bit x, given ws = floor(w 2^64 / p), w < p.
+__host__ __device__ __forceinline__ u64 mulhi_u64(u64 a, u64 b) {
+#ifdef __CUDA_ARCH__
+  return __umul64hi(a, b);
+#else
+  return (u64)(((unsigned __int128)a * b) >> 64);
+#endif
+}
+__host__ __device__ __forceinline__ u64 shoup_lazy(u64 x, u64 w, u64 ws, u64 p) {
+  return x * w - mulhi_u64(x, ws) * p;
+}
+__host__ __device__ __forceinline__ u64 csub(u64 x, u64 p) { return x >= p ? x - p : x; }
+__host__ __device__ __forceinline__ u64 shoup_full(u64 x, u64 w, u64 ws, u64 p) {
+  return csub(shoup_lazy(x, w, ws, p), p);
+}
+// a * b * 2^-64 mod p in (0, 2p); needs b < p (a arbitrary 64-bit), pinv = p^-1 mod 2^64.
+__host__ __device__ __forceinline__ u64 mont_lazy(u64 a, u64 b, u64 p, u64 pinv) {
+  u64 lo = a * b, hi = mulhi_u64(a, b);
+  u64 h2 = mulhi_u64(lo * pinv, p);
+  return hi - h2 + p;
+}
+__host__ __device__ __forceinline__ u64 addmod(u64 a, u64 b, u64 p) { return csub(a + b, p); }
+// residue of a small signed integer
+__host__ __device__ __forceinline__ u64 lift_small(int v, u64 p) {
+  return v < 0 ? p - (u64)(-v) : (u64)v;
+}
+
+// ---------------------------------------------------------------------------
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) and the samplers
+// ---------------------------------------------------------------------------
+struct Philox {
+  u32 k0, k1;
+};
+__host__ __device__ __forceinline__ void philox4x32_10(u32 k0, u32 k1, u32 c0, u32 c1, u32 c2,
+                                                        u32 c3, u32& o0, u32& o1, u32& o2,
+                                                        u32& o3) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    u64 p0 = (u64)0xD2511F53u * c0;
+    u64 p1 = (u64)0xCD9E8D57u * c2;
+    u32 n0 = (u32)(p1 >> 32) ^ c1 ^ k0;
+    u32 n2 = (u32)(p0 >> 32) ^ c3 ^ k1;
+    c1 = (u32)p1;
+    c3 = (u32)p0;
+    c0 = n0;
+    c2 = n2;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  o0 = c0;
+  o1 = c1;
+  o2 = c2;
+  o3 = c3;
+}
+
+// Stream tags (fourth counter word, low byte)
+enum : u32 {
+  TAG_SECRET = 1,
+  TAG_PK_ERR = 2,
+  TAG_P1 = 3,
+  TAG_ENC_U = 4,
+  TAG_ENC_E0 = 5,
+  TAG_ENC_E1 = 6,
+  TAG_DEC_ERR = 7
+};
+
+// One stream: counter = (j, idx, party | recipient << 16, tag | attempt << 8).
+struct Stream {
+  u32 k0, k1;  // seed words
+  u32 c1, c2, tag;
+  __host__ __device__ __forceinline__ Stream(u64 seed, u32 tag_, u32 idx, u32 party, u32 recipient)
+      : k0((u32)seed), k1((u32)(seed >> 32)), c1(idx), c2(party | (recipient << 16)), tag(tag_) {}
+  __host__ __device__ __forceinline__ u64 draw64(u32 j, u32 attempt = 0) const {
+    u32 o0, o1, o2, o3;
+    philox4x32_10(k0, k1, j, c1, c2, tag | (attempt << 8), o0, o1, o2, o3);
+    return ((u64)o0 << 32) | o1;
+  }
+  // uniform in {-1, 0, 1}: floor(3 w0 / 2^32) - 1
+  __host__ __device__ __forceinline__ int ternary(u32 j) const {
+    u32 o0, o1, o2, o3;
+    philox4x32_10(k0, k1, j, c1, c2, tag, o0, o1, o2, o3);
+    return (int)(((u64)o0 * 3u) >> 32) - 1;
+  }
+};
+
+// Discrete Gaussian by inversion of the cumulative table: -B + #{k : r >= cdt[k]}.
+// lut[r >> 56] = (#thresholds <= bucket start) | (#thresholds inside the bucket) << 8.
+#define D2MHE_GAUSS_B 19
+#define D2MHE_CDT_LEN 38
+struct GaussTab {
+  u64 cdt[D2MHE_CDT_LEN];
+  unsigned short lut[256];
+};
+__device__ __forceinline__ int gauss_from_r(const GaussTab& g, u64 r) {
+  u32 e = g.lut[r >> 56];
+  u32 base = e & 0xffu, inside = e >> 8;
+  u32 cnt = base;
+  for (u32 i = 0; i < inside; ++i) cnt += (r >= g.cdt[base + i]) ? 1u : 0u;
+  return (int)cnt - D2MHE_GAUSS_B;
+}
+// uniform on Z_p by rejection on bitlen(p)-bit draws (attempt index in the counter)
+__host__ __device__ __forceinline__ u64 uniform_mod(const Stream& s, u32 j, u64 p, u64 mask) {
+  for (u32 attempt = 0; attempt < 255; ++attempt) {
+    u64 r = s.draw64(j, attempt) & mask;
+    if (r < p) return r;
+  }
+  return s.draw64(j, 255) % p;
+}
+
+// ---------------------------------------------------------------------------
+// Shared-memory NTT engine
+//
+// One CTA transforms one residue polynomial of N = 2^logn coefficients held in shared
+// memory.  Work is organised in radix-8 rounds: in the round that starts at stage s
+// (m = 2^s butterfly groups) a thread owns the "octet" of coefficients
+//     i * (N/m) + o + k * st,  k = 0..7,  st = N / (8m),
+// applies three butterfly stages to it in registers and writes it back; rounds are
+// separated by one barrier.  When log2 N is not a multiple of 3 the first forward
+// (last inverse) round applies only 1 or 2 stages.  The forward transform is
+// Cooley-Tukey with twiddles psi^brv(m+i) (natural order in, bit-reversed out), the
+// inverse is Gentleman-Sande; values stay in [0,4p) / [0,2p) between butterflies
+// (Harvey's lazy reduction with Shoup multiplication).
+//
+// The last forward round has st = 1: the thread ends with positions 8q..8q+7 in
+// registers, exactly the operands of the first inverse round, so pointwise products
+// are fused between the two without touching memory.
+// ---------------------------------------------------------------------------
+
+// Shared-memory index swizzle: XOR the low four index bits with bits 4..6 so that the
+// 16 threads of a half warp hit 16 distinct 8-byte banks for every stride (.., 64, 8, 1).
+__device__ __forceinline__ u32 swz(u32 a) { return a ^ ((a >> 4) & 7u) ^ (((a >> 6) & 1u) << 3); }
+
+__device__ __forceinline__ void ct_bfly(u64& X, u64& Y, const ulonglong2 w, u64 p, u64 twop) {
+  u64 x = csub(X, twop);
+  u64 t = shoup_lazy(Y, w.x, w.y, p);
+  X = x + t;
+  Y = x - t + twop;
+}
+__device__ __forceinline__ void gs_bfly(u64& X, u64& Y, const ulonglong2 w, u64 p, u64 twop) {
+  u64 s = X + Y;
+  u64 d = X - Y + twop;
+  X = csub(s, twop);
+  Y = shoup_lazy(d, w.x, w.y, p);
+}
+
+// three (or fewer) forward stages on an octet; m = groups at the first stage, i = group index
+__device__ __forceinline__ void fwd_octet(u64 (&x)[8], const ulonglong2* __restrict__ W, u32 m,
+                                          u32 i, int nst, u64 p, u64 twop) {
+  {
+    const ulonglong2 w = __ldg(W + m + i);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) ct_bfly(x[k], x[k + 4], w, p, twop);
+  }
+  if (nst >= 2) {
+    const ulonglong2 w0 = __ldg(W + 2 * m + 2 * i), w1 = __ldg(W + 2 * m + 2 * i + 1);
+    ct_bfly(x[0], x[2], w0, p, twop);
+    ct_bfly(x[1], x[3], w0, p, twop);
+    ct_bfly(x[4], x[6], w1, p, twop);
+    ct_bfly(x[5], x[7], w1, p, twop);
+  }
+  if (nst >= 3) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const ulonglong2 w = __ldg(W + 4 * m + 4 * i + r);
+      ct_bfly(x[2 * r], x[2 * r + 1], w, p, twop);
+    }
+  }
+}
+__device__ __forceinline__ void inv_octet(u64 (&x)[8], const ulonglong2* __restrict__ IW, u32 m,
+                                          u32 i, int nst, u64 p, u64 twop) {
+  if (nst >= 3) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const ulonglong2 w = __ldg(IW + 4 * m + 4 * i + r);
+      gs_bfly(x[2 * r], x[2 * r + 1], w, p, twop);
+    }
+  }
+  if (nst >= 2) {
+    const ulonglong2 w0 = __ldg(IW + 2 * m + 2 * i), w1 = __ldg(IW + 2 * m + 2 * i + 1);
+    gs_bfly(x[0], x[2], w0, p, twop);
+    gs_bfly(x[1], x[3], w0, p, twop);
+    gs_bfly(x[4], x[6], w1, p, twop);
+    gs_bfly(x[5], x[7], w1, p, twop);
+  }
+  {
+    const ulonglong2 w = __ldg(IW + m + i);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) gs_bfly(x[k], x[k + 4], w, p, twop);
+  }
+}
+
+// Geometry shared by all kernels: LOGN > 0 fixes the size at compile time (strides and
+// loop counts fold to constants); LOGN == 0 takes it from the run-time argument.
+template <int LOGN, int G>
+struct NttGeom {
+  u32 logn, n, octets, r0;
+  __device__ __forceinline__ explicit NttGeom(u32 logn_rt) {
+    logn = LOGN ? (u32)LOGN : logn_rt;
+    n = 1u << logn;
+    octets = n >> 3;
+    r0 = logn % 3u;
+  }
+};
+
+// Forward transform.  load(j) returns coefficient j in [0, p) (or any value < 4p);
+// emit(g, q, x) receives the octet of positions 8q..8q+7 (values in [0,4p)), q = tid + g*T.
+template <int LOGN, int G, class Load, class Emit>
+__device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
+                                            Load load, Emit emit) {
+  const NttGeom<LOGN, G> ge(logn_rt);
+  const u32 T = blockDim.x, tid = threadIdx.x;
+  const u64 p = lt.p, twop = lt.twop;
+  const ulonglong2* __restrict__ W = lt.W;
+  u64 x[8];
+  __syncthreads();  // previous users of sm are done
+  u32 s = 0;
+  bool from_load = true;
+  if (ge.r0) {
+    const u32 st = ge.octets;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const u32 q = tid + g * T;
+      if (q < ge.octets) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = load(q + k * st);
+        fwd_octet(x, W, 1, 0, (int)ge.r0, p, twop);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) sm[swz(q + k * st)] = x[k];
+      }
+    }
+    s = ge.r0;
+    from_load = false;
+    __syncthreads();
+  }
+  for (; s < ge.logn; s += 3) {
+    const u32 sh = ge.logn - s - 3;  // log2 of the stride
+    const u32 st = 1u << sh, m = 1u << s;
+    const bool last = (s + 3 == ge.logn);
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const u32 q = tid + g * T;
+      if (q < ge.octets) {
+        const u32 i = q >> sh, o = q & (st - 1);
+        const u32 base = ((i << 3) << sh) + o;
+        if (from_load) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) x[k] = load(base + k * st);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) x[k] = sm[swz(base + k * st)];
+        }
+        fwd_octet(x, W, m, i, 3, p, twop);
+        if (last) {
+          emit(g, q, x);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) sm[swz(base + k * st)] = x[k];
+        }
+      }
+    }
+    from_load = false;
+    if (!last) __syncthreads();
+  }
+}
+
+// Inverse transform (without the N^-1 scaling: fold it into an operand).
+// fetch(g, q, x) fills the octet of positions 8q..8q+7 with values in [0,2p);
+// store(j, v) receives coefficient j, v in [0,2p).
+template <int LOGN, int G, class Fetch, class Store>
+__device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
+                                            Fetch fetch, Store store) {
+  const NttGeom<LOGN, G> ge(logn_rt);
+  const u32 T = blockDim.x, tid = threadIdx.x;
+  const u64 p = lt.p, twop = lt.twop;
+  const ulonglong2* __restrict__ IW = lt.IW;
+  u64 x[8];
+  __syncthreads();  // previous users of sm are done
+  bool from_fetch = true;
+  for (int s = (int)ge.logn - 3; s >= (int)ge.r0; s -= 3) {
+    const u32 sh = ge.logn - (u32)s - 3;
+    const u32 st = 1u << sh, m = 1u << s;
+    const bool final_round = (s == 0);
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const u32 q = tid + g * T;
+      if (q < ge.octets) {
+        const u32 i = q >> sh, o = q & (st - 1);
+        const u32 base = ((i << 3) << sh) + o;
+        if (from_fetch) {
+          fetch(g, q, x);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) x[k] = sm[swz(base + k * st)];
+        }
+        inv_octet(x, IW, m, i, 3, p, twop);
+        if (final_round) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) store(base + k * st, x[k]);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) sm[swz(base + k * st)] = x[k];
+        }
+      }
+    }
+    from_fetch = false;
+    if (!final_round) __syncthreads();
+  }
+  if (ge.r0) {
+    const u32 st = ge.octets;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const u32 q = tid + g * T;
+      if (q < ge.octets) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = sm[swz(q + k * st)];
+        inv_octet(x, IW, 1, 0, (int)ge.r0, p, twop);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) store(q + k * st, x[k]);
+      }
+    }
+  }
+}

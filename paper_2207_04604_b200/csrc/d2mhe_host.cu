@@ -1,0 +1,818 @@
+// Host side of the C ABI: parameter validation, table construction, argument checks,
+// index staging and the chunked whole-round driver.
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/d2mhe.h"
+#include "d2mhe_internal.h"
+
+typedef unsigned __int128 u128;
+
+namespace {
+
+const u64 kGaussCdt[D2MHE_CDT_LEN] = {
+#include "dgauss_cdt.inc"
+};
+
+// ---- host arithmetic (table construction only) ------------------------------------
+u64 h_mul(u64 a, u64 b, u64 p) { return (u64)((u128)a * b % p); }
+u64 h_pow(u64 a, u64 e, u64 p) {
+  u64 r = 1 % p;
+  a %= p;
+  for (; e; e >>= 1) {
+    if (e & 1) r = h_mul(r, a, p);
+    a = h_mul(a, a, p);
+  }
+  return r;
+}
+u64 h_inv(u64 a, u64 p) { return h_pow(a, p - 2, p); }
+u64 h_shoup(u64 w, u64 p) { return (u64)(((u128)w << 64) / p); }
+
+bool h_is_prime(u64 n) {
+  if (n < 2) return false;
+  static const u64 bases[] = {2, 3, 5, 7, 11, 13, 17, 19, 23, 29, 31, 37};
+  for (u64 b : bases) {
+    if (n % b == 0) return n == b;
+  }
+  u64 d = n - 1;
+  int r = 0;
+  while ((d & 1) == 0) {
+    d >>= 1;
+    ++r;
+  }
+  for (u64 a : bases) {
+    u64 x = h_pow(a, d, n);
+    if (x == 1 || x == n - 1) continue;
+    bool composite = true;
+    for (int i = 1; i < r; ++i) {
+      x = h_mul(x, x, n);
+      if (x == n - 1) {
+        composite = false;
+        break;
+      }
+    }
+    if (composite) return false;
+  }
+  return true;
+}
+
+// first g^((p-1)/2N), g = 2, 3, ..., of multiplicative order exactly 2N
+u64 h_find_root(u64 p, u32 logn) {
+  const u64 two_n = (u64)2 << logn, n = (u64)1 << logn;
+  for (u64 g = 2; g < 4096; ++g) {
+    u64 c = h_pow(g, (p - 1) / two_n, p);
+    if (h_pow(c, n, p) == p - 1) return c;
+  }
+  return 0;
+}
+
+// smallest primitive root of the prime t
+u64 h_primitive_root(u64 t) {
+  std::vector<u64> factors;
+  u64 m = t - 1;
+  for (u64 f = 2; f * f <= m; ++f) {
+    if (m % f == 0) {
+      factors.push_back(f);
+      while (m % f == 0) m /= f;
+    }
+  }
+  if (m > 1) factors.push_back(m);
+  for (u64 g = 2; g < t; ++g) {
+    bool ok = true;
+    for (u64 f : factors) {
+      if (h_pow(g, (t - 1) / f, t) == 1) {
+        ok = false;
+        break;
+      }
+    }
+    if (ok) return g;
+  }
+  return 0;
+}
+
+u32 h_brv(u32 x, u32 bits) {
+  u32 r = 0;
+  for (u32 i = 0; i < bits; ++i) {
+    r = (r << 1) | (x & 1);
+    x >>= 1;
+  }
+  return r;
+}
+
+const size_t kIdxSlotWords = (size_t)1 << 21;  // u32 words per staging slot (8 MiB)
+const int kIdxSlots = 4;
+
+}  // namespace
+
+struct d2mhe_ctx {
+  d2mhe_params params;
+  std::vector<u64> moduli;
+  std::vector<u64> roots;
+  u64 psi_t = 0;
+  bool can_pack = false;
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  DevView view;
+  std::vector<void*> allocs;        // device allocations to free
+  std::vector<bool> has_share;
+  std::vector<u32> pk_parties;      // party set of the last collective_pk
+  bool has_pk = false;
+  u64 launches = 0;
+  // index staging: pinned host ring + device ring, one event per slot
+  u32* idx_host = nullptr;
+  u32* idx_dev = nullptr;
+  cudaEvent_t idx_event[kIdxSlots] = {};
+  bool idx_event_valid[kIdxSlots] = {};
+  int idx_next = 0;
+  cudaError_t last_cuda = cudaSuccess;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+    if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+template <class T>
+T* dev_upload(d2mhe_ctx* c, const std::vector<T>& h, cudaError_t* err) {
+  void* d = nullptr;
+  size_t bytes = std::max<size_t>(h.size() * sizeof(T), 16);
+  *err = cudaMalloc(&d, bytes);
+  if (*err != cudaSuccess) return nullptr;
+  c->allocs.push_back(d);
+  if (!h.empty()) *err = cudaMemcpy(d, h.data(), h.size() * sizeof(T), cudaMemcpyHostToDevice);
+  return reinterpret_cast<T*>(d);
+}
+template <class T>
+T* dev_alloc(d2mhe_ctx* c, size_t count, cudaError_t* err) {
+  void* d = nullptr;
+  *err = cudaMalloc(&d, std::max<size_t>(count * sizeof(T), 16));
+  if (*err != cudaSuccess) return nullptr;
+  c->allocs.push_back(d);
+  return reinterpret_cast<T*>(d);
+}
+
+d2mhe_status fail_cuda(d2mhe_ctx* c, cudaError_t e) {
+  if (c) c->last_cuda = e;
+  return D2MHE_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Stage host index arrays into the next ring slot; returns device pointers for each.
+// The slot is reused only after the work that read it has finished (event per slot).
+struct Staged {
+  const u32* dev[4] = {nullptr, nullptr, nullptr, nullptr};
+  int slot = -1;
+};
+d2mhe_status stage_indices(d2mhe_ctx* c, const u32* const* arrays, const size_t* counts, int n_arrays,
+                           Staged* out) {
+  size_t total = 0;
+  for (int i = 0; i < n_arrays; ++i) total += (counts[i] + 3) & ~(size_t)3;
+  if (total > kIdxSlotWords) return D2MHE_ERR_RANGE;
+  const int slot = c->idx_next;
+  c->idx_next = (c->idx_next + 1) % kIdxSlots;
+  if (c->idx_event_valid[slot]) {
+    cudaError_t e = cudaEventSynchronize(c->idx_event[slot]);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+  }
+  u32* h = c->idx_host + (size_t)slot * kIdxSlotWords;
+  u32* d = c->idx_dev + (size_t)slot * kIdxSlotWords;
+  size_t off = 0;
+  for (int i = 0; i < n_arrays; ++i) {
+    std::memcpy(h + off, arrays[i], counts[i] * sizeof(u32));
+    out->dev[i] = d + off;
+    off += (counts[i] + 3) & ~(size_t)3;
+  }
+  cudaError_t e = cudaMemcpyAsync(d, h, off * sizeof(u32), cudaMemcpyHostToDevice, c->stream);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  out->slot = slot;
+  return D2MHE_OK;
+}
+d2mhe_status release_slot(d2mhe_ctx* c, const Staged& s) {
+  cudaError_t e = cudaEventRecord(c->idx_event[s.slot], c->stream);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->idx_event_valid[s.slot] = true;
+  return D2MHE_OK;
+}
+
+d2mhe_status check_party_list(const d2mhe_ctx* c, const u32* parties, u32 n, bool need_share,
+                              bool distinct) {
+  if (!parties || n == 0) return D2MHE_ERR_INVALID_ARG;
+  std::vector<bool> seen(distinct ? c->params.num_parties : 0, false);
+  for (u32 i = 0; i < n; ++i) {
+    if (parties[i] >= c->params.num_parties) return D2MHE_ERR_RANGE;
+    if (need_share && !c->has_share[parties[i]]) return D2MHE_ERR_STATE;
+    if (distinct) {
+      if (seen[parties[i]]) return D2MHE_ERR_INVALID_ARG;
+      seen[parties[i]] = true;
+    }
+  }
+  return D2MHE_OK;
+}
+
+d2mhe_status build_tables(d2mhe_ctx* c) {
+  const d2mhe_params& P = c->params;
+  const u32 logn = P.log2_n, n = 1u << logn, L = P.num_limbs;
+  const u64 t = P.plain_modulus;
+  cudaError_t err = cudaSuccess;
+
+  // q as a little-endian multi-word integer is never needed: everything about q that the
+  // kernels use is a residue, computed limb by limb.
+  std::vector<LimbTab> limbs(L);
+  // (q-1)/2 mod m and q mod m for a word-size m: q = prod q_l, so q mod m by repeated products;
+  // (q-1)/2 mod m = (q-1) * 2^-1 mod m for odd m.
+  auto q_mod = [&](u64 m) {
+    u64 r = 1 % m;
+    for (u32 l = 0; l < L; ++l) r = h_mul(r, c->moduli[l] % m, m);
+    return r;
+  };
+  // floor(q/t) mod q_l: q = Delta t + (q mod t)  =>  Delta = -(q mod t) t^-1 (mod q_l)
+  const u64 q_mod_t = q_mod(t);
+
+  for (u32 l = 0; l < L; ++l) {
+    const u64 p = c->moduli[l];
+    LimbTab& T = limbs[l];
+    T.p = p;
+    T.twop = 2 * p;
+    u64 inv = 1;  // Newton iteration for p^-1 mod 2^64
+    for (int i = 0; i < 6; ++i) inv *= 2 - p * inv;
+    T.pinv = inv;
+    T.one_sh = h_shoup(1, p);
+    T.ninv = h_inv(n % p, p);
+    T.ninv_sh = h_shoup(T.ninv, p);
+    const u64 r64 = (u64)(((u128)1 << 64) % p);
+    T.mont_ninv = h_mul(T.ninv, r64, p);
+    T.mont_ninv_sh = h_shoup(T.mont_ninv, p);
+    T.rmod = r64;
+    T.rmod_sh = h_shoup(r64, p);
+    T.delta = h_mul((p - q_mod_t % p) % p, h_inv(t % p, p), p);
+    T.delta_sh = h_shoup(T.delta, p);
+    T.tmod = t % p;
+    T.tmod_sh = h_shoup(T.tmod, p);
+    // (q-1)/2 mod q_l: q = 0 mod q_l, so (q-1)/2 = -(2^-1) mod q_l = (q_l - 1)/2
+    T.half = (p - 1) / 2;
+    const u64 two61 = (u64)1 << 61;
+    T.cq = ((two61 + p - 1) / p) * p;
+    u32 bits = 0;
+    for (u64 x = p; x; x >>= 1) ++bits;
+    T.mask = bits >= 64 ? ~(u64)0 : (((u64)1 << bits) - 1);
+
+    const u64 psi = c->roots[l], psi_inv = h_inv(psi, p);
+    std::vector<u64> pw(n), ipw(n);
+    pw[0] = ipw[0] = 1;
+    for (u32 i = 1; i < n; ++i) {
+      pw[i] = h_mul(pw[i - 1], psi, p);
+      ipw[i] = h_mul(ipw[i - 1], psi_inv, p);
+    }
+    std::vector<ulonglong2> W(n), IW(n);
+    for (u32 i = 0; i < n; ++i) {
+      const u32 r = h_brv(i, logn);
+      W[i] = make_ulonglong2(pw[r], h_shoup(pw[r], p));
+      IW[i] = make_ulonglong2(ipw[r], h_shoup(ipw[r], p));
+    }
+    T.W = dev_upload(c, W, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    T.IW = dev_upload(c, IW, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+  }
+  c->view.limbs = dev_upload(c, limbs, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+
+  // Gaussian table and its first-level lookup on the top byte
+  {
+    std::vector<GaussTab> g(1);
+    for (int k = 0; k < D2MHE_CDT_LEN; ++k) g[0].cdt[k] = kGaussCdt[k];
+    for (u32 b = 0; b < 256; ++b) {
+      const u64 lo = (u64)b << 56;
+      const u64 hi = b == 255 ? ~(u64)0 : (((u64)(b + 1) << 56) - 1);
+      u32 base = 0, inside = 0;
+      for (int k = 0; k < D2MHE_CDT_LEN; ++k) {
+        if (kGaussCdt[k] <= lo)
+          ++base;
+        else if (kGaussCdt[k] <= hi)
+          ++inside;
+      }
+      g[0].lut[b] = (unsigned short)(base | (inside << 8));
+    }
+    c->view.gauss = dev_upload(c, g, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+  }
+
+  // plaintext-modulus transforms
+  PlainTab& pt = c->view.plain;
+  std::memset(&pt, 0, sizeof(pt));
+  pt.t = (u32)t;
+  pt.twot = (u32)(2 * t);
+  pt.half = (u32)((t - 1) / 2);
+  if (c->can_pack) {
+    const u64 g = h_primitive_root(t);
+    c->psi_t = h_pow(g, (t - 1) / ((u64)2 << logn), t);
+    const u64 psi = c->psi_t, psi_inv = h_inv(psi, t);
+    auto sh32 = [&](u64 w) { return (u32)((w << 32) / t); };
+    std::vector<u64> pw(n), ipw(n);
+    pw[0] = ipw[0] = 1;
+    for (u32 i = 1; i < n; ++i) {
+      pw[i] = h_mul(pw[i - 1], psi, t);
+      ipw[i] = h_mul(ipw[i - 1], psi_inv, t);
+    }
+    std::vector<uint2> W(n), IW(n);
+    for (u32 i = 0; i < n; ++i) {
+      const u32 r = h_brv(i, logn);
+      W[i] = make_uint2((u32)pw[r], sh32(pw[r]));
+      IW[i] = make_uint2((u32)ipw[r], sh32(ipw[r]));
+    }
+    pt.W = dev_upload(c, W, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    pt.IW = dev_upload(c, IW, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    pt.ninv = (u32)h_inv(n % t, t);
+    pt.ninv_sh = sh32(pt.ninv);
+  }
+
+  // exact scale-and-round constants
+  RoundTab& rt = c->view.round;
+  {
+    std::vector<ulonglong2> ginv((size_t)L * L, make_ulonglong2(0, 0));
+    std::vector<u64> prefix(L);
+    u64 acc = 1 % t;
+    for (u32 i = 0; i < L; ++i) {
+      prefix[i] = acc;
+      acc = h_mul(acc, c->moduli[i] % t, t);
+      for (u32 j = 0; j < i; ++j) {
+        const u64 pi = c->moduli[i];
+        const u64 w = h_inv(c->moduli[j] % pi, pi);
+        ginv[(size_t)i * L + j] = make_ulonglong2(w, h_shoup(w, pi));
+      }
+    }
+    rt.ginv = dev_upload(c, ginv, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    rt.prefix_mod_t = dev_upload(c, prefix, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    rt.t = t;
+    rt.t_sh = h_shoup(1, t);
+    // (q-1)/2 mod t = (q mod t - 1) * 2^-1 mod t   (t odd)
+    rt.half_mod_t = h_mul((q_mod_t + t - 1) % t, h_inv(2, t), t);
+    rt.qinv_mod_t = h_inv(q_mod_t, t);
+  }
+
+  // key storage
+  const size_t poly = (size_t)L * n;
+  c->view.s_mont = dev_alloc<u64>(c, (size_t)P.num_parties * poly, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  c->view.pk_mont = dev_alloc<u64>(c, 2 * poly, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  c->view.pk_coef = dev_alloc<u64>(c, 2 * poly, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  c->view.range_flag = dev_alloc<u32>(c, 4, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  err = cudaMemset(c->view.range_flag, 0, 16);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+
+  c->view.seed = P.seed;
+  c->view.logn = logn;
+  c->view.n = n;
+  c->view.L = L;
+  c->view.K = P.num_parties;
+
+  // index staging ring
+  err = cudaMallocHost(reinterpret_cast<void**>(&c->idx_host), kIdxSlots * kIdxSlotWords * sizeof(u32));
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  c->idx_dev = dev_alloc<u32>(c, kIdxSlots * kIdxSlotWords, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  for (int i = 0; i < kIdxSlots; ++i) {
+    err = cudaEventCreateWithFlags(&c->idx_event[i], cudaEventDisableTiming);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    c->idx_event_valid[i] = false;
+  }
+  return D2MHE_OK;
+}
+
+bool protocol_ok(const d2mhe_ctx* c) { return c->params.log2_n <= D2MHE_MAX_SMEM_LOGN; }
+
+}  // namespace
+
+extern "C" {
+
+const char* d2mhe_strerror(d2mhe_status s) {
+  switch (s) {
+    case D2MHE_OK: return "success";
+    case D2MHE_ERR_INVALID_ARG: return "invalid argument";
+    case D2MHE_ERR_BAD_PARAMS: return "bad scheme parameters";
+    case D2MHE_ERR_STATE: return "call out of order";
+    case D2MHE_ERR_WORKSPACE: return "workspace too small";
+    case D2MHE_ERR_CUDA: return "CUDA error";
+    case D2MHE_ERR_RANGE: return "index or value out of range";
+    case D2MHE_ERR_UNSUPPORTED: return "unsupported for these parameters";
+    default: return "unknown status";
+  }
+}
+
+d2mhe_status d2mhe_create(const d2mhe_params* P, d2mhe_ctx** out) {
+  if (out) *out = nullptr;
+  if (!P || !out) return D2MHE_ERR_INVALID_ARG;
+  if (P->struct_size != sizeof(d2mhe_params)) return D2MHE_ERR_INVALID_ARG;
+  if (!P->moduli) return D2MHE_ERR_INVALID_ARG;
+  if (P->log2_n < 3 || P->log2_n > 16) return D2MHE_ERR_BAD_PARAMS;
+  if (P->num_limbs < 1 || P->num_limbs > D2MHE_MAX_LIMBS) return D2MHE_ERR_BAD_PARAMS;
+  if (P->num_parties < 1 || P->num_parties > 65535) return D2MHE_ERR_BAD_PARAMS;
+  if (P->gauss_bound != D2MHE_GAUSS_B || P->flags != 0) return D2MHE_ERR_BAD_PARAMS;
+  const u64 t = P->plain_modulus, two_n = (u64)2 << P->log2_n;
+  if (t < 3 || t >= ((u64)1 << 30) || !h_is_prime(t)) return D2MHE_ERR_BAD_PARAMS;
+  for (u32 l = 0; l < P->num_limbs; ++l) {
+    const u64 p = P->moduli[l];
+    if (p >= ((u64)1 << 61) || p <= two_n || p % two_n != 1 || p == t || !h_is_prime(p))
+      return D2MHE_ERR_BAD_PARAMS;
+    for (u32 m = 0; m < l; ++m)
+      if (P->moduli[m] == p) return D2MHE_ERR_BAD_PARAMS;
+  }
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || P->device < 0 || P->device >= n_dev)
+    return D2MHE_ERR_CUDA;
+
+  d2mhe_ctx* c = new (std::nothrow) d2mhe_ctx();
+  if (!c) return D2MHE_ERR_CUDA;
+  c->params = *P;
+  c->moduli.assign(P->moduli, P->moduli + P->num_limbs);
+  c->params.moduli = reinterpret_cast<const uint64_t*>(c->moduli.data());
+  c->device = P->device;
+  c->can_pack = (t - 1) % two_n == 0;
+  c->has_share.assign(P->num_parties, false);
+  std::memset(&c->view, 0, sizeof(c->view));
+  for (u32 l = 0; l < P->num_limbs; ++l) {
+    u64 r = h_find_root(c->moduli[l], P->log2_n);
+    if (!r) {
+      delete c;
+      return D2MHE_ERR_BAD_PARAMS;
+    }
+    c->roots.push_back(r);
+  }
+  DeviceGuard guard(c->device);
+  if (!guard.ok) {
+    delete c;
+    return D2MHE_ERR_CUDA;
+  }
+  d2mhe_status st = build_tables(c);
+  if (st != D2MHE_OK) {
+    d2mhe_destroy(c);
+    return st;
+  }
+  *out = c;
+  return D2MHE_OK;
+}
+
+void d2mhe_destroy(d2mhe_ctx* c) {
+  if (!c) return;
+  DeviceGuard guard(c->device);
+  cudaDeviceSynchronize();
+  for (void* p : c->allocs) cudaFree(p);
+  if (c->idx_host) cudaFreeHost(c->idx_host);
+  for (int i = 0; i < kIdxSlots; ++i)
+    if (c->idx_event[i]) cudaEventDestroy(c->idx_event[i]);
+  delete c;
+}
+
+d2mhe_status d2mhe_set_stream(d2mhe_ctx* c, void* stream) {
+  if (!c) return D2MHE_ERR_INVALID_ARG;
+  c->stream = reinterpret_cast<cudaStream_t>(stream);
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_sync(d2mhe_ctx* c) {
+  if (!c) return D2MHE_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  u32 flag = 0;
+  e = cudaMemcpy(&flag, c->view.range_flag, sizeof(u32), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (flag) {
+    e = cudaMemset(c->view.range_flag, 0, sizeof(u32));
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    return D2MHE_ERR_RANGE;
+  }
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_keygen_share(d2mhe_ctx* c, const u32* parties, u32 n_parties) {
+  if (!c) return D2MHE_ERR_INVALID_ARG;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  d2mhe_status st = check_party_list(c, parties, n_parties, false, true);
+  if (st != D2MHE_OK) return st;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[1] = {parties};
+  const size_t counts[1] = {n_parties};
+  if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::keygen(c->view, c->stream, sg.dev[0], n_parties);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  for (u32 i = 0; i < n_parties; ++i) c->has_share[parties[i]] = true;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_collective_pk(d2mhe_ctx* c, const u32* parties, u32 n_parties,
+                                 uint64_t* pk_shares_dev, uint64_t* pk_dev) {
+  if (!c) return D2MHE_ERR_INVALID_ARG;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  d2mhe_status st = check_party_list(c, parties, n_parties, true, true);
+  if (st != D2MHE_OK) return st;
+  if (!aligned16(pk_shares_dev) || !aligned16(pk_dev)) return D2MHE_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[1] = {parties};
+  const size_t counts[1] = {n_parties};
+  if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::collective_pk(c->view, c->stream, sg.dev[0], n_parties,
+                                              reinterpret_cast<u64*>(pk_shares_dev));
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  if (pk_dev) {
+    e = cudaMemcpyAsync(pk_dev, c->view.pk_coef, 2 * (size_t)c->view.L * c->view.n * sizeof(u64),
+                        cudaMemcpyDeviceToDevice, c->stream);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+  }
+  c->pk_parties.assign(parties, parties + n_parties);
+  c->has_pk = true;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_encode(d2mhe_ctx* c, const int32_t* values_dev, u32 n_cts, u32* plain_dev) {
+  if (!c || !values_dev || !plain_dev || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(values_dev) || !aligned16(plain_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!c->can_pack || c->params.log2_n > 15) return D2MHE_ERR_UNSUPPORTED;
+  DeviceGuard guard(c->device);
+  cudaError_t e = d2mhe_launch::encode(c->view, c->stream, values_dev, n_cts, plain_dev);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_decode(d2mhe_ctx* c, const u32* plain_dev, u32 n_cts, int32_t* values_dev) {
+  if (!c || !values_dev || !plain_dev || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(values_dev) || !aligned16(plain_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!c->can_pack || c->params.log2_n > 15) return D2MHE_ERR_UNSUPPORTED;
+  DeviceGuard guard(c->device);
+  cudaError_t e = d2mhe_launch::decode(c->view, c->stream, plain_dev, n_cts, values_dev);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_encrypt(d2mhe_ctx* c, const u32* parties, u32 n_parties, u32 ct_first, u32 n_cts,
+                           const u32* plain_dev, uint64_t* ct_dev) {
+  if (!c || !plain_dev || !ct_dev || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(plain_dev) || !aligned16(ct_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  if (!c->has_pk) return D2MHE_ERR_STATE;
+  d2mhe_status st = check_party_list(c, parties, n_parties, false, false);
+  if (st != D2MHE_OK) return st;
+  if ((u64)ct_first + n_cts > 0xffffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)n_parties * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[1] = {parties};
+  const size_t counts[1] = {n_parties};
+  if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::encrypt(c->view, c->stream, sg.dev[0], n_parties, ct_first, n_cts,
+                                        plain_dev, reinterpret_cast<u64*>(ct_dev));
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_aggregate(d2mhe_ctx* c, const uint64_t* ct_dev, u32 n_rows, u32 n_cts,
+                             const u32* nbr_offsets, const u32* nbr_rows, u32 n_out,
+                             uint64_t* agg_dev) {
+  if (!c || !ct_dev || !agg_dev || !nbr_offsets || n_rows == 0 || n_cts == 0 || n_out == 0)
+    return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(ct_dev) || !aligned16(agg_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (n_out > 65536) return D2MHE_ERR_RANGE;
+  if (nbr_offsets[0] != 0) return D2MHE_ERR_INVALID_ARG;
+  for (u32 i = 0; i < n_out; ++i)
+    if (nbr_offsets[i + 1] < nbr_offsets[i]) return D2MHE_ERR_INVALID_ARG;
+  const u32 nnz = nbr_offsets[n_out];
+  if (nnz > 1048576) return D2MHE_ERR_RANGE;
+  if (nnz && !nbr_rows) return D2MHE_ERR_INVALID_ARG;
+  for (u32 a = 0; a < nnz; ++a)
+    if (nbr_rows[a] >= n_rows) return D2MHE_ERR_RANGE;
+  if ((u64)n_out * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32 dummy = 0;
+  const u32* arrays[2] = {nbr_offsets, nnz ? nbr_rows : &dummy};
+  const size_t counts[2] = {(size_t)n_out + 1, nnz ? (size_t)nnz : 1};
+  d2mhe_status st = stage_indices(c, arrays, counts, 2, &sg);
+  if (st != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::aggregate(c->view, c->stream, reinterpret_cast<const u64*>(ct_dev), n_cts,
+                                          sg.dev[0], sg.dev[1], n_out, reinterpret_cast<u64*>(agg_dev));
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_partial_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev, const u32* recipients, u32 n_rec,
+                                   const u32* parties, u32 n_parties, u32 ct_first, u32 n_cts,
+                                   uint64_t* shares_dev) {
+  if (!c || !agg_dev || !shares_dev || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(agg_dev) || !aligned16(shares_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  d2mhe_status st = check_party_list(c, recipients, n_rec, false, false);
+  if (st != D2MHE_OK) return st;
+  st = check_party_list(c, parties, n_parties, true, true);
+  if (st != D2MHE_OK) return st;
+  if ((u64)ct_first + n_cts > 0xffffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)n_rec * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[2] = {recipients, parties};
+  const size_t counts[2] = {n_rec, n_parties};
+  if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::partial_decrypt(
+      c->view, c->stream, reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1], n_parties,
+      ct_first, n_cts, reinterpret_cast<u64*>(shares_dev));
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_combine_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev,
+                                   const uint64_t* shares_dev, u32 n_rec,
+                                   u32 n_shares, u32 n_cts, u32* plain_dev) {
+  if (!c || !agg_dev || !shares_dev || !plain_dev || n_rec == 0 || n_cts == 0)
+    return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(agg_dev) || !aligned16(shares_dev) || !aligned16(plain_dev))
+    return D2MHE_ERR_INVALID_ARG;
+  if (!c->has_pk) return D2MHE_ERR_STATE;
+  if (n_shares != c->pk_parties.size()) return D2MHE_ERR_INVALID_ARG;
+  if ((u64)n_rec * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  cudaError_t e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
+                                        reinterpret_cast<const u64*>(shares_dev), n_rec, n_shares, n_cts,
+                                        plain_dev);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return D2MHE_OK;
+}
+
+static d2mhe_status ntt_common(d2mhe_ctx* c, u64* polys_dev, u32 batch, bool inverse) {
+  if (!c || !polys_dev || batch == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(polys_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (c->params.log2_n > D2MHE_MAX_SMEM_LOGN) return D2MHE_ERR_UNSUPPORTED;
+  if ((u64)batch * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  cudaError_t e = d2mhe_launch::ntt(c->view, c->stream, polys_dev, batch, inverse);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return D2MHE_OK;
+}
+d2mhe_status d2mhe_ntt_forward(d2mhe_ctx* c, uint64_t* polys_dev, u32 batch) {
+  return ntt_common(c, reinterpret_cast<u64*>(polys_dev), batch, false);
+}
+d2mhe_status d2mhe_ntt_inverse(d2mhe_ctx* c, uint64_t* polys_dev, u32 batch) {
+  return ntt_common(c, reinterpret_cast<u64*>(polys_dev), batch, true);
+}
+
+d2mhe_status d2mhe_poly_muladd(d2mhe_ctx* c, const uint64_t* a, const uint64_t* b,
+                               const uint64_t* cc, uint64_t* d, u32 batch) {
+  if (!c || !a || !b || !cc || !d || batch == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(a) || !aligned16(b) || !aligned16(cc) || !aligned16(d)) return D2MHE_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  cudaError_t e = d2mhe_launch::muladd(c->view, c->stream, reinterpret_cast<const u64*>(a),
+                                       reinterpret_cast<const u64*>(b), reinterpret_cast<const u64*>(cc),
+                                       reinterpret_cast<u64*>(d), batch);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return D2MHE_OK;
+}
+
+// ---- whole round ---------------------------------------------------------------------
+
+// Per ciphertext index of a chunk: plain K*N u32, ct and agg K*2*L*N u64 each,
+// shares K*K*L*N u64 (S = K share holders).
+static size_t round_bytes_per_ct(const d2mhe_ctx* c) {
+  const size_t K = c->params.num_parties, S = c->pk_parties.empty() ? K : c->pk_parties.size();
+  const size_t n = c->view.n, poly = (size_t)c->view.L * n * sizeof(u64);
+  return K * n * sizeof(u32) + 2 * (K * 2 * poly) + K * S * poly;
+}
+
+size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* c, u32 chunk_cts) {
+  if (!c || chunk_cts == 0) return 0;
+  return round_bytes_per_ct(c) * chunk_cts + 256;
+}
+
+static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io, u32 ct_first,
+                               u32 n_cts, const u32* nbr_offsets, const u32* nbr_rows,
+                               int32_t* sums, void* ws, size_t ws_bytes) {
+  if (!c || !values || !sums || !nbr_offsets || !nbr_rows || !ws || n_cts == 0)
+    return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(ws) || (!host_io && (!aligned16(values) || !aligned16(sums))))
+    return D2MHE_ERR_INVALID_ARG;
+  if (!protocol_ok(c) || !c->can_pack) return D2MHE_ERR_UNSUPPORTED;
+  if (!c->has_pk) return D2MHE_ERR_STATE;
+  const u32 K = c->params.num_parties, S = (u32)c->pk_parties.size();
+  const size_t n = c->view.n, polyw = (size_t)c->view.L * n;
+  const size_t per_ct = round_bytes_per_ct(c);
+  if (ws_bytes < per_ct + 256) return D2MHE_ERR_WORKSPACE;
+  u32 chunk = (u32)std::min<size_t>((ws_bytes - 256) / per_ct, n_cts);
+  // The in/out staging of the host variant lives in the plain/decoded area of the chunk.
+  std::vector<u32> all(K);
+  for (u32 i = 0; i < K; ++i) all[i] = i;
+
+  DeviceGuard guard(c->device);
+  unsigned char* base = reinterpret_cast<unsigned char*>(ws);
+  for (u32 done = 0; done < n_cts; done += chunk) {
+    const u32 cc = std::min(chunk, n_cts - done);
+    // layout for this chunk (all 16-byte aligned: every block is a multiple of 16 bytes)
+    u32* plain = reinterpret_cast<u32*>(base);
+    u64* ct = reinterpret_cast<u64*>(base + (size_t)K * cc * n * sizeof(u32));
+    u64* agg = ct + (size_t)K * cc * 2 * polyw;
+    u64* shares = agg + (size_t)K * cc * 2 * polyw;
+    // values are [K, n_cts, N]: gather the chunk's columns party by party
+    int32_t* vals_dev = reinterpret_cast<int32_t*>(plain);  // encode runs in place
+    for (u32 k = 0; k < K; ++k) {
+      const int32_t* src = values + ((size_t)k * n_cts + done) * n;
+      cudaError_t e = cudaMemcpyAsync(vals_dev + (size_t)k * cc * n, src, (size_t)cc * n * sizeof(int32_t),
+                                      host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice,
+                                      c->stream);
+      if (e != cudaSuccess) return fail_cuda(c, e);
+    }
+    d2mhe_status st;
+    if ((st = d2mhe_encode(c, vals_dev, K * cc, plain)) != D2MHE_OK) return st;
+    if ((st = d2mhe_encrypt(c, all.data(), K, ct_first + done, cc, plain, reinterpret_cast<uint64_t*>(ct))) != D2MHE_OK) return st;
+    if ((st = d2mhe_aggregate(c, reinterpret_cast<uint64_t*>(ct), K, cc, nbr_offsets, nbr_rows, K,
+                              reinterpret_cast<uint64_t*>(agg))) != D2MHE_OK) return st;
+    if ((st = d2mhe_partial_decrypt(c, reinterpret_cast<uint64_t*>(agg), all.data(), K,
+                                    c->pk_parties.data(), S, ct_first + done, cc,
+                                    reinterpret_cast<uint64_t*>(shares))) != D2MHE_OK)
+      return st;
+    if ((st = d2mhe_combine_decrypt(c, reinterpret_cast<uint64_t*>(agg), reinterpret_cast<uint64_t*>(shares),
+                                    K, S, cc, plain)) != D2MHE_OK) return st;
+    if ((st = d2mhe_decode(c, plain, K * cc, vals_dev)) != D2MHE_OK) return st;
+    for (u32 k = 0; k < K; ++k) {
+      int32_t* dst = sums + ((size_t)k * n_cts + done) * n;
+      cudaError_t e = cudaMemcpyAsync(dst, vals_dev + (size_t)k * cc * n, (size_t)cc * n * sizeof(int32_t),
+                                      host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice,
+                                      c->stream);
+      if (e != cudaSuccess) return fail_cuda(c, e);
+    }
+  }
+  if (host_io) {
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+  }
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_round_device(d2mhe_ctx* c, const int32_t* values_dev, u32 ct_first, u32 n_cts,
+                                const u32* nbr_offsets, const u32* nbr_rows, int32_t* sums_dev,
+                                void* workspace_dev, size_t workspace_bytes) {
+  return round_impl(c, values_dev, false, ct_first, n_cts, nbr_offsets, nbr_rows, sums_dev,
+                    workspace_dev, workspace_bytes);
+}
+d2mhe_status d2mhe_round_host(d2mhe_ctx* c, const int32_t* values_host, u32 ct_first, u32 n_cts,
+                              const u32* nbr_offsets, const u32* nbr_rows, int32_t* sums_host,
+                              void* workspace_dev, size_t workspace_bytes) {
+  return round_impl(c, values_host, true, ct_first, n_cts, nbr_offsets, nbr_rows, sums_host,
+                    workspace_dev, workspace_bytes);
+}
+
+// ---- test hooks ----------------------------------------------------------------------
+
+d2mhe_status d2mhe_debug_export_secret(d2mhe_ctx* c, u32 party, int8_t* s_host) {
+  if (!c || !s_host) return D2MHE_ERR_INVALID_ARG;
+  if (party >= c->params.num_parties) return D2MHE_ERR_RANGE;
+  if (!c->has_share[party]) return D2MHE_ERR_STATE;
+  const Stream st(c->params.seed, TAG_SECRET, 0, party, 0);
+  for (u32 j = 0; j < c->view.n; ++j) s_host[j] = (int8_t)st.ternary(j);
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_get_root(const d2mhe_ctx* c, u32 limb, uint64_t* psi) {
+  if (!c || !psi) return D2MHE_ERR_INVALID_ARG;
+  if (limb >= c->params.num_limbs) return D2MHE_ERR_RANGE;
+  *psi = c->roots[limb];
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_get_plain_root(const d2mhe_ctx* c, uint64_t* psi_t) {
+  if (!c || !psi_t) return D2MHE_ERR_INVALID_ARG;
+  if (!c->can_pack) return D2MHE_ERR_UNSUPPORTED;
+  *psi_t = c->psi_t;
+  return D2MHE_OK;
+}
+
+uint64_t d2mhe_launch_count(const d2mhe_ctx* c) { return c ? c->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,63 @@
+// Host-side view of the context and the kernel launch entry points.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "d2mhe_device.cuh"
+
+#define D2MHE_MAX_LIMBS 24
+#define D2MHE_MAX_SMEM_LOGN 14  // largest polynomial that fits one CTA's shared memory
+
+// Constants for the plaintext-modulus transforms (32-bit arithmetic).
+struct PlainTab {
+  u32 t, twot;
+  u32 ninv, ninv_sh;   // N^-1 mod t with 32-bit Shoup companion
+  u32 half;            // (t-1)/2
+  const uint2* W;      // [N] psi_t^brv(i) as {w, floor(w 2^32 / t)}
+  const uint2* IW;     // [N] inverses
+};
+
+// Constants of the exact scale-and-round (mixed-radix conversion).
+struct RoundTab {
+  const ulonglong2* ginv;  // [L*L]: entry i*L+j (j < i) = q_j^-1 mod q_i with Shoup companion
+  const u64* prefix_mod_t; // [L]: prod_{j<i} q_j mod t
+  u64 t, t_sh;             // t and floor(2^64 / t)
+  u64 half_mod_t;          // (q-1)/2 mod t
+  u64 qinv_mod_t;          // q^-1 mod t
+};
+
+// Everything a kernel needs, passed by value.
+struct DevView {
+  const LimbTab* limbs;
+  const GaussTab* gauss;
+  PlainTab plain;
+  RoundTab round;
+  u64 seed;
+  u32 logn, n, L, K;
+  u64* s_mont;   // [K][L][N]  NTT(s_k) * N^-1 in Montgomery form
+  u64* pk_mont;  // [2][L][N]  NTT(p_0), NTT(p_1) * N^-1 in Montgomery form
+  u64* pk_coef;  // [2][L][N]  (p_0, p_1), coefficient domain
+  u32* range_flag;
+};
+
+namespace d2mhe_launch {
+cudaError_t keygen(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 n_parties);
+cudaError_t collective_pk(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 n_parties,
+                          u64* shares_out);
+cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain);
+cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values);
+cudaError_t encrypt(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 n_parties,
+                    u32 ct_first, u32 n_cts, const u32* plain, u64* ct);
+cudaError_t aggregate(const DevView& v, cudaStream_t s, const u64* ct, u32 n_cts,
+                      const u32* offsets_dev, const u32* rows_dev, u32 n_out, u64* agg);
+cudaError_t partial_decrypt(const DevView& v, cudaStream_t s, const u64* agg,
+                            const u32* recipients_dev, u32 n_rec, const u32* parties_dev,
+                            u32 n_parties, u32 ct_first, u32 n_cts, u64* shares);
+cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
+                    u32 n_shares, u32 n_cts, u32* plain);
+cudaError_t ntt(const DevView& v, cudaStream_t s, u64* polys, u32 batch, bool inverse);
+cudaError_t muladd(const DevView& v, cudaStream_t s, const u64* a, const u64* b, const u64* c,
+                   u64* d, u32 batch);
+// number of kernel launches the call above performed (for bookkeeping)
+}  // namespace d2mhe_launch

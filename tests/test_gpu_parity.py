@@ -1,0 +1,401 @@
+"""GPU parity: every output of the CUDA library against the CPU oracle, bit for bit,
+through the C ABI (via the thin ctypes binding)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2207_04604_b200 import workloads as wl
+
+from common import T, make_oracle, psi_t_for, small_moduli
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def d2():
+    from paper_2207_04604_b200 import build, d2mhe
+
+    build.build()
+    assert torch.cuda.is_available()
+    return d2mhe
+
+
+def _brv(n_bits):
+    n = 1 << n_bits
+    idx = np.arange(n)
+    out = np.zeros(n, dtype=np.int64)
+    for b in range(n_bits):
+        out |= ((idx >> b) & 1) << (n_bits - 1 - b)
+    return out
+
+
+# ----------------------------------------------------------------------------------
+# transforms and multiply-add
+# ----------------------------------------------------------------------------------
+
+
+@pytest.mark.parametrize("log2_n,bits,L,batch", [
+    (3, 30, 1, 2), (4, 36, 2, 3), (5, 54, 3, 2), (6, 60, 2, 5), (7, 50, 2, 2), (8, 54, 1, 3),
+    (9, 60, 2, 2), (10, 36, 3, 2), (11, 54, 2, 2), (12, 36, 3, 5), (12, 60, 4, 3),
+    (13, 54, 4, 3), (13, 60, 1, 7), (14, 54, 8, 2), (14, 60, 3, 3),
+])
+def test_ntt_forward_inverse_against_oracle(d2, log2_n, bits, L, batch):
+    moduli = wl.ntt_primes(bits, 1 << 17, L) if bits >= 50 else small_moduli(log2_n, bits, L)
+    ctx = d2.Context(log2_n, moduli, 2, seed=1)
+    o = make_oracle(log2_n, moduli, seed=1)
+    a = wl.random_polys(moduli, log2_n, batch, seed=log2_n)
+    # edge values
+    a[0, :, 0] = 0
+    a[0, :, 1] = np.array(moduli, dtype=np.uint64) - 1
+    psi = [ctx.get_root(l) for l in range(L)]
+    for l, p in enumerate(moduli):
+        assert pow(psi[l], 1 << log2_n, p) == p - 1
+    dev = d2.from_u64_numpy(a, ctx.device)
+    ctx.ntt_forward(dev, batch)
+    got = d2.to_u64_numpy(dev)
+    want = o.ntt(a, psi)  # natural order: value j = a(psi^(2j+1))
+    perm = _brv(log2_n)
+    assert np.array_equal(got, want[..., perm])  # position p holds value brv(p)
+    ctx.ntt_inverse(dev, batch)
+    ctx.sync()
+    assert np.array_equal(d2.to_u64_numpy(dev), a)
+    # inverse alone, from the oracle's transform
+    dev2 = d2.from_u64_numpy(np.ascontiguousarray(want[..., perm]), ctx.device)
+    ctx.ntt_inverse(dev2, batch)
+    assert np.array_equal(d2.to_u64_numpy(dev2), a)
+    ctx.close()
+
+
+@pytest.mark.parametrize("log2_n,bits,L,batch", [(4, 36, 2, 3), (12, 60, 4, 3), (13, 54, 3, 2), (16, 60, 2, 1)])
+def test_poly_muladd_against_oracle(d2, log2_n, bits, L, batch):
+    moduli = wl.ntt_primes(bits, 2 << log2_n, L)
+    ctx = d2.Context(log2_n, moduli, 2, seed=1)
+    o = make_oracle(log2_n, moduli, seed=1)
+    a, b, c = (wl.random_polys(moduli, log2_n, batch, seed=s) for s in (1, 2, 3))
+    a[0, :, :4] = np.array(moduli, dtype=np.uint64)[:, None] - 1
+    b[0, :, :2] = np.array(moduli, dtype=np.uint64)[:, None] - 1
+    c[0, :, 0] = np.array(moduli, dtype=np.uint64) - 1
+    da, db, dc = (d2.from_u64_numpy(x, ctx.device) for x in (a, b, c))
+    dd = torch.empty_like(da)
+    ctx.poly_muladd(da, db, dc, dd, batch)
+    ctx.sync()
+    assert np.array_equal(d2.to_u64_numpy(dd), o.poly_muladd(a, b, c))
+    ctx.poly_muladd(da, db, dc, da, batch)  # aliasing d = a
+    assert np.array_equal(d2.to_u64_numpy(da), o.poly_muladd(a, b, c))
+    ctx.close()
+
+
+def test_ring_product_through_transforms_equals_schoolbook(d2):
+    """INTT(NTT(a) . NTT(b)) = a*b in Z_p[X]/(X^N+1) for tiny N (definition by brute force)."""
+    from oracle import d2mhe_oracle as orc
+
+    for log2_n in (3, 4, 5, 6):
+        moduli = small_moduli(log2_n, 54, 2)
+        ctx = d2.Context(log2_n, moduli, 2, seed=1)
+        a, b = (wl.random_polys(moduli, log2_n, 1, seed=s) for s in (5, 6))
+        da, db = d2.from_u64_numpy(a, ctx.device), d2.from_u64_numpy(b, ctx.device)
+        zero = torch.zeros_like(da)
+        ctx.ntt_forward(da, 1)
+        ctx.ntt_forward(db, 1)
+        ctx.poly_muladd(da, db, zero, da, 1)
+        ctx.ntt_inverse(da, 1)
+        got = d2.to_u64_numpy(da)
+        for l, p in enumerate(moduli):
+            assert np.array_equal(got[0, l], orc.negacyclic_schoolbook(a[0, l], b[0, l], p))
+        ctx.close()
+
+
+# ----------------------------------------------------------------------------------
+# packing
+# ----------------------------------------------------------------------------------
+
+
+@pytest.mark.parametrize("log2_n", [4, 6, 9, 12, 13, 14, 15])
+def test_encode_decode_against_oracle(d2, log2_n):
+    moduli = wl.ntt_primes(54, 2 << log2_n, 1)
+    ctx = d2.Context(log2_n, moduli, 2, seed=1)
+    o = make_oracle(log2_n, moduli, seed=1)
+    assert ctx.get_plain_root() == psi_t_for(log2_n)
+    n = 1 << log2_n
+    rng = np.random.default_rng(log2_n)
+    half = (T - 1) // 2
+    vals = rng.integers(-half, half + 1, size=(3, n)).astype(np.int32)
+    vals[0, :3] = [half, -half, 0]
+    dv = torch.from_numpy(vals).to(ctx.device)
+    dp = ctx.empty_u32(3, n)
+    ctx.encode(dv, 3, dp)
+    ctx.sync()
+    want = o.encode(vals)
+    assert np.array_equal(d2.to_u32_numpy(dp), want)
+    back = torch.empty_like(dv)
+    ctx.decode(dp, 3, back)
+    assert np.array_equal(back.cpu().numpy(), vals)
+    # decode of arbitrary plaintext polynomials
+    m = rng.integers(0, T, size=(2, n)).astype(np.uint32)
+    dm = d2.from_u32_numpy(m, ctx.device)
+    out = torch.empty((2, n), dtype=torch.int32, device=ctx.device)
+    ctx.decode(dm, 2, out)
+    assert np.array_equal(out.cpu().numpy(), o.decode(m))
+    # in place
+    ctx.encode(dv, 3, dv)
+    assert np.array_equal(d2.to_u32_numpy(dv), want)
+    ctx.close()
+
+
+def test_encode_flags_out_of_range_values(d2):
+    ctx = d2.Context(12, wl.round_config(1).moduli, 2, seed=1)
+    vals = torch.zeros((1, 4096), dtype=torch.int32, device=ctx.device)
+    vals[0, 17] = (T - 1) // 2 + 1
+    out = ctx.empty_u32(1, 4096)
+    ctx.encode(vals, 1, out)
+    with pytest.raises(d2.D2mheError) as e:
+        ctx.sync()
+    assert e.value.status == d2.ERR_RANGE
+    ctx.sync()  # flag cleared
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------------
+# the protocol, step by step
+# ----------------------------------------------------------------------------------
+
+
+def _run_round(d2, ctx, o, cfg_k, parties, offsets, rows, values, ct_first):
+    """Runs every step on the GPU and on the oracle and compares all messages."""
+    n_cts = values.shape[1]
+    K = len(parties)
+    L, n = o.num_limbs, o.n
+    dev = ctx.device
+    # keys
+    ctx.keygen_share(parties)
+    pk = ctx.empty_u64(2, L, n)
+    pk_shares = ctx.empty_u64(K, L, n)
+    ctx.collective_pk(parties, pk_shares, pk)
+    ctx.sync()
+    for k in parties:
+        assert np.array_equal(ctx.debug_export_secret(k), o.secret_share(k))
+    want_pk = o.collective_pk(parties)
+    assert np.array_equal(d2.to_u64_numpy(pk), want_pk)
+    got_shares = d2.to_u64_numpy(pk_shares)
+    for a, k in enumerate(parties):
+        assert np.array_equal(got_shares[a], o.pk_share(k, want_pk[1]))
+    # encode + encrypt
+    dv = torch.from_numpy(values).to(dev)
+    plain = ctx.empty_u32(K, n_cts, n)
+    ctx.encode(dv, K * n_cts, plain)
+    want_plain = o.encode(values)
+    assert np.array_equal(d2.to_u32_numpy(plain), want_plain)
+    ct = ctx.empty_u64(K, n_cts, 2, L, n)
+    ctx.encrypt(parties, ct_first, n_cts, plain, ct)
+    want_ct = o.encrypt(want_pk, parties, ct_first, want_plain)
+    assert np.array_equal(d2.to_u64_numpy(ct), want_ct)
+    # aggregate
+    n_out = len(offsets) - 1
+    agg = ctx.empty_u64(n_out, n_cts, 2, L, n)
+    ctx.aggregate(ct, K, n_cts, offsets, rows, agg)
+    want_agg = o.aggregate(want_ct, offsets, rows)
+    assert np.array_equal(d2.to_u64_numpy(agg), want_agg)
+    # shares
+    recipients = [i % K for i in range(n_out)]
+    shares = ctx.empty_u64(n_out, K, n_cts, L, n)
+    ctx.partial_decrypt(agg, recipients, parties, ct_first, n_cts, shares)
+    want_shares = o.partial_decrypt(want_agg, recipients, parties, ct_first)
+    assert np.array_equal(d2.to_u64_numpy(shares), want_shares)
+    # combine + decode
+    out_plain = ctx.empty_u32(n_out, n_cts, n)
+    ctx.combine_decrypt(agg, shares, n_out, K, n_cts, out_plain)
+    want_out = o.combine(want_agg, want_shares)
+    assert np.array_equal(d2.to_u32_numpy(out_plain), want_out)
+    sums = torch.empty((n_out, n_cts, n), dtype=torch.int32, device=dev)
+    ctx.decode(out_plain, n_out * n_cts, sums)
+    ctx.sync()
+    got = sums.cpu().numpy()
+    assert np.array_equal(got, o.decode(want_out))
+    for i in range(n_out):
+        lst = rows[offsets[i]:offsets[i + 1]]
+        assert np.array_equal(got[i], values[lst].astype(np.int64).sum(axis=0))
+    return got
+
+
+@pytest.mark.parametrize("log2_n,bits,L,K", [(4, 30, 2, 3), (5, 36, 3, 4), (6, 54, 2, 2), (8, 60, 3, 3), (10, 54, 5, 3)])
+def test_small_rings_every_message(d2, log2_n, bits, L, K):
+    moduli = small_moduli(log2_n, bits, L)
+    seed = 77 + log2_n
+    ctx = d2.Context(log2_n, moduli, K, seed=seed)
+    o = make_oracle(log2_n, moduli, seed=seed)
+    parties = list(range(K))
+    rng = np.random.default_rng(log2_n)
+    values = rng.integers(-3000, 3001, size=(K, 3, 1 << log2_n)).astype(np.int32)
+    # irregular lists, one of them empty
+    offsets = np.array([0, K, K, K + 1], dtype=np.uint32)
+    rows = np.array(list(range(K)) + [K - 1], dtype=np.uint32)
+    _run_round(d2, ctx, o, K, parties, offsets, rows, values, ct_first=11)
+    ctx.close()
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_config1_every_message(d2, seed):
+    cfg = wl.round_config(1)
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, cfg.num_parties, seed=seed)
+    o = make_oracle(cfg.log2_n, cfg.moduli, seed=seed)
+    offsets, rows = wl.regular_graph(cfg.num_parties, cfg.degree, seed)
+    values = wl.gradients(cfg, seed)
+    _run_round(d2, ctx, o, cfg.num_parties, list(range(cfg.num_parties)), offsets, rows, values, 0)
+    ctx.close()
+
+
+def test_config2_every_message(d2):
+    cfg = wl.round_config(2)
+    seed = 1
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, cfg.num_parties, seed=seed)
+    o = make_oracle(cfg.log2_n, cfg.moduli, seed=seed)
+    offsets, rows = wl.regular_graph(cfg.num_parties, cfg.degree, seed)
+    values = wl.gradients(cfg, seed)
+    _run_round(d2, ctx, o, cfg.num_parties, list(range(cfg.num_parties)), offsets, rows, values, 0)
+    ctx.close()
+
+
+@pytest.mark.parametrize("index,sample", [(3, [0, 65]), (4, [341, 682])])
+def test_large_configs_on_sampled_ciphertext_indices(d2, index, sample):
+    """Configurations 3 and 4 at full K, N, L on two ciphertext indices each (the last one
+    holds the ragged, zero-padded tail): every message is addressable by its counters."""
+    cfg = wl.round_config(index)
+    seed = 1
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, cfg.num_parties, seed=seed)
+    o = make_oracle(cfg.log2_n, cfg.moduli, seed=seed)
+    offsets, rows = wl.regular_graph(cfg.num_parties, cfg.degree, seed)
+    parties = list(range(cfg.num_parties))
+    ctx.keygen_share(parties)
+    pk = ctx.empty_u64(2, cfg.num_limbs, cfg.n)
+    ctx.collective_pk(parties, None, pk)
+    want_pk = o.collective_pk(parties)
+    assert np.array_equal(d2.to_u64_numpy(pk), want_pk)
+    K, L, n = cfg.num_parties, cfg.num_limbs, cfg.n
+    for c in sample:
+        values = wl.gradients(cfg, seed, ct_first=c, n_cts=1)
+        dv = torch.from_numpy(values).to(ctx.device)
+        plain = ctx.empty_u32(K, 1, n)
+        ctx.encode(dv, K, plain)
+        ct = ctx.empty_u64(K, 1, 2, L, n)
+        ctx.encrypt(parties, c, 1, plain, ct)
+        agg = ctx.empty_u64(K, 1, 2, L, n)
+        ctx.aggregate(ct, K, 1, offsets, rows, agg)
+        # shares for three recipients only (each needs all K share holders)
+        rec = [0, K // 2, K - 1]
+        agg_sel = agg[rec].contiguous()
+        shares = ctx.empty_u64(len(rec), K, 1, L, n)
+        ctx.partial_decrypt(agg_sel, rec, parties, c, 1, shares)
+        out_plain = ctx.empty_u32(len(rec), 1, n)
+        ctx.combine_decrypt(agg_sel, shares, len(rec), K, 1, out_plain)
+        sums = torch.empty((len(rec), 1, n), dtype=torch.int32, device=ctx.device)
+        ctx.decode(out_plain, len(rec), sums)
+        ctx.sync()
+        want_plain = o.encode(values)
+        want_ct = o.encrypt(want_pk, parties, c, want_plain)
+        assert np.array_equal(d2.to_u64_numpy(ct), want_ct)
+        want_agg = o.aggregate(want_ct, offsets, rows)
+        assert np.array_equal(d2.to_u64_numpy(agg), want_agg)
+        want_shares = o.partial_decrypt(want_agg[rec], rec, parties, c)
+        assert np.array_equal(d2.to_u64_numpy(shares), want_shares)
+        want_out = o.combine(want_agg[rec], want_shares)
+        assert np.array_equal(d2.to_u32_numpy(out_plain), want_out)
+        got = sums.cpu().numpy()
+        for a, i in enumerate(rec):
+            lst = rows[offsets[i]:offsets[i + 1]]
+            assert np.array_equal(got[a], values[lst].astype(np.int64).sum(axis=0))
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------------
+# whole-round driver, chunking, determinism, error paths
+# ----------------------------------------------------------------------------------
+
+
+def test_round_driver_matches_stepwise_and_plain_sums(d2):
+    cfg = wl.round_config(2)
+    seed = 2
+    K, n, C = cfg.num_parties, cfg.n, cfg.num_cts
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, K, seed=seed)
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    offsets, rows = wl.regular_graph(K, cfg.degree, seed)
+    values = wl.gradients(cfg, seed)
+    want = np.stack([values[rows[offsets[i]:offsets[i + 1]]].astype(np.int64).sum(axis=0) for i in range(K)])
+    dv = torch.from_numpy(values).to(ctx.device)
+    for chunk in (1, 5, C):
+        ws = torch.empty(ctx.round_workspace_bytes(chunk), dtype=torch.uint8, device=ctx.device)
+        sums = torch.zeros((K, C, n), dtype=torch.int32, device=ctx.device)
+        ctx.round_device(dv, 0, C, offsets, rows, sums, ws)
+        ctx.sync()
+        assert np.array_equal(sums.cpu().numpy(), want)
+    # host variant, pinned buffers
+    hv = torch.from_numpy(values).pin_memory()
+    hs = torch.zeros((K, C, n), dtype=torch.int32).pin_memory()
+    ws = torch.empty(ctx.round_workspace_bytes(4), dtype=torch.uint8, device=ctx.device)
+    ctx.round_host(hv, 0, C, offsets, rows, hs, ws)
+    assert np.array_equal(hs.numpy(), want)
+    # too small a workspace is refused
+    tiny = torch.empty(1024, dtype=torch.uint8, device=ctx.device)
+    with pytest.raises(d2.D2mheError) as e:
+        ctx.round_device(dv, 0, C, offsets, rows, sums, tiny)
+    assert e.value.status == d2.ERR_WORKSPACE
+    ctx.close()
+
+
+def test_ciphertext_index_shards_reproduce_the_whole(d2):
+    """Index ranges are independent: two half-ranges equal the full range bit for bit
+    (this is how several GPUs split a round without exchanging data)."""
+    cfg = wl.round_config(1)
+    K, L, n = cfg.num_parties, cfg.num_limbs, cfg.n
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, K, seed=5)
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    plain = d2.from_u32_numpy(np.random.default_rng(1).integers(0, T, size=(K, 4, n)).astype(np.uint32), ctx.device)
+    whole = ctx.empty_u64(K, 4, 2, L, n)
+    ctx.encrypt(parties, 0, 4, plain, whole)
+    for first in (0, 2):
+        first_r, cnt = wl.shard_ct_range(first // 2, 2, 2)
+        part = ctx.empty_u64(K, 2, 2, L, n)
+        ctx.encrypt(parties, first_r, cnt, plain[:, first_r:first_r + cnt].contiguous(), part)
+        assert torch.equal(part, whole[:, first_r:first_r + cnt])
+    again = ctx.empty_u64(K, 4, 2, L, n)
+    ctx.encrypt(parties, 0, 4, plain, again)
+    assert torch.equal(again, whole)  # deterministic
+    ctx.close()
+
+
+def test_error_statuses(d2):
+    cfg = wl.round_config(1)
+    K, L, n = cfg.num_parties, cfg.num_limbs, cfg.n
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, K, seed=1)
+    plain = ctx.empty_u32(K, 1, n)
+    ct = ctx.empty_u64(K, 1, 2, L, n)
+
+    def status(fn, *a):
+        with pytest.raises(d2.D2mheError) as e:
+            fn(*a)
+        return e.value.status
+
+    assert status(ctx.encrypt, [0, 1, 2, 3], 0, 1, plain, ct) == d2.ERR_STATE  # no pk yet
+    assert status(ctx.collective_pk, [0, 1]) == d2.ERR_STATE  # no key shares yet
+    assert status(ctx.keygen_share, [0, K]) == d2.ERR_RANGE
+    assert status(ctx.keygen_share, [0, 0]) == d2.ERR_INVALID_ARG
+    ctx.keygen_share([0, 1, 2])
+    assert status(ctx.collective_pk, [0, 1, 2, 3]) == d2.ERR_STATE  # party 3 has no share
+    ctx.collective_pk([0, 1, 2])
+    agg = ctx.empty_u64(1, 1, 2, L, n)
+    assert status(ctx.aggregate, ct, K, 1, [0, 2], [0, K], agg) == d2.ERR_RANGE
+    assert status(ctx.aggregate, ct, K, 1, [1, 2], [0, 1], agg) == d2.ERR_INVALID_ARG
+    shares = ctx.empty_u64(1, 3, 1, L, n)
+    assert status(ctx.partial_decrypt, agg, [0], [0, 1, 3], 0, 1, shares) == d2.ERR_STATE
+    out = ctx.empty_u32(1, 1, n)
+    assert status(ctx.combine_decrypt, agg, shares, 1, 2, 1, out) == d2.ERR_INVALID_ARG  # a share is missing
+    misaligned = ctx.empty_u64(2 * L * n + 1)[1:]
+    assert status(ctx.ntt_forward, misaligned, 1) == d2.ERR_INVALID_ARG
+    ctx.sync()
+    big = d2.Context(15, wl.ntt_primes(54, 1 << 16, 1), 2, seed=1)
+    assert status(big.keygen_share, [0]) == d2.ERR_UNSUPPORTED
+    big.close()
+    ctx.close()

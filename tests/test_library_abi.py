@@ -1,0 +1,61 @@
+"""No GPU needed: the shared library loads and exports every symbol the header declares."""
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "d2mhe.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(d2mhe_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported():
+    from paper_2207_04604_b200 import build, d2mhe
+
+    build.build()
+    lib = d2mhe.load()
+    names = _declared_symbols()
+    assert len(names) >= 20
+    for name in names:
+        assert hasattr(lib, name), name
+    assert sorted(d2mhe.EXPORTS) == names
+
+
+def test_strerror_needs_no_device():
+    from paper_2207_04604_b200 import d2mhe
+
+    assert d2mhe.strerror(0) == "success"
+    assert "range" in d2mhe.strerror(d2mhe.ERR_RANGE)
+    assert d2mhe.strerror(-99) == "unknown status"
+
+
+def test_create_rejects_bad_arguments_before_touching_the_device():
+    import ctypes
+
+    from paper_2207_04604_b200 import d2mhe
+
+    lib = d2mhe.load()
+    h = ctypes.c_void_p()
+    assert lib.d2mhe_create(None, ctypes.byref(h)) == d2mhe.ERR_INVALID_ARG
+    p = d2mhe.Params()
+    p.struct_size = 4
+    assert lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h)) == d2mhe.ERR_INVALID_ARG
+    mods = (ctypes.c_uint64 * 2)(0xFFFFEE001, 0xFFFFEE001)
+    p.struct_size = ctypes.sizeof(d2mhe.Params)
+    p.log2_n, p.num_limbs, p.num_parties = 12, 2, 4
+    p.moduli = ctypes.cast(mods, ctypes.POINTER(ctypes.c_uint64))
+    p.plain_modulus, p.seed, p.gauss_bound, p.flags, p.device = 65537, 1, 19, 0, 0
+    assert lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h)) == d2mhe.ERR_BAD_PARAMS  # repeated prime
+    mods[1] = 0xFFFFEE003  # not 1 mod 2N
+    assert lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h)) == d2mhe.ERR_BAD_PARAMS
+    mods[1] = 0xFFFFC4001
+    p.gauss_bound = 20
+    assert lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h)) == d2mhe.ERR_BAD_PARAMS
+    p.gauss_bound = 19
+    p.plain_modulus = 65536
+    assert lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h)) == d2mhe.ERR_BAD_PARAMS
+    assert not h.value
