@@ -1,0 +1,428 @@
+#!/usr/bin/env python
+"""Benchmark of the D2-MHE private gradient update on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic gradients:
+encode -> encrypt -> neighbour sums -> decryption shares -> combine (scale-and-round) -> decode,
+with every protocol message (ciphertexts, aggregates, shares) written to and read from HBM.
+Metric: gradient coefficients per second per full round = K * params / t_round.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same configuration on its
+own range of ciphertext indices; nothing is exchanged inside a round (weak scaling).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2207_04604_b200 import workloads as wl  # noqa: E402
+
+METRIC = "gradient coefficients/sec per full MHE round (enc+agg+dec); NTT GB/s vs HBM peak"
+UNIT = "coeff/s"
+STEP_CALLS = ["encode", "encrypt", "aggregate", "partial_decrypt", "combine_decrypt", "decode"]
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.rows = []
+        self.proc = None
+        self.device_index = device_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.device_index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(cfg, n_cts):
+    """Protocol bytes per call for n_cts ciphertext indices of all K users (S = K share holders)."""
+    K, S, A = cfg.num_parties, cfg.num_parties, cfg.degree + 1
+    P = 8 * cfg.n * cfg.num_limbs
+    units = K * n_cts
+    return {
+        "encode": units * cfg.n * 8,
+        "encrypt": units * (4 * cfg.n + 2 * P),
+        "aggregate": units * (A * 2 * P + 2 * P),
+        "partial_decrypt": units * (P + S * P),
+        "combine_decrypt": units * (P + S * P + 4 * cfg.n),
+        "decode": units * cfg.n * 8,
+    }
+
+
+# ----------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands
+# ----------------------------------------------------------------------------------
+
+
+def oracle_round(cfg, seed, ct_first, n_cts, o=None, pk=None):
+    from oracle import d2mhe_oracle as orc
+
+    if o is None:
+        psi_t = pow(3, (wl.PLAIN_MODULUS - 1) // (2 * cfg.n), wl.PLAIN_MODULUS)
+        o = orc.Oracle(cfg.log2_n, cfg.moduli, wl.PLAIN_MODULUS, seed, psi_t=psi_t)
+    K = cfg.num_parties
+    parties = list(range(K))
+    if pk is None:
+        pk = o.collective_pk(parties)
+    offsets, rows = wl.regular_graph(K, cfg.degree, seed)
+    values = wl.gradients(cfg, seed, ct_first, n_cts)
+    t0 = time.perf_counter()
+    ct = o.encrypt(pk, parties, ct_first, o.encode(values))
+    agg = o.aggregate(ct, offsets, rows)
+    shares = o.partial_decrypt(agg, parties, parties, ct_first)
+    sums = o.decode(o.combine(agg, shares))
+    dt = time.perf_counter() - t0
+    return dt, sums, values, offsets, rows, o, pk
+
+
+def cpu_baseline(cfg, seed, budget_s=12.0):
+    """Times the oracle on as many ciphertext indices of the workload as fit the budget."""
+    from oracle import d2mhe_oracle as orc
+
+    dt1, _, _, _, _, o, pk = oracle_round(cfg, seed, 0, 1)
+    n_cts = int(max(1, min(cfg.num_cts, budget_s / max(dt1, 1e-6))))
+    dt, sums, values, offsets, rows, _, _ = oracle_round(cfg, seed, 0, n_cts, o, pk)
+    coeffs = cfg.num_parties * min(cfg.params, n_cts * cfg.n)
+    return {"value": coeffs / dt, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
+            "sample": "ciphertext indices 0..%d of %d, all %d users and share holders, %.2f s"
+                      % (n_cts - 1, cfg.num_cts, cfg.num_parties, dt)}
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import d2mhe_oracle as orc
+
+    dt1, _, _, _, _, o, pk = oracle_round(cfg, args.seed, 0, 1)
+    per_step_budget = 120.0 / max(1, args.steps + args.warmup)
+    n_cts = int(max(1, min(cfg.num_cts, per_step_budget / max(dt1, 1e-6))))
+    for _ in range(args.warmup):
+        oracle_round(cfg, args.seed, 0, n_cts, o, pk)
+    total = 0.0
+    for _ in range(args.steps):
+        dt, *_ = oracle_round(cfg, args.seed, 0, n_cts, o, pk)
+        total += dt
+    coeffs = cfg.num_parties * min(cfg.params, n_cts * cfg.n)
+    value = coeffs * args.steps / total
+    sample = "each step: ciphertext indices 0..%d of %d, all %d users and share holders" % (
+        n_cts - 1, cfg.num_cts, cfg.num_parties)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+        "config": {"workload": cfg.name, "K": cfg.num_parties, "N": cfg.n, "L": cfg.num_limbs,
+                   "cts_per_user": cfg.num_cts, "params_per_user": cfg.params},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------
+# the CUDA arm
+# ----------------------------------------------------------------------------------
+
+
+def run_cuda(args, cfg):
+    import torch
+
+    from paper_2207_04604_b200 import build, d2mhe, parallel
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    rank, local_rank, world = parallel.init()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if rank == 0:
+        build.build()
+    parallel.barrier(dev)
+
+    K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, cfg.num_cts
+    parties = list(range(K))
+    offsets, rows = wl.regular_graph(K, cfg.degree, args.seed)
+    ct_first, _ = wl.shard_ct_range(rank, world, C)  # each rank: its own C ciphertext indices
+    ctx = d2mhe.Context(cfg.log2_n, cfg.moduli, K, seed=args.seed, device=local_rank)
+    stream = torch.cuda.current_stream(dev)
+
+    # Initialization (reported separately, as the paper does): key shares and the collective key.
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    ev1.record(stream)
+    ctx.sync()
+    init_ms = ev0.elapsed_time(ev1)
+
+    # chunking: keep all protocol messages of a chunk in HBM at once
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    per_ct = ctx.round_workspace_bytes(1) - 256
+    chunk = int(max(1, min(C, (int(free_b * 0.4)) // per_ct)))
+    if args.chunk:
+        chunk = min(chunk, args.chunk)
+    values_np = wl.gradients(cfg, args.seed, ct_first, C)
+    values = torch.from_numpy(values_np).to(dev)
+
+    def alloc(cc):
+        return (torch.empty((K, cc, n), dtype=torch.int32, device=dev), ctx.empty_u32(K, cc, n),
+                ctx.empty_u64(K, cc, 2, L, n), ctx.empty_u64(K, cc, 2, L, n), ctx.empty_u64(K, K, cc, L, n),
+                ctx.empty_u32(K, cc, n), torch.empty((K, cc, n), dtype=torch.int32, device=dev))
+
+    bufs = {chunk: alloc(chunk)}
+    if C % chunk:
+        bufs[C % chunk] = alloc(C % chunk)  # the ragged last chunk has buffers of its own size
+    sums = torch.empty((K, C, n), dtype=torch.int32, device=dev)
+    flush = torch.empty(384 * 1024 * 1024, dtype=torch.uint8, device=dev)  # > 126 MB L2
+
+    def step(events=None):
+        """One full round over all C ciphertext indices, chunk by chunk."""
+        for first in range(0, C, chunk):
+            cc = min(chunk, C - first)
+            v, p, c_, a, s, o_, r = bufs[cc]
+            v.copy_(values[:, first:first + cc])
+            marks = []
+
+            def mark():
+                if events is not None:
+                    e = torch.cuda.Event(enable_timing=True)
+                    e.record(stream)
+                    marks.append(e)
+
+            mark()
+            ctx.encode(v, K * cc, p)
+            mark()
+            ctx.encrypt(parties, ct_first + first, cc, p, c_)
+            mark()
+            ctx.aggregate(c_, K, cc, offsets, rows, a)
+            mark()
+            ctx.partial_decrypt(a, parties, parties, ct_first + first, cc, s)
+            mark()
+            ctx.combine_decrypt(a, s, K, K, cc, o_)
+            mark()
+            ctx.decode(o_, K * cc, r)
+            mark()
+            sums[:, first:first + cc].copy_(r)
+            if events is not None:
+                events.append(marks)
+
+    def barrier():
+        parallel.barrier(dev)
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    barrier()
+
+    # correctness of what is being timed: every decrypted sum equals the plaintext neighbour sum
+    want = np.stack([values_np[rows[offsets[i]:offsets[i + 1]]].astype(np.int64).sum(axis=0) for i in range(K)])
+    if not np.array_equal(sums.cpu().numpy(), want):
+        raise RuntimeError("decrypted neighbour sums differ from the plaintext sums")
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count()
+    step_events, chunk_events = [], []
+    barrier()
+    wall0 = time.perf_counter()
+    for _ in range(args.steps):
+        flush.zero_()  # evict the previous step's messages from L2 (outside the timed events)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        step(chunk_events)
+        e1.record(stream)
+        step_events.append((e0, e1))
+    barrier()
+    wall = time.perf_counter() - wall0
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+
+    step_ms = sum(a.elapsed_time(b) for a, b in step_events) / args.steps
+    per_call = {name: 0.0 for name in STEP_CALLS}
+    for marks in chunk_events:
+        for i, name in enumerate(STEP_CALLS):
+            per_call[name] += marks[i].elapsed_time(marks[i + 1])
+    n_chunks_total = len(chunk_events)
+    step_ms_max = parallel.max_over_ranks(step_ms, dev)
+    coeffs_per_step = world * K * cfg.params
+    value = coeffs_per_step / (step_ms_max * 1e-3)
+
+    # end to end through the host-buffer entry point: H2D of the gradients, the round, D2H of the sums
+    hv = torch.from_numpy(values_np).pin_memory()
+    hs = torch.zeros((K, C, n), dtype=torch.int32).pin_memory()
+    bufs.clear()
+    torch.cuda.empty_cache()
+    ws = torch.empty(ctx.round_workspace_bytes(chunk), dtype=torch.uint8, device=dev)
+    for _ in range(2):
+        ctx.round_host(hv, ct_first, C, offsets, rows, hs, ws)
+    if not np.array_equal(hs.numpy(), want):
+        raise RuntimeError("host-buffer round differs from the plaintext sums")
+    e2e_steps = max(3, min(args.steps, 10))
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        flush.zero_()
+        ctx.round_host(hv, ct_first, C, offsets, rows, hs, ws)
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+    e2e_ms_max = parallel.max_over_ranks(e2e_ms, dev)
+    e2e_value = coeffs_per_step / (e2e_ms_max * 1e-3)
+
+    # transform / multiply-add micro-benchmark on this configuration's ring (batch > L2)
+    ntt = None
+    if rank == 0:
+        del ws
+        torch.cuda.empty_cache()
+        batch = max(1, (384 << 20) // (8 * n * L))
+        polys = torch.randint(0, min(cfg.moduli), (batch, L, n), dtype=torch.int64, device=dev)
+        other = polys.clone()
+        third = polys.clone()
+        res = torch.empty_like(polys)
+
+        def timed(fn, reps=5):
+            fn()
+            best = None
+            for _ in range(reps):
+                flush.zero_()
+                a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a_.record(stream)
+                fn()
+                b_.record(stream)
+                torch.cuda.synchronize(dev)
+                ms = a_.elapsed_time(b_)
+                best = ms if best is None else min(best, ms)
+            return best
+
+        nbytes = 16.0 * n * L * batch
+        f_ms = timed(lambda: ctx.ntt_forward(polys, batch))
+        i_ms = timed(lambda: ctx.ntt_inverse(polys, batch))
+        m_ms = timed(lambda: ctx.poly_muladd(polys, other, third, res, batch))
+        ntt = {"shape": [batch, L, n], "forward_GBps": nbytes / 1e9 / (f_ms * 1e-3),
+               "inverse_GBps": nbytes / 1e9 / (i_ms * 1e-3), "muladd_GBps": 2 * nbytes / 1e9 / (m_ms * 1e-3),
+               "bytes_per_coeff": {"ntt": 16, "muladd": 32}}
+        del polys, other, third, res
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        ab = algorithmic_bytes(cfg, C)
+        for k_ in ("forward_GBps", "inverse_GBps", "muladd_GBps"):
+            ntt[k_.replace("GBps", "frac_of_hbm")] = ntt[k_] / peak
+        total_ms = sum(per_call.values())
+        kernels = {}
+        for name in STEP_CALLS:
+            ms = per_call[name] / args.steps  # per step, summed over chunks
+            kernels[name] = {"ms_per_step": ms, "share": per_call[name] / total_ms if total_ms else None,
+                             "algorithmic_GB": ab[name] / 1e9, "GBps": ab[name] / 1e9 / (ms * 1e-3) if ms else None}
+        dominant = max(STEP_CALLS, key=lambda k_: per_call[k_])
+        launches_dom = n_chunks_total
+        dur_ms = per_call[dominant] / launches_dom
+        bytes_per_launch = ab[dominant] / (n_chunks_total / args.steps)
+        achieved = bytes_per_launch / 1e9 / (dur_ms * 1e-3)
+        roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": None,
+                    "avg_launch_ms": dur_ms}
+        round_bytes = sum(ab.values())
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": step_ms_max, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": cfg.name, "K": K, "N": n, "L": L, "cts_per_user": C, "params_per_user": cfg.params,
+                       "graph_degree": cfg.degree, "share_holders": K, "chunk_cts": chunk,
+                       "l2": "384 MB buffer written between timed steps (L2 flush)",
+                       "parallelism": "ciphertext-index shards, no exchange" if world > 1 else "single GPU"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": K * C * n * 4,
+                    "d2h_bytes_per_step": K * C * n * 4, "ms_per_step": e2e_ms_max},
+            "gpu_launches": int(launches),
+            "roofline": roofline,
+            "round_hbm_frac": round_bytes / 1e9 / (step_ms_max * 1e-3) / peak,
+            "kernels": kernels,
+            "ntt": ntt,
+            "init_ms": init_ms,
+            "wall_ms_per_step_incl_flush": wall * 1e3 / args.steps,
+            "cpu_baseline": cpu_baseline(cfg, args.seed) if world == 1 and not args.no_cpu_baseline else None,
+        }
+        print(json.dumps(line))
+    ctx.close()
+    parallel.finish()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="round configuration 1..4 (default: MNIST-shaped)")
+    ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--chunk", type=int, default=0, help="ciphertext indices per chunk (0: as many as fit)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = wl.round_config(args.config)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_cuda(args, cfg)
+
+
+if __name__ == "__main__":
+    main()
