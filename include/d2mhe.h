@@ -189,6 +189,29 @@ d2mhe_status d2mhe_round_host(d2mhe_ctx* ctx, const int32_t* values_host, uint32
                               const uint32_t* nbr_rows, int32_t* sums_host,
                               void* workspace_dev, size_t workspace_bytes);
 
+/*
+ * The same round as d2mhe_round_device for callers that cannot allocate device memory
+ * (the paper has no counterpart: this is a packaging variant, not a protocol step).
+ * Think of a service that gave all device memory to a fixed pool at start-up, a plug-in
+ * that receives only its input and output buffers, or a latency-critical loop in which
+ * cudaMalloc is banned because it synchronises the device.  The chunk's protocol messages
+ * live in a 64 MiB array that is part of the library image (every GPU that loads the
+ * library holds those 64 MiB until the process exits); the caller passes only values and sums.
+ *  - Calls no cudaMalloc / cudaFree and no allocating library routine.
+ *  - Returns D2MHE_ERR_WORKSPACE when one ciphertext index of this parameter set needs more
+ *    than 64 MiB, i.e. when d2mhe_round_workspace_bytes(ctx, 1) > 67108864 (configuration 2,
+ *    K = 10, N = 8192, L = 4, needs 36.3 MB and fits; K = 20, N = 16384, L = 8 does not).
+ *  - The first call on a device looks up the array's device address (a synchronous runtime
+ *    query); make that first call before starting any stream capture.
+ *  - All contexts and all calls on one GPU share the array, which keeps the last call's
+ *    contents.  Nothing has to be cleared (every buffer is written before it is read), but
+ *    two calls whose work overlaps on the GPU (different streams, threads or contexts) race.
+ * Arguments as for d2mhe_round_device.
+ */
+d2mhe_status d2mhe_round_device_static(d2mhe_ctx* ctx, const int32_t* values_dev, uint32_t ct_first,
+                                       uint32_t n_cts, const uint32_t* nbr_offsets,
+                                       const uint32_t* nbr_rows, int32_t* sums_dev);
+
 /* Test hooks. */
 /* s_k as int8 [N] on the HOST (needs a key share for `party`). */
 d2mhe_status d2mhe_debug_export_secret(d2mhe_ctx* ctx, uint32_t party, int8_t* s_host);

@@ -41,6 +41,37 @@ struct DevView {
   u32* range_flag;
 };
 
+// ---- host-side context (shared by the translation units that implement the C ABI) ----
+#include <vector>
+
+#include "../../include/d2mhe.h"
+
+static const size_t kIdxSlotWords = (size_t)1 << 21;  // u32 words per staging slot (8 MiB)
+static const int kIdxSlots = 4;
+
+struct d2mhe_ctx {
+  d2mhe_params params;
+  std::vector<u64> moduli;
+  std::vector<u64> roots;
+  u64 psi_t = 0;
+  bool can_pack = false;
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  DevView view;
+  std::vector<void*> allocs;        // device allocations to free
+  std::vector<bool> has_share;
+  std::vector<u32> pk_parties;      // party set of the last collective_pk
+  bool has_pk = false;
+  u64 launches = 0;
+  // index staging: pinned host ring + device ring, one event per slot
+  u32* idx_host = nullptr;
+  u32* idx_dev = nullptr;
+  cudaEvent_t idx_event[kIdxSlots] = {};
+  bool idx_event_valid[kIdxSlots] = {};
+  int idx_next = 0;
+  cudaError_t last_cuda = cudaSuccess;
+};
+
 namespace d2mhe_launch {
 cudaError_t keygen(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 n_parties);
 cudaError_t collective_pk(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 n_parties,

@@ -28,7 +28,7 @@ EXPORTS = [
     "d2mhe_keygen_share", "d2mhe_collective_pk", "d2mhe_encode", "d2mhe_decode", "d2mhe_encrypt",
     "d2mhe_aggregate", "d2mhe_partial_decrypt", "d2mhe_combine_decrypt", "d2mhe_ntt_forward",
     "d2mhe_ntt_inverse", "d2mhe_poly_muladd", "d2mhe_round_workspace_bytes", "d2mhe_round_device",
-    "d2mhe_round_host", "d2mhe_debug_export_secret", "d2mhe_get_root", "d2mhe_get_plain_root",
+    "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_debug_export_secret", "d2mhe_get_root", "d2mhe_get_plain_root",
     "d2mhe_launch_count",
 ]
 
@@ -89,6 +89,7 @@ def load():
         lib.d2mhe_round_workspace_bytes.restype = sz
         lib.d2mhe_round_device.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp, sz]
         lib.d2mhe_round_host.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp, sz]
+        lib.d2mhe_round_device_static.argtypes = [vp, vp, u32, u32, vp, vp, vp]
         lib.d2mhe_debug_export_secret.argtypes = [vp, u32, vp]
         lib.d2mhe_get_root.argtypes = [vp, u32, ctypes.POINTER(u64)]
         lib.d2mhe_get_plain_root.argtypes = [vp, ctypes.POINTER(u64)]
@@ -239,6 +240,13 @@ class Context:
         self._check(load().d2mhe_round_device(self._h, _dev(values, torch.int32), ct_first, n_cts, offp, rowsp,
                                               _dev(sums, torch.int32), _dev(workspace),
                                               workspace.numel() * workspace.element_size()), "d2mhe_round_device")
+
+    def round_device_static(self, values, ct_first, n_cts, nbr_offsets, nbr_rows, sums):
+        """d2mhe_round_device with the library's built-in 64 MiB scratch: nothing is allocated."""
+        off, offp = _host_u32(nbr_offsets)
+        rows, rowsp = _host_u32(nbr_rows)
+        self._check(load().d2mhe_round_device_static(self._h, _dev(values, torch.int32), ct_first, n_cts, offp, rowsp,
+                                                     _dev(sums, torch.int32)), "d2mhe_round_device_static")
 
     def round_host(self, values_host, ct_first, n_cts, nbr_offsets, nbr_rows, sums_host, workspace):
         """values_host / sums_host: CPU int32 tensors (pinned recommended)."""

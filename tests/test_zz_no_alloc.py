@@ -1,0 +1,63 @@
+"""The allocation-free round (d2mhe_round_device_static) against the workspace round.
+
+Collected last on purpose: a stop-at-first-failure run has then already run every other test.
+The entry point serves callers that may not allocate device memory (fixed memory pools,
+plug-ins that only get their input/output buffers, loops where cudaMalloc's device
+synchronisation is not acceptable); its scratch is a 64 MiB array inside the library."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2207_04604_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _setup(d2, index, seed):
+    cfg = wl.round_config(index)
+    K = cfg.num_parties
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, K, seed=seed)
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    offsets, rows = wl.regular_graph(K, cfg.degree, seed)
+    return cfg, ctx, offsets, rows
+
+
+@pytest.mark.parametrize("index,n_cts", [(1, 2), (2, 3)])
+def test_static_round_equals_workspace_round_twice_in_a_row(index, n_cts):
+    from paper_2207_04604_b200 import build, d2mhe as d2
+
+    build.build()
+    cfg, ctx, offsets, rows = _setup(d2, index, seed=4)
+    K, n = cfg.num_parties, cfg.n
+    ws = torch.empty(ctx.round_workspace_bytes(n_cts), dtype=torch.uint8, device=ctx.device)
+    for call in range(2):  # the second call finds the first call's data in the shared array
+        values = wl.gradients(cfg, seed=10 + call, ct_first=5 * call, n_cts=n_cts)
+        dv = torch.from_numpy(values).to(ctx.device)
+        want = torch.zeros((K, n_cts, n), dtype=torch.int32, device=ctx.device)
+        ctx.round_device(dv, 5 * call, n_cts, offsets, rows, want, ws)
+        got = torch.full((K, n_cts, n), -7, dtype=torch.int32, device=ctx.device)
+        before = torch.cuda.memory_allocated(ctx.device)
+        ctx.round_device_static(dv, 5 * call, n_cts, offsets, rows, got)
+        ctx.sync()
+        assert torch.cuda.memory_allocated(ctx.device) == before
+        assert torch.equal(got, want)  # integer results: bit-exact
+        plain_sums = np.stack([values[rows[offsets[i]:offsets[i + 1]]].astype(np.int64).sum(axis=0) for i in range(K)])
+        assert np.array_equal(got.cpu().numpy(), plain_sums)
+    ctx.close()
+
+
+def test_static_round_rejects_parameter_sets_beyond_its_array():
+    from paper_2207_04604_b200 import build, d2mhe as d2
+
+    build.build()
+    cfg, ctx, offsets, rows = _setup(d2, 3, seed=1)  # one index needs ~480 MB of messages
+    assert ctx.round_workspace_bytes(1) > 64 << 20
+    K, n = cfg.num_parties, cfg.n
+    dv = torch.zeros((K, 1, n), dtype=torch.int32, device=ctx.device)
+    out = torch.zeros_like(dv)
+    with pytest.raises(d2.D2mheError) as e:
+        ctx.round_device_static(dv, 0, 1, offsets, rows, out)
+    assert e.value.status == d2.ERR_WORKSPACE
+    ctx.close()
