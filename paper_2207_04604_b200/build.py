@@ -7,7 +7,8 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libd2mhe.so")
-SOURCES = ["d2mhe_kernels.cu", "d2mhe_host.cu", "d2mhe_round_static.cu"]
+SOURCES = ["kern_pdec.cu", "kern_encrypt.cu", "kern_ntt.cu", "kern_keys.cu", "kern_stream.cu", "d2mhe_host.cu",
+           "d2mhe_round_static.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--extended-lambda", "-Xcompiler", "-fPIC",
@@ -31,14 +32,14 @@ def _stale():
     return any(os.path.getmtime(d) > built for d in deps if os.path.isfile(d))
 
 
-def build(force=False, verbose=False):
+def build(force=False, verbose=False, defines=()):
     """Compile every .cu for sm_100a and link the shared library next to this file."""
     if not force and not _stale():
         return LIB
     obj_dir = os.path.join(HERE, "_build")
     os.makedirs(obj_dir, exist_ok=True)
     nvcc = _nvcc()
-    extra = ["-Xptxas", "-v"] if verbose else []
+    extra = (["-Xptxas", "-v"] if verbose else []) + ["-D" + d for d in defines]
 
     def compile_one(src):
         obj = os.path.join(obj_dir, src.replace(".cu", ".o"))
@@ -61,4 +62,5 @@ def build(force=False, verbose=False):
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv,
+                defines=[a[2:] for a in sys.argv if a.startswith("-D")]))

@@ -13,6 +13,7 @@ typedef unsigned int u32;
 struct LimbTab {
   u64 p;             // q_l
   u64 twop;          // 2 q_l
+  u64 np;            // -q_l mod 2^64
   u64 pinv;          // q_l^-1 mod 2^64 (Montgomery)
   u64 one_sh;        // floor(2^64 / q_l): Shoup companion of 1, reduces any 64-bit value
   u64 ninv, ninv_sh; // N^-1 mod q_l with Shoup companion
@@ -61,9 +62,6 @@ __host__ __device__ __forceinline__ u64 lift_small(int v, u64 p) {
 // ---------------------------------------------------------------------------
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) and the samplers
 // ---------------------------------------------------------------------------
-struct Philox {
-  u32 k0, k1;
-};
 __host__ __device__ __forceinline__ void philox4x32_10(u32 k0, u32 k1, u32 c0, u32 c1, u32 c2,
                                                         u32 c3, u32& o0, u32& o1, u32& o2,
                                                         u32& o3) {
@@ -163,131 +161,246 @@ __host__ __device__ __forceinline__ u64 uniform_mod(const Stream& s, u32 j, u64 
 // 16 threads of a half warp hit 16 distinct 8-byte banks for every stride (.., 64, 8, 1).
 __device__ __forceinline__ u32 swz(u32 a) { return a ^ ((a >> 4) & 7u) ^ (((a >> 6) & 1u) << 3); }
 
-__device__ __forceinline__ void ct_bfly(u64& X, u64& Y, const ulonglong2 w, u64 p, u64 twop) {
-  u64 x = csub(X, twop);
-  u64 t = shoup_lazy(Y, w.x, w.y, p);
-  X = x + t;
-  Y = x - t + twop;
+// --- multiplication by a constant with an approximate quotient -------------------------
+// Returns y*w - q*p (mod 2^64) with q = ah*bh + hi32(ah*bl) + hi32(al*bh) for a = y,
+// b = ws = floor(w 2^64 / p): q is the true floor(y ws / 2^64) or up to 2 below it, so the
+// result is congruent to y*w and lies in [0, 4p) for ANY 64-bit y.  Five widening and four
+// 32-bit multiply-adds; no carry chains (the integer multiplier is the scarce pipe on B200).
+__device__ __forceinline__ u64 madwide(u32 a, u32 b, u64 c) {
+  u64 r;
+  asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "r"(b), "l"(c));
+  return r;
 }
-__device__ __forceinline__ void gs_bfly(u64& X, u64& Y, const ulonglong2 w, u64 p, u64 twop) {
-  u64 s = X + Y;
-  u64 d = X - Y + twop;
-  X = csub(s, twop);
-  Y = shoup_lazy(d, w.x, w.y, p);
+__device__ __forceinline__ u32 madlo(u32 a, u32 b, u32 c) {
+  u32 r;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+__device__ __forceinline__ u64 shoup_approx(u64 y, u64 w, u64 ws, u64 np) {
+  const u32 yl = (u32)y, yh = (u32)(y >> 32), sl = (u32)ws, sh = (u32)(ws >> 32);
+  const u64 t1 = (u64)yh * sl, t2 = (u64)yl * sh;
+  const u64 q = madwide(yh, sh, t1 >> 32) + (t2 >> 32);
+  const u32 ql = (u32)q, qh = (u32)(q >> 32), wl = (u32)w, wh = (u32)(w >> 32);
+  const u32 nl = (u32)np, nh = (u32)(np >> 32);
+  u64 r = madwide(ql, nl, (u64)yl * wl);
+  u32 rh = (u32)(r >> 32);
+  rh = madlo(yl, wh, rh);
+  rh = madlo(yh, wl, rh);
+  rh = madlo(ql, nh, rh);
+  rh = madlo(qh, nl, rh);
+  return ((u64)rh << 32) | (u32)r;
+}
+
+// Lazy-reduction policy.  WIDE (every prime below 2^57): values may grow across stages, so
+// the forward transform needs no conditional subtraction at all and the inverse reduces only
+// the one element per octet that accumulates the sums.  Otherwise (primes up to 2^61) values
+// are kept below 8p with one conditional subtraction per butterfly.
+struct Mod {
+  u64 p, np, twop, fourp;
+  const u64 one_sh;
+  __device__ __forceinline__ explicit Mod(const LimbTab& lt)
+      : p(lt.p), np(lt.np), twop(lt.twop), fourp(2 * lt.twop), one_sh(lt.one_sh) {}
+};
+
+// forward (Cooley-Tukey): (X, Y) -> (X + wY, X - wY)
+template <bool WIDE>
+__device__ __forceinline__ void ct_bfly(u64& X, u64& Y, const ulonglong2 w, const Mod& m) {
+  const u64 x = WIDE ? X : csub(X, m.fourp);
+  const u64 t = shoup_approx(Y, w.x, w.y, m.np);  // [0,4p)
+  X = x + t;
+  Y = x - t + m.fourp;
+}
+// inverse (Gentleman-Sande): (X, Y) -> (X + Y, w(X - Y)); c >= bound of Y, a multiple of p
+template <bool WIDE>
+__device__ __forceinline__ void gs_bfly(u64& X, u64& Y, const ulonglong2 w, const Mod& m, u64 c) {
+  const u64 s = X + Y;
+  const u64 d = X - Y + (WIDE ? c : m.fourp);
+  X = WIDE ? s : csub(s, m.fourp);
+  Y = shoup_approx(d, w.x, w.y, m.np);
 }
 
 // three (or fewer) forward stages on an octet; m = groups at the first stage, i = group index
+template <bool WIDE>
 __device__ __forceinline__ void fwd_octet(u64 (&x)[8], const ulonglong2* __restrict__ W, u32 m,
-                                          u32 i, int nst, u64 p, u64 twop) {
+                                          u32 i, int nst, const Mod& md) {
   {
     const ulonglong2 w = __ldg(W + m + i);
 #pragma unroll
-    for (int k = 0; k < 4; ++k) ct_bfly(x[k], x[k + 4], w, p, twop);
+    for (int k = 0; k < 4; ++k) ct_bfly<WIDE>(x[k], x[k + 4], w, md);
   }
   if (nst >= 2) {
     const ulonglong2 w0 = __ldg(W + 2 * m + 2 * i), w1 = __ldg(W + 2 * m + 2 * i + 1);
-    ct_bfly(x[0], x[2], w0, p, twop);
-    ct_bfly(x[1], x[3], w0, p, twop);
-    ct_bfly(x[4], x[6], w1, p, twop);
-    ct_bfly(x[5], x[7], w1, p, twop);
+    ct_bfly<WIDE>(x[0], x[2], w0, md);
+    ct_bfly<WIDE>(x[1], x[3], w0, md);
+    ct_bfly<WIDE>(x[4], x[6], w1, md);
+    ct_bfly<WIDE>(x[5], x[7], w1, md);
   }
   if (nst >= 3) {
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       const ulonglong2 w = __ldg(W + 4 * m + 4 * i + r);
-      ct_bfly(x[2 * r], x[2 * r + 1], w, p, twop);
+      ct_bfly<WIDE>(x[2 * r], x[2 * r + 1], w, md);
     }
   }
 }
+// Inverse stages on an octet whose inputs are all below 16p (WIDE) / 4p (otherwise).
+// WIDE bounds after the round: x0 < 128p, x1 < 16p, x2, x3 < 8p, x4..x7 < 4p; x0 is brought
+// back below 4p here, so every output is again below 16p.
+template <bool WIDE>
 __device__ __forceinline__ void inv_octet(u64 (&x)[8], const ulonglong2* __restrict__ IW, u32 m,
-                                          u32 i, int nst, u64 p, u64 twop) {
+                                          u32 i, int nst, const Mod& md) {
+  const u64 c16 = md.fourp << 2, c32 = md.fourp << 3, c64 = md.fourp << 4;
   if (nst >= 3) {
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       const ulonglong2 w = __ldg(IW + 4 * m + 4 * i + r);
-      gs_bfly(x[2 * r], x[2 * r + 1], w, p, twop);
+      gs_bfly<WIDE>(x[2 * r], x[2 * r + 1], w, md, c16);
     }
   }
   if (nst >= 2) {
     const ulonglong2 w0 = __ldg(IW + 2 * m + 2 * i), w1 = __ldg(IW + 2 * m + 2 * i + 1);
-    gs_bfly(x[0], x[2], w0, p, twop);
-    gs_bfly(x[1], x[3], w0, p, twop);
-    gs_bfly(x[4], x[6], w1, p, twop);
-    gs_bfly(x[5], x[7], w1, p, twop);
+    gs_bfly<WIDE>(x[0], x[2], w0, md, c32);
+    gs_bfly<WIDE>(x[1], x[3], w0, md, c32);
+    gs_bfly<WIDE>(x[4], x[6], w1, md, c32);
+    gs_bfly<WIDE>(x[5], x[7], w1, md, c32);
   }
   {
     const ulonglong2 w = __ldg(IW + m + i);
 #pragma unroll
-    for (int k = 0; k < 4; ++k) gs_bfly(x[k], x[k + 4], w, p, twop);
+    for (int k = 0; k < 4; ++k) gs_bfly<WIDE>(x[k], x[k + 4], w, md, c64);
   }
+  if (WIDE) x[0] = shoup_approx(x[0], 1, md.one_sh, md.np);
 }
 
-// Geometry shared by all kernels: LOGN > 0 fixes the size at compile time (strides and
-// loop counts fold to constants); LOGN == 0 takes it from the run-time argument.
+// Brings the outputs of the last inverse round below 4p.  After a full round the bounds are
+// those listed at inv_octet; a 2-stage round leaves x1 < 64p, x2, x3 < 8p and a 1-stage round
+// x1..x3 < 32p (x0 has already been reduced, x4..x7 are products).
+template <bool WIDE>
+__device__ __forceinline__ void finish_octet(u64 (&x)[8], int nst, const Mod& md) {
+  if (WIDE) {
+    if (nst >= 3) {
+      x[1] = csub(csub(x[1], md.fourp << 1), md.fourp);
+    } else {
+      x[1] = shoup_approx(x[1], 1, md.one_sh, md.np);
+    }
+    if (nst >= 2) {
+      x[2] = csub(x[2], md.fourp);
+      x[3] = csub(x[3], md.fourp);
+    } else {
+      x[2] = shoup_approx(x[2], 1, md.one_sh, md.np);
+      x[3] = shoup_approx(x[3], 1, md.one_sh, md.np);
+    }
+  }
+}
+// canonical representative of a value below 4p
+__device__ __forceinline__ u64 canon4(u64 v, const LimbTab& lt) { return csub(csub(v, lt.twop), lt.p); }
+
+// Geometry shared by all kernels: LOGN > 0 fixes the size at compile time (strides, loop
+// counts and shared-memory offsets fold to constants); LOGN == 0 takes it from the run-time
+// argument.  T = threads per CTA = N / (8 G) (at least one warp).
 template <int LOGN, int G>
 struct NttGeom {
-  u32 logn, n, octets, r0;
+  u32 logn, n, octets, r0, T;
   __device__ __forceinline__ explicit NttGeom(u32 logn_rt) {
     logn = LOGN ? (u32)LOGN : logn_rt;
     n = 1u << logn;
     octets = n >> 3;
     r0 = logn % 3u;
+    T = LOGN ? ((octets / G) < 32u ? 32u : (octets / G)) : blockDim.x;
   }
 };
 
-// Forward transform.  load(j) returns coefficient j in [0, p) (or any value < 4p);
-// emit(g, q, x) receives the octet of positions 8q..8q+7 (values in [0,4p)), q = tid + g*T.
-template <int LOGN, int G, class Load, class Emit>
+// Byte offsets into the swizzled shared-memory polynomial for the eight elements
+// base + (k << sh) of an octet.  The swizzle XORs the low four index bits with bits 4..6;
+// for the strides that occur (sh = 0, 3, 6 and >= 7) most of it is per-octet work, so an
+// element costs at most one XOR:
+//   sh >= 7: swz(base) + k*st            sh == 6: (swz(base) ^ 12*(k&1)) + 64k
+//   sh == 3: base - o + 16(k>>1) + ((o ^ 12*bit6(base)) ^ (8(k&1) ^ (k>>1)))
+//   sh == 0: swz(base) ^ k
+struct OctAddr {
+  u32 a, b;
+  __device__ __forceinline__ OctAddr(u32 base, u32 sh) {
+    if (sh >= 6 || sh == 0) {
+      a = swz(base) << 3;
+      b = a ^ (12u << 3);
+    } else if (sh == 3) {
+      const u32 o = base & 7u;
+      a = (base - o) << 3;
+      b = (o ^ (((base >> 6) & 1u) * 12u)) << 3;
+    } else {
+      a = base;
+      b = 0;
+    }
+  }
+  __device__ __forceinline__ u32 at(int k, u32 sh) const {
+    if (sh >= 7) return a + ((u32)k << (sh + 3));
+    if (sh == 6) return ((k & 1) ? b : a) + ((u32)k << 9);
+    if (sh == 3) return a + 128u * (u32)(k >> 1) + (b ^ ((u32)((8 * (k & 1)) ^ (k >> 1)) << 3));
+    if (sh == 0) return a ^ ((u32)k << 3);
+    return swz(a + ((u32)k << sh)) << 3;
+  }
+};
+__device__ __forceinline__ u64& sm_at(u64* sm, u32 byte_off) {
+  return *reinterpret_cast<u64*>(reinterpret_cast<unsigned char*>(sm) + byte_off);
+}
+
+// Forward transform.  load(j) returns coefficient j in [0, p);
+// emit(g, q, x) receives the octet of positions 8q..8q+7 (lazily reduced values: below 66p when
+// WIDE, below 8p otherwise), q = tid + g*T.
+template <int LOGN, int G, bool WIDE, class Load, class Emit>
 __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
                                             Load load, Emit emit) {
   const NttGeom<LOGN, G> ge(logn_rt);
-  const u32 T = blockDim.x, tid = threadIdx.x;
-  const u64 p = lt.p, twop = lt.twop;
+  const u32 T = ge.T, tid = threadIdx.x;
+  const Mod md(lt);
   const ulonglong2* __restrict__ W = lt.W;
   u64 x[8];
   __syncthreads();  // previous users of sm are done
   u32 s = 0;
   bool from_load = true;
   if (ge.r0) {
-    const u32 st = ge.octets;
+    const u32 sh = ge.logn - 3;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       const u32 q = tid + g * T;
-      if (q < ge.octets) {
+      if (LOGN || q < ge.octets) {
+        const OctAddr ad(q, sh);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) x[k] = load(q + k * st);
-        fwd_octet(x, W, 1, 0, (int)ge.r0, p, twop);
+        for (int k = 0; k < 8; ++k) x[k] = load(q + ((u32)k << sh));
+        fwd_octet<WIDE>(x, W, 1, 0, (int)ge.r0, md);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) sm[swz(q + k * st)] = x[k];
+        for (int k = 0; k < 8; ++k) sm_at(sm, ad.at(k, sh)) = x[k];
       }
     }
     s = ge.r0;
     from_load = false;
     __syncthreads();
   }
+#pragma unroll
   for (; s < ge.logn; s += 3) {
     const u32 sh = ge.logn - s - 3;  // log2 of the stride
-    const u32 st = 1u << sh, m = 1u << s;
+    const u32 m = 1u << s;
     const bool last = (s + 3 == ge.logn);
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       const u32 q = tid + g * T;
-      if (q < ge.octets) {
-        const u32 i = q >> sh, o = q & (st - 1);
+      if (LOGN || q < ge.octets) {
+        const u32 i = q >> sh, o = q & ((1u << sh) - 1);
         const u32 base = ((i << 3) << sh) + o;
+        const OctAddr ad(base, sh);
         if (from_load) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) x[k] = load(base + k * st);
+          for (int k = 0; k < 8; ++k) x[k] = load(base + ((u32)k << sh));
         } else {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) x[k] = sm[swz(base + k * st)];
+          for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
         }
-        fwd_octet(x, W, m, i, 3, p, twop);
+        fwd_octet<WIDE>(x, W, m, i, 3, md);
         if (last) {
           emit(g, q, x);
         } else {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) sm[swz(base + k * st)] = x[k];
+          for (int k = 0; k < 8; ++k) sm_at(sm, ad.at(k, sh)) = x[k];
         }
       }
     }
@@ -297,41 +410,44 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
 }
 
 // Inverse transform (without the N^-1 scaling: fold it into an operand).
-// fetch(g, q, x) fills the octet of positions 8q..8q+7 with values in [0,2p);
-// store(j, v) receives coefficient j, v in [0,2p).
-template <int LOGN, int G, class Fetch, class Store>
+// fetch(g, q, x) fills the octet of positions 8q..8q+7 with values below 4p (below 16p when WIDE);
+// store(j, v) receives coefficient j, v in [0,4p).
+template <int LOGN, int G, bool WIDE, class Fetch, class Store>
 __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
                                             Fetch fetch, Store store) {
   const NttGeom<LOGN, G> ge(logn_rt);
-  const u32 T = blockDim.x, tid = threadIdx.x;
-  const u64 p = lt.p, twop = lt.twop;
+  const u32 T = ge.T, tid = threadIdx.x;
+  const Mod md(lt);
   const ulonglong2* __restrict__ IW = lt.IW;
   u64 x[8];
   __syncthreads();  // previous users of sm are done
   bool from_fetch = true;
+#pragma unroll
   for (int s = (int)ge.logn - 3; s >= (int)ge.r0; s -= 3) {
     const u32 sh = ge.logn - (u32)s - 3;
-    const u32 st = 1u << sh, m = 1u << s;
+    const u32 m = 1u << s;
     const bool final_round = (s == 0);
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       const u32 q = tid + g * T;
-      if (q < ge.octets) {
-        const u32 i = q >> sh, o = q & (st - 1);
+      if (LOGN || q < ge.octets) {
+        const u32 i = q >> sh, o = q & ((1u << sh) - 1);
         const u32 base = ((i << 3) << sh) + o;
+        const OctAddr ad(base, sh);
         if (from_fetch) {
           fetch(g, q, x);
         } else {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) x[k] = sm[swz(base + k * st)];
+          for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
         }
-        inv_octet(x, IW, m, i, 3, p, twop);
+        inv_octet<WIDE>(x, IW, m, i, 3, md);
         if (final_round) {
+          finish_octet<WIDE>(x, 3, md);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) store(base + k * st, x[k]);
+          for (int k = 0; k < 8; ++k) store(base + ((u32)k << sh), x[k]);
         } else {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) sm[swz(base + k * st)] = x[k];
+          for (int k = 0; k < 8; ++k) sm_at(sm, ad.at(k, sh)) = x[k];
         }
       }
     }
@@ -339,16 +455,18 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
     if (!final_round) __syncthreads();
   }
   if (ge.r0) {
-    const u32 st = ge.octets;
+    const u32 sh = ge.logn - 3;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       const u32 q = tid + g * T;
-      if (q < ge.octets) {
+      if (LOGN || q < ge.octets) {
+        const OctAddr ad(q, sh);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) x[k] = sm[swz(q + k * st)];
-        inv_octet(x, IW, 1, 0, (int)ge.r0, p, twop);
+        for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
+        inv_octet<WIDE>(x, IW, 1, 0, (int)ge.r0, md);
+        finish_octet<WIDE>(x, (int)ge.r0, md);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) store(q + k * st, x[k]);
+        for (int k = 0; k < 8; ++k) store(q + ((u32)k << sh), x[k]);
       }
     }
   }

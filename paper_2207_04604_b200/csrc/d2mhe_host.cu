@@ -220,6 +220,7 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
     LimbTab& T = limbs[l];
     T.p = p;
     T.twop = 2 * p;
+    T.np = 0 - p;
     u64 inv = 1;  // Newton iteration for p^-1 mod 2^64
     for (int i = 0; i < 6; ++i) inv *= 2 - p * inv;
     T.pinv = inv;
@@ -261,6 +262,7 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
     T.IW = dev_upload(c, IW, &err);
     if (err != cudaSuccess) return fail_cuda(c, err);
   }
+  for (u32 l = 0; l < L; ++l) c->limb_params.limbs[l] = limbs[l];
   c->view.limbs = dev_upload(c, limbs, &err);
   if (err != cudaSuccess) return fail_cuda(c, err);
 
@@ -359,6 +361,9 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   c->view.n = n;
   c->view.L = L;
   c->view.K = P.num_parties;
+  c->view.wide = 1;
+  for (u32 l = 0; l < L; ++l)
+    if (c->moduli[l] >= ((u64)1 << 57)) c->view.wide = 0;
 
   // index staging ring
   err = cudaMallocHost(reinterpret_cast<void**>(&c->idx_host), kIdxSlots * kIdxSlotWords * sizeof(u32));
@@ -424,6 +429,7 @@ d2mhe_status d2mhe_create(const d2mhe_params* P, d2mhe_ctx** out) {
   c->can_pack = (t - 1) % two_n == 0;
   c->has_share.assign(P->num_parties, false);
   std::memset(&c->view, 0, sizeof(c->view));
+  std::memset(&c->limb_params, 0, sizeof(c->limb_params));
   for (u32 l = 0; l < P->num_limbs; ++l) {
     u64 r = h_find_root(c->moduli[l], P->log2_n);
     if (!r) {
@@ -489,7 +495,7 @@ d2mhe_status d2mhe_keygen_share(d2mhe_ctx* c, const u32* parties, u32 n_parties)
   const u32* arrays[1] = {parties};
   const size_t counts[1] = {n_parties};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::keygen(c->view, c->stream, sg.dev[0], n_parties);
+  cudaError_t e = d2mhe_launch::keygen(c->view, c->limb_params, c->stream, sg.dev[0], n_parties);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
   for (u32 i = 0; i < n_parties; ++i) c->has_share[parties[i]] = true;
@@ -508,7 +514,7 @@ d2mhe_status d2mhe_collective_pk(d2mhe_ctx* c, const u32* parties, u32 n_parties
   const u32* arrays[1] = {parties};
   const size_t counts[1] = {n_parties};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::collective_pk(c->view, c->stream, sg.dev[0], n_parties,
+  cudaError_t e = d2mhe_launch::collective_pk(c->view, c->limb_params, c->stream, sg.dev[0], n_parties,
                                               reinterpret_cast<u64*>(pk_shares_dev));
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
@@ -559,7 +565,7 @@ d2mhe_status d2mhe_encrypt(d2mhe_ctx* c, const u32* parties, u32 n_parties, u32 
   const u32* arrays[1] = {parties};
   const size_t counts[1] = {n_parties};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::encrypt(c->view, c->stream, sg.dev[0], n_parties, ct_first, n_cts,
+  cudaError_t e = d2mhe_launch::encrypt(c->view, c->limb_params, c->stream, sg.dev[0], n_parties, ct_first, n_cts,
                                         plain_dev, reinterpret_cast<u64*>(ct_dev));
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
@@ -614,7 +620,7 @@ d2mhe_status d2mhe_partial_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev, const 
   const size_t counts[2] = {n_rec, n_parties};
   if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
   cudaError_t e = d2mhe_launch::partial_decrypt(
-      c->view, c->stream, reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1], n_parties,
+      c->view, c->limb_params, c->stream, reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1], n_parties,
       ct_first, n_cts, reinterpret_cast<u64*>(shares_dev));
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
@@ -646,7 +652,7 @@ static d2mhe_status ntt_common(d2mhe_ctx* c, u64* polys_dev, u32 batch, bool inv
   if (c->params.log2_n > D2MHE_MAX_SMEM_LOGN) return D2MHE_ERR_UNSUPPORTED;
   if ((u64)batch * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
-  cudaError_t e = d2mhe_launch::ntt(c->view, c->stream, polys_dev, batch, inverse);
+  cudaError_t e = d2mhe_launch::ntt(c->view, c->limb_params, c->stream, polys_dev, batch, inverse);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
   return D2MHE_OK;

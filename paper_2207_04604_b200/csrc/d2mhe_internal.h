@@ -27,6 +27,13 @@ struct RoundTab {
   u64 qinv_mod_t;          // q^-1 mod t
 };
 
+// The per-limb constants travel as a kernel parameter (constant bank): indexed by the
+// CTA-uniform limb number they are read through the uniform datapath instead of occupying
+// vector registers in every thread.
+struct LimbParams {
+  LimbTab limbs[D2MHE_MAX_LIMBS];
+};
+
 // Everything a kernel needs, passed by value.
 struct DevView {
   const LimbTab* limbs;
@@ -35,6 +42,7 @@ struct DevView {
   RoundTab round;
   u64 seed;
   u32 logn, n, L, K;
+  u32 wide;      // 1 if every q_l < 2^57: lazy-reduction policy with no conditional subtractions
   u64* s_mont;   // [K][L][N]  NTT(s_k) * N^-1 in Montgomery form
   u64* pk_mont;  // [2][L][N]  NTT(p_0), NTT(p_1) * N^-1 in Montgomery form
   u64* pk_coef;  // [2][L][N]  (p_0, p_1), coefficient domain
@@ -58,6 +66,7 @@ struct d2mhe_ctx {
   int device = 0;
   cudaStream_t stream = nullptr;
   DevView view;
+  LimbParams limb_params;
   std::vector<void*> allocs;        // device allocations to free
   std::vector<bool> has_share;
   std::vector<u32> pk_parties;      // party set of the last collective_pk
@@ -73,21 +82,21 @@ struct d2mhe_ctx {
 };
 
 namespace d2mhe_launch {
-cudaError_t keygen(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 n_parties);
-cudaError_t collective_pk(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 n_parties,
+cudaError_t keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties);
+cudaError_t collective_pk(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
                           u64* shares_out);
 cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain);
 cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values);
-cudaError_t encrypt(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 n_parties,
+cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
                     u32 ct_first, u32 n_cts, const u32* plain, u64* ct);
 cudaError_t aggregate(const DevView& v, cudaStream_t s, const u64* ct, u32 n_cts,
                       const u32* offsets_dev, const u32* rows_dev, u32 n_out, u64* agg);
-cudaError_t partial_decrypt(const DevView& v, cudaStream_t s, const u64* agg,
+cudaError_t partial_decrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
                             const u32* recipients_dev, u32 n_rec, const u32* parties_dev,
                             u32 n_parties, u32 ct_first, u32 n_cts, u64* shares);
 cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
                     u32 n_shares, u32 n_cts, u32* plain);
-cudaError_t ntt(const DevView& v, cudaStream_t s, u64* polys, u32 batch, bool inverse);
+cudaError_t ntt(const DevView& v, const LimbParams& lp, cudaStream_t s, u64* polys, u32 batch, bool inverse);
 cudaError_t muladd(const DevView& v, cudaStream_t s, const u64* a, const u64* b, const u64* c,
                    u64* d, u32 batch);
 // number of kernel launches the call above performed (for bookkeeping)

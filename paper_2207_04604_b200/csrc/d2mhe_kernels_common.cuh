@@ -1,0 +1,189 @@
+// Shared pieces of the kernel translation units: shared-memory layout, octet I/O, dispatch.
+#pragma once
+#include <cooperative_groups.h>
+#include <cstdlib>
+
+#include "d2mhe_internal.h"
+
+// Octets per thread and round (G) and resident CTAs per SM aimed at, per ring degree.
+// Threads per CTA = N / (8 G).
+#ifndef D2MHE_G12
+#define D2MHE_G12 4
+#endif
+#ifndef D2MHE_G13
+#define D2MHE_G13 2
+#endif
+#ifndef D2MHE_G14
+#define D2MHE_G14 4
+#endif
+#ifndef D2MHE_MINB12
+#define D2MHE_MINB12 4
+#endif
+#ifndef D2MHE_MINB13
+#define D2MHE_MINB13 2
+#endif
+#ifndef D2MHE_MINB14
+#define D2MHE_MINB14 1
+#endif
+
+namespace {
+
+constexpr int ntt_minb_ct(int logn) {
+  return logn == 12 ? D2MHE_MINB12 : logn == 13 ? D2MHE_MINB13 : logn == 14 ? D2MHE_MINB14 : 1;
+}
+
+// Shared-memory layout of the transform kernels: [GaussTab][polynomial].
+__device__ __forceinline__ void load_gauss(GaussTab* dst, const GaussTab* __restrict__ src) {
+  const u32* s = reinterpret_cast<const u32*>(src);
+  u32* d = reinterpret_cast<u32*>(dst);
+  for (u32 i = threadIdx.x; i < sizeof(GaussTab) / 4; i += blockDim.x) d[i] = s[i];
+  __syncthreads();
+}
+
+extern __shared__ __align__(16) unsigned char smem_raw[];
+
+// [GaussTab][small-sample bytes: extra_bytes][polynomial]
+#define D2MHE_GAUSS_BYTES (((sizeof(GaussTab) + 15) / 16) * 16)
+__device__ __forceinline__ GaussTab* gauss_smem() { return reinterpret_cast<GaussTab*>(smem_raw); }
+__device__ __forceinline__ signed char* bytes_smem() {
+  return reinterpret_cast<signed char*>(smem_raw + D2MHE_GAUSS_BYTES);
+}
+__device__ __forceinline__ u64* poly_smem(u32 extra_bytes = 0) {
+  return reinterpret_cast<u64*>(smem_raw + D2MHE_GAUSS_BYTES + extra_bytes);
+}
+
+__device__ __forceinline__ void store_octet(u64* __restrict__ dst, const u64 (&x)[8]) {
+  ulonglong2* d = reinterpret_cast<ulonglong2*>(dst);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) d[k] = make_ulonglong2(x[2 * k], x[2 * k + 1]);
+}
+__device__ __forceinline__ void load_octet(const u64* __restrict__ src, u64 (&x)[8]) {
+  const ulonglong2* s = reinterpret_cast<const ulonglong2*>(src);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    ulonglong2 v = __ldg(s + k);
+    x[2 * k] = v.x;
+    x[2 * k + 1] = v.y;
+  }
+}
+
+// plain (coherent) load of an octet that this kernel wrote earlier
+__device__ __forceinline__ void load_octet_rw(const u64* src, u64 (&x)[8]) {
+  const ulonglong2* s = reinterpret_cast<const ulonglong2*>(src);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    ulonglong2 v = s[k];
+    x[2 * k] = v.x;
+    x[2 * k + 1] = v.y;
+  }
+}
+
+// v (below 4p) + small signed e, canonical in [0, p)
+__device__ __forceinline__ u64 add_small_canon(u64 v, int e, const LimbTab& lt) {
+  const u64 s = v + lt.p + (u64)(long long)e;  // below 5p + 19
+  return csub(csub(csub(s, 2 * lt.twop), lt.twop), lt.p);
+}
+
+constexpr u32 ntt_threads_ct(int logn, int g) {
+  return logn == 0 ? 1024u : (((1u << logn) / 8u / (u32)g) < 32u ? 32u : ((1u << logn) / 8u / (u32)g));
+}
+
+inline size_t poly_bytes(u32 n, size_t extra_bytes = 0) {
+  return D2MHE_GAUSS_BYTES + extra_bytes + (size_t)n * sizeof(u64);
+}
+inline u32 ntt_threads(u32 n, int g) {
+  u32 t = n / 8 / g;
+  return t < 32 ? 32 : t;
+}
+
+// Largest divisor of L that is a portable thread-block-cluster size.
+inline u32 cluster_size_for(u32 L) {
+  for (u32 cs = 8; cs > 1; --cs)
+    if (L % cs == 0) return cs;
+  return 1;
+}
+
+// Launch with a thread-block cluster of `cs` CTAs along x (cs = 1: plain launch).  Falls back
+// to cs = 1 when the device cannot co-schedule such a cluster for this kernel.
+template <class... KArgs, class... Args>
+cudaError_t launch_clustered(void (*kernel)(KArgs...), u32 grid, u32 threads, size_t smem,
+                             cudaStream_t stream, u32 cs, Args... args) {
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(threads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cs > 1) {
+    int max_clusters = 0;
+    cudaError_t e = cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg);
+    if (e != cudaSuccess || max_clusters < 1) {
+      (void)cudaGetLastError();
+      attr[0].val.clusterDim.x = 1;
+    }
+  }
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+#define D2MHE_LAUNCH_ONE(KERNEL, LOGN_, G_, WIDE_, grid, stream, cs, ...)                      \
+  do {                                                                                         \
+    cudaError_t e_ = launch_clustered(KERNEL<LOGN_, G_, WIDE_>, grid, ntt_threads(n_, G_),     \
+                                      smem_, stream, cs, __VA_ARGS__);                         \
+    if (e_ != cudaSuccess) return e_;                                                          \
+  } while (0)
+
+#define D2MHE_LAUNCH_W(KERNEL, LOGN_, G_, wide, grid, stream, cs, ...)                         \
+  do {                                                                                         \
+    if (wide)                                                                                  \
+      D2MHE_LAUNCH_ONE(KERNEL, LOGN_, G_, true, grid, stream, cs, __VA_ARGS__);                \
+    else                                                                                       \
+      D2MHE_LAUNCH_ONE(KERNEL, LOGN_, G_, false, grid, stream, cs, __VA_ARGS__);               \
+  } while (0)
+
+// Picks the instantiation for the ring degree: compile-time sizes for the production
+// degrees (with the octets-per-thread count G chosen per degree), the run-time-size build
+// for everything else; `wide` selects the lazy-reduction policy (all primes below 2^57).
+// extra = bytes of small-sample storage in front of the polynomial; cs = cluster size.
+#define D2MHE_DISPATCH_EX(KERNEL, view, grid, stream, extra, cs, ...)                          \
+  do {                                                                                         \
+    const u32 logn_ = (view).logn, n_ = 1u << logn_;                                           \
+    const size_t smem_ = poly_bytes(n_, extra);                                                \
+    const bool wide_ = (view).wide != 0;                                                       \
+    switch (logn_) {                                                                           \
+      case 12:                                                                                 \
+        D2MHE_LAUNCH_W(KERNEL, 12, D2MHE_G12, wide_, grid, stream, cs, __VA_ARGS__);           \
+        break;                                                                                 \
+      case 13:                                                                                 \
+        D2MHE_LAUNCH_W(KERNEL, 13, D2MHE_G13, wide_, grid, stream, cs, __VA_ARGS__);           \
+        break;                                                                                 \
+      case 14:                                                                                 \
+        D2MHE_LAUNCH_W(KERNEL, 14, D2MHE_G14, wide_, grid, stream, cs, __VA_ARGS__);           \
+        break;                                                                                 \
+      default:                                                                                 \
+        if (logn_ > 13) return cudaErrorInvalidValue;                                          \
+        D2MHE_LAUNCH_W(KERNEL, 0, 1, wide_, grid, stream, cs, __VA_ARGS__);                    \
+        break;                                                                                 \
+    }                                                                                          \
+    return cudaGetLastError();                                                                 \
+  } while (0)
+
+#define D2MHE_DISPATCH(KERNEL, view, grid, stream, ...) \
+  D2MHE_DISPATCH_EX(KERNEL, view, grid, stream, 0, 1, __VA_ARGS__)
+
+template <class K>
+cudaError_t set_smem(K kernel, size_t bytes) {
+  if (bytes <= 48 * 1024) return cudaSuccess;
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+}  // namespace

@@ -1,0 +1,100 @@
+// Key material: MBFV.SecKeyGen and MBFV.PubKeyGen (executed once per training).
+#include "d2mhe_kernels_common.cuh"
+
+namespace {
+
+// s_k from R_3, kept as NTT(s_k) * N^-1 in Montgomery form.   grid = n_parties * L
+template <int LOGN, int G, bool WIDE>
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+    k_keygen(DevView v, const __grid_constant__ LimbParams lp, const u32* __restrict__ parties) {
+  const u32 l = blockIdx.x % v.L, party = parties[blockIdx.x / v.L];
+  const LimbTab& lt = lp.limbs[l];
+  const Stream st(v.seed, TAG_SECRET, 0, party, 0);
+  u64* out = v.s_mont + ((size_t)party * v.L + l) * v.n;
+  ntt_forward<LOGN, G, WIDE>(
+      poly_smem(), lt, v.logn, [&](u32 j) { return lift_small(st.ternary(j), lt.p); },
+      [&](int, u32 q, u64(&x)[8]) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = shoup_full(x[k], lt.mont_ninv, lt.mont_ninv_sh, lt.p);
+        store_octet(out + 8 * (size_t)q, x);
+      });
+}
+
+// p_1 uniform; p_{0,k} = -(p_1 s_k + e_k); p_0 = sum_k p_{0,k}.
+// grid = L: one CTA per limb walks over the parties.
+template <int LOGN, int G, bool WIDE>
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+    k_collective_pk(DevView v, const __grid_constant__ LimbParams lp, const u32* __restrict__ parties, u32 n_parties,
+                    u64* __restrict__ shares_out) {
+  const u32 l = blockIdx.x;
+  const LimbTab& lt = lp.limbs[l];
+  GaussTab* gt = gauss_smem();
+  load_gauss(gt, v.gauss);
+  u64* sm = poly_smem();
+  const size_t row = (size_t)l * v.n, poly = (size_t)v.L * v.n;
+  u64* p0c = v.pk_coef + row;
+  u64* p1c = v.pk_coef + poly + row;
+  u64 p1h[G][8];
+  {
+    const Stream st(v.seed, TAG_P1, l, 0, 0);
+    ntt_forward<LOGN, G, WIDE>(
+        sm, lt, v.logn,
+        [&](u32 j) {
+          u64 r = uniform_mod(st, j, lt.p, lt.mask);
+          p1c[j] = r;
+          p0c[j] = 0;
+          return r;
+        },
+        [&](int g, u32 q, u64(&x)[8]) {
+          u64 y[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            p1h[g][k] = x[k];
+            y[k] = shoup_full(x[k], lt.mont_ninv, lt.mont_ninv_sh, lt.p);
+          }
+          store_octet(v.pk_mont + poly + row + 8 * (size_t)q, y);
+        });
+  }
+  for (u32 a = 0; a < n_parties; ++a) {
+    const u32 party = parties[a];
+    const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
+    const Stream se(v.seed, TAG_PK_ERR, 0, party, 0);
+    u64* share = shares_out ? shares_out + ((size_t)a * v.L + l) * v.n : nullptr;
+    ntt_inverse<LOGN, G, WIDE>(
+        sm, lt, v.logn,
+        [&](int g, u32 q, u64(&x)[8]) {
+          load_octet(sk + 8 * (size_t)q, x);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) x[k] = mont_lazy(p1h[g][k], x[k], lt.p, lt.pinv);
+        },
+        [&](u32 j, u64 val) {
+          val = add_small_canon(val, gauss_from_r(*gt, se.draw64(j)), lt);
+          val = val ? lt.p - val : 0;
+          if (share) share[j] = val;
+          p0c[j] = addmod(p0c[j], val, lt.p);  // the same thread owns j for every party
+        });
+  }
+  __syncthreads();  // p0c complete and visible to the whole CTA
+  ntt_forward<LOGN, G, WIDE>(
+      sm, lt, v.logn, [&](u32 j) { return p0c[j]; },
+      [&](int, u32 q, u64(&x)[8]) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = shoup_full(x[k], lt.mont_ninv, lt.mont_ninv_sh, lt.p);
+        store_octet(v.pk_mont + row + 8 * (size_t)q, x);
+      });
+}
+
+}  // namespace
+
+namespace d2mhe_launch {
+
+cudaError_t keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties) {
+  D2MHE_DISPATCH(k_keygen, v, n_parties * v.L, s, v, lp, parties_dev);
+}
+
+cudaError_t collective_pk(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
+                          u64* shares_out) {
+  D2MHE_DISPATCH(k_collective_pk, v, v.L, s, v, lp, parties_dev, n_parties, shares_out);
+}
+
+}  // namespace d2mhe_launch

@@ -1,0 +1,232 @@
+// Streaming kernels: RNS multiply-add, neighbour sums, combine + exact scale-and-round, packing.
+#include "d2mhe_kernels_common.cuh"
+
+namespace {
+
+// d = a (.) b + c per residue; two residues per thread (16-byte accesses).
+__global__ void __launch_bounds__(256) k_muladd(DevView v, const u64* __restrict__ a,
+                                                const u64* __restrict__ b,
+                                                const u64* __restrict__ c, u64* __restrict__ d,
+                                                size_t n_pairs) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_pairs; e += stride) {
+    const u32 l = (u32)(((e * 2) >> v.logn) % v.L);
+    const LimbTab* lt = v.limbs + l;
+    const u64 p = lt->p, pinv = lt->pinv, r = lt->rmod, rs = lt->rmod_sh;
+    const ulonglong2 av = reinterpret_cast<const ulonglong2*>(a)[e];
+    const ulonglong2 bv = reinterpret_cast<const ulonglong2*>(b)[e];
+    const ulonglong2 cv = reinterpret_cast<const ulonglong2*>(c)[e];
+    ulonglong2 o;
+    o.x = addmod(shoup_full(mont_lazy(av.x, bv.x, p, pinv), r, rs, p), cv.x, p);
+    o.y = addmod(shoup_full(mont_lazy(av.y, bv.y, p, pinv), r, rs, p), cv.y, p);
+    reinterpret_cast<ulonglong2*>(d)[e] = o;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// BFV.Add over neighbour lists.  grid = (n_out * n_cts, chunks); two residues per thread.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+    k_aggregate(DevView v, const u64* __restrict__ ct, u32 n_cts, const u32* __restrict__ offsets,
+                const u32* __restrict__ rows, u64* __restrict__ agg) {
+  const u32 unit = blockIdx.x, i = unit / n_cts, c = unit % n_cts;
+  const size_t ct_pairs = (size_t)v.L * v.n;  // 2*L*N residues = L*N pairs
+  const u32 beg = offsets[i], end = offsets[i + 1];
+  ulonglong2* out = reinterpret_cast<ulonglong2*>(agg) + (size_t)unit * ct_pairs;
+  for (size_t e = (size_t)blockIdx.y * blockDim.x + threadIdx.x; e < ct_pairs;
+       e += (size_t)gridDim.y * blockDim.x) {
+    const u32 l = (u32)(((e * 2) >> v.logn) % v.L);
+    const u64 p = v.limbs[l].p;
+    ulonglong2 acc = make_ulonglong2(0, 0);
+    for (u32 a = beg; a < end; ++a) {
+      const ulonglong2 x =
+          __ldg(reinterpret_cast<const ulonglong2*>(ct) + ((size_t)rows[a] * n_cts + c) * ct_pairs + e);
+      acc.x = addmod(acc.x, x.x, p);
+      acc.y = addmod(acc.y, x.y, p);
+    }
+    out[e] = acc;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Combine + exact scale-and-round.  One thread per coefficient.
+//   v_l = c_0 + sum_k h_k mod q_l;  w'_l = t v_l + (q-1)/2 mod q_l;
+//   mixed-radix digits d_i of w' in [0,q);  w' mod t = sum d_i prod_{j<i} q_j mod t;
+//   x = ((q-1)/2 - w') q^-1 mod t  =  round(t v / q) mod t.
+// grid = (n_rec * n_cts, N / 256)
+// ---------------------------------------------------------------------------
+template <int LMAX>
+__global__ void __launch_bounds__(256)
+    k_combine(DevView v, const u64* __restrict__ agg, const u64* __restrict__ shares, u32 n_shares,
+              u32 n_cts, u32* __restrict__ plain) {
+  const u32 unit = blockIdx.x, irec = unit / n_cts, cl = unit % n_cts;
+  const u32 j = blockIdx.y * blockDim.x + threadIdx.x;
+  if (j >= v.n) return;
+  const u32 L = v.L;
+  const size_t poly = (size_t)L * v.n;
+  const u64* c0 = agg + (size_t)unit * 2 * poly;
+  u64 d[LMAX];
+#pragma unroll
+  for (int l = 0; l < LMAX; ++l) {
+    if (l < (int)L) {
+      const LimbTab* lt = v.limbs + l;
+      const u64 p = lt->p;
+      u64 acc = __ldg(c0 + (size_t)l * v.n + j);
+      for (u32 k = 0; k < n_shares; ++k)
+        acc = addmod(acc, __ldg(shares + (((size_t)irec * n_shares + k) * n_cts + cl) * poly +
+                                (size_t)l * v.n + j), p);
+      d[l] = addmod(shoup_full(acc, lt->tmod, lt->tmod_sh, p), lt->half, p);
+    }
+  }
+  // mixed-radix (Garner) digits in place: d_i <- ((w'_i - d_0) q_0^-1 - d_1) q_1^-1 ... mod q_i
+#pragma unroll
+  for (int i = 1; i < LMAX; ++i) {
+    if (i < (int)L) {
+      const LimbTab* lt = v.limbs + i;
+      const u64 p = lt->p, cq = lt->cq;
+      u64 tmp = d[i];
+#pragma unroll
+      for (int jj = 0; jj < i; ++jj) {
+        const ulonglong2 gi = __ldg(v.round.ginv + i * L + jj);
+        tmp = shoup_full(tmp + cq - d[jj], gi.x, gi.y, p);
+      }
+      d[i] = tmp;
+    }
+  }
+  const u64 t = v.round.t, tsh = v.round.t_sh;
+  u64 acc = 0;
+#pragma unroll
+  for (int i = 0; i < LMAX; ++i) {
+    if (i < (int)L) {
+      const u64 di = shoup_full(d[i], 1, tsh, t);  // d_i mod t
+      acc = shoup_full(acc + di * v.round.prefix_mod_t[i], 1, tsh, t);
+    }
+  }
+  const u64 diff = v.round.half_mod_t + t - acc;  // in (0, 2t)
+  plain[(size_t)unit * v.n + j] = (u32)shoup_full(diff * v.round.qinv_mod_t, 1, tsh, t);
+}
+
+// ---------------------------------------------------------------------------
+// Packing: negacyclic transforms mod t in shared memory (32-bit arithmetic).
+// Slot j sits at transform position brv(j).  grid = n_cts
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ u32 shoup32_lazy(u32 x, uint2 w, u32 t) {
+  return x * w.x - __umulhi(x, w.y) * t;
+}
+__device__ __forceinline__ u32 csub32(u32 x, u32 t) { return x >= t ? x - t : x; }
+
+__global__ void __launch_bounds__(1024)
+    k_encode(DevView v, const int32_t* __restrict__ values, u32* __restrict__ plain) {
+  u32* sm = reinterpret_cast<u32*>(smem_raw);
+  const PlainTab pt = v.plain;
+  const u32 n = v.n, logn = v.logn, t = pt.t, twot = pt.twot;
+  const int32_t* in = values + (size_t)blockIdx.x * n;
+  u32* out = plain + (size_t)blockIdx.x * n;
+  bool bad = false;
+  for (u32 j = threadIdx.x; j < n; j += blockDim.x) {
+    const int32_t val = in[j];
+    bad |= (val > (int32_t)pt.half) || (val < -(int32_t)pt.half);
+    int32_t r = val % (int32_t)t;
+    if (r < 0) r += (int32_t)t;
+    sm[__brev(j) >> (32 - logn)] = (u32)r;
+  }
+  if (bad) atomicOr(v.range_flag, 1u);
+  __syncthreads();
+  u32 lt = 0;  // log2 of the butterfly span
+  for (u32 m = n >> 1; m >= 1; m >>= 1, ++lt) {
+    for (u32 b = threadIdx.x; b < (n >> 1); b += blockDim.x) {
+      const u32 i = b >> lt, jj = b & ((1u << lt) - 1);
+      const u32 idx = (i << (lt + 1)) + jj;
+      const u32 X = sm[idx], Y = sm[idx + (1u << lt)];
+      const uint2 w = __ldg(pt.IW + m + i);
+      sm[idx] = csub32(X + Y, twot);
+      sm[idx + (1u << lt)] = shoup32_lazy(X - Y + twot, w, t);
+    }
+    __syncthreads();
+  }
+  const uint2 ninv = make_uint2(pt.ninv, pt.ninv_sh);
+  for (u32 j = threadIdx.x; j < n; j += blockDim.x) out[j] = csub32(shoup32_lazy(sm[j], ninv, t), t);
+}
+
+__global__ void __launch_bounds__(1024)
+    k_decode(DevView v, const u32* __restrict__ plain, int32_t* __restrict__ values) {
+  u32* sm = reinterpret_cast<u32*>(smem_raw);
+  const PlainTab pt = v.plain;
+  const u32 n = v.n, logn = v.logn, t = pt.t, twot = pt.twot;
+  const u32* in = plain + (size_t)blockIdx.x * n;
+  int32_t* out = values + (size_t)blockIdx.x * n;
+  for (u32 j = threadIdx.x; j < n; j += blockDim.x) sm[j] = in[j];
+  __syncthreads();
+  u32 lt = logn - 1;
+  for (u32 m = 1; m < n; m <<= 1, --lt) {
+    for (u32 b = threadIdx.x; b < (n >> 1); b += blockDim.x) {
+      const u32 i = b >> lt, jj = b & ((1u << lt) - 1);
+      const u32 idx = (i << (lt + 1)) + jj;
+      const u32 X = csub32(sm[idx], twot);
+      const uint2 w = __ldg(pt.W + m + i);
+      const u32 T = shoup32_lazy(sm[idx + (1u << lt)], w, t);
+      sm[idx] = X + T;
+      sm[idx + (1u << lt)] = X - T + twot;
+    }
+    __syncthreads();
+  }
+  for (u32 j = threadIdx.x; j < n; j += blockDim.x) {
+    const u32 y = csub32(csub32(sm[__brev(j) >> (32 - logn)], twot), t);
+    out[j] = y > pt.half ? (int32_t)y - (int32_t)t : (int32_t)y;
+  }
+}
+
+}  // namespace
+
+namespace d2mhe_launch {
+
+cudaError_t muladd(const DevView& v, cudaStream_t s, const u64* a, const u64* b, const u64* c,
+                   u64* d, u32 batch) {
+  const size_t n_pairs = (size_t)batch * v.L * v.n / 2;
+  size_t blocks = (n_pairs + 255) / 256;
+  if (blocks > 148 * 32) blocks = 148 * 32;
+  k_muladd<<<(u32)blocks, 256, 0, s>>>(v, a, b, c, d, n_pairs);
+  return cudaGetLastError();
+}
+
+cudaError_t aggregate(const DevView& v, cudaStream_t s, const u64* ct, u32 n_cts,
+                      const u32* offsets_dev, const u32* rows_dev, u32 n_out, u64* agg) {
+  const size_t ct_pairs = (size_t)v.L * v.n;
+  u32 by = (u32)((ct_pairs + 255) / 256);
+  if (by > 32768) by = 32768;
+  dim3 grid(n_out * n_cts, by);
+  k_aggregate<<<grid, 256, 0, s>>>(v, ct, n_cts, offsets_dev, rows_dev, agg);
+  return cudaGetLastError();
+}
+
+cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
+                    u32 n_shares, u32 n_cts, u32* plain) {
+  dim3 grid(n_rec * n_cts, (v.n + 255) / 256);
+  if (v.L <= 4)
+    k_combine<4><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, n_cts, plain);
+  else if (v.L <= 8)
+    k_combine<8><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, n_cts, plain);
+  else
+    k_combine<D2MHE_MAX_LIMBS><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, n_cts, plain);
+  return cudaGetLastError();
+}
+
+cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain) {
+  const size_t smem = (size_t)v.n * 4;
+  cudaError_t e = set_smem(k_encode, smem);
+  if (e != cudaSuccess) return e;
+  u32 threads = v.n / 2 < 1024 ? (v.n / 2 < 32 ? 32 : v.n / 2) : 1024;
+  k_encode<<<n_cts, threads, smem, s>>>(v, values, plain);
+  return cudaGetLastError();
+}
+
+cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values) {
+  const size_t smem = (size_t)v.n * 4;
+  cudaError_t e = set_smem(k_decode, smem);
+  if (e != cudaSuccess) return e;
+  u32 threads = v.n / 2 < 1024 ? (v.n / 2 < 32 ? 32 : v.n / 2) : 1024;
+  k_decode<<<n_cts, threads, smem, s>>>(v, plain, values);
+  return cudaGetLastError();
+}
+
+}  // namespace d2mhe_launch
