@@ -155,6 +155,8 @@ d2mhe_status d2mhe_combine_decrypt(d2mhe_ctx* ctx, const uint64_t* agg_dev,
  * Batched negacyclic number-theoretic transform of [batch, L, N], in place.
  * Forward: position p of limb l receives a(psi_l^(2 brv(p) + 1)), brv = reversal of
  * the log2_n-bit index, psi_l the root reported by d2mhe_get_root.  Inverse undoes it.
+ * N <= 16384 runs as one kernel with the polynomial in shared memory; N = 32768, 65536 run
+ * as two passes (the first 3 or 4 stages in registers, then 4096-point blocks).
  * These are the ring isomorphism behind every product of Sec. 3.2 / 4.2.
  */
 d2mhe_status d2mhe_ntt_forward(d2mhe_ctx* ctx, uint64_t* polys_dev, uint32_t batch);

@@ -164,8 +164,9 @@ __device__ __forceinline__ u32 swz(u32 a) { return a ^ ((a >> 4) & 7u) ^ (((a >>
 // --- multiplication by a constant with an approximate quotient -------------------------
 // Returns y*w - q*p (mod 2^64) with q = ah*bh + hi32(ah*bl) + hi32(al*bh) for a = y,
 // b = ws = floor(w 2^64 / p): q is the true floor(y ws / 2^64) or up to 2 below it, so the
-// result is congruent to y*w and lies in [0, 4p) for ANY 64-bit y.  Five widening and four
-// 32-bit multiply-adds; no carry chains (the integer multiplier is the scarce pipe on B200).
+// result is congruent to y*w and lies in [0, 4p) for ANY 64-bit y.  Five widening / high and
+// four 32-bit multiply-adds, written with explicit 32-bit halves so that no 64-bit multiply
+// is synthesised (the integer multiplier is the scarce pipe on B200).
 __device__ __forceinline__ u64 madwide(u32 a, u32 b, u64 c) {
   u64 r;
   asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "r"(b), "l"(c));
@@ -176,19 +177,40 @@ __device__ __forceinline__ u32 madlo(u32 a, u32 b, u32 c) {
   asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
   return r;
 }
+__device__ __forceinline__ u64 mulwide(u32 a, u32 b) {
+  u64 r;
+  asm("mul.wide.u32 %0, %1, %2;" : "=l"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ u32 mulhi32(u32 a, u32 b) {
+  u32 r;
+  asm("mul.hi.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ void split64(u64 x, u32& lo, u32& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(x));
+}
+__device__ __forceinline__ u64 join64(u32 lo, u32 hi) {
+  u64 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
 __device__ __forceinline__ u64 shoup_approx(u64 y, u64 w, u64 ws, u64 np) {
-  const u32 yl = (u32)y, yh = (u32)(y >> 32), sl = (u32)ws, sh = (u32)(ws >> 32);
-  const u64 t1 = (u64)yh * sl, t2 = (u64)yl * sh;
-  const u64 q = madwide(yh, sh, t1 >> 32) + (t2 >> 32);
-  const u32 ql = (u32)q, qh = (u32)(q >> 32), wl = (u32)w, wh = (u32)(w >> 32);
-  const u32 nl = (u32)np, nh = (u32)(np >> 32);
-  u64 r = madwide(ql, nl, (u64)yl * wl);
-  u32 rh = (u32)(r >> 32);
+  u32 yl, yh, sl, sh, wl, wh, nl, nh;
+  split64(y, yl, yh);
+  split64(ws, sl, sh);
+  split64(w, wl, wh);
+  split64(np, nl, nh);
+  u64 q = madwide(yh, sh, join64(mulhi32(yh, sl), 0u));
+  q += (u64)mulhi32(yl, sh);
+  u32 ql, qh, rl, rh;
+  split64(q, ql, qh);
+  split64(madwide(ql, nl, mulwide(yl, wl)), rl, rh);
   rh = madlo(yl, wh, rh);
   rh = madlo(yh, wl, rh);
   rh = madlo(ql, nh, rh);
   rh = madlo(qh, nl, rh);
-  return ((u64)rh << 32) | (u32)r;
+  return join64(rl, rh);
 }
 
 // Lazy-reduction policy.  WIDE (every prime below 2^57): values may grow across stages, so
@@ -344,12 +366,16 @@ __device__ __forceinline__ u64& sm_at(u64* sm, u32 byte_off) {
   return *reinterpret_cast<u64*>(reinterpret_cast<unsigned char*>(sm) + byte_off);
 }
 
-// Forward transform.  load(j) returns coefficient j in [0, p);
+// A transform of size N' = 2^logn can also be block `blk` of a larger transform whose first
+// `soff` stages were applied elsewhere (two-pass transforms for N > 16384): the block then
+// uses the twiddles of the sub-tree below node (soff, blk), i.e. index (m << soff) + (blk << s) + i.
+//
+// Forward transform.  load(j) returns coefficient j (any lazily reduced value below 8p);
 // emit(g, q, x) receives the octet of positions 8q..8q+7 (lazily reduced values: below 66p when
 // WIDE, below 8p otherwise), q = tid + g*T.
 template <int LOGN, int G, bool WIDE, class Load, class Emit>
 __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
-                                            Load load, Emit emit) {
+                                            Load load, Emit emit, u32 soff = 0, u32 blk = 0) {
   const NttGeom<LOGN, G> ge(logn_rt);
   const u32 T = ge.T, tid = threadIdx.x;
   const Mod md(lt);
@@ -367,7 +393,7 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
         const OctAddr ad(q, sh);
 #pragma unroll
         for (int k = 0; k < 8; ++k) x[k] = load(q + ((u32)k << sh));
-        fwd_octet<WIDE>(x, W, 1, 0, (int)ge.r0, md);
+        fwd_octet<WIDE>(x, W, 1u << soff, blk, (int)ge.r0, md);
 #pragma unroll
         for (int k = 0; k < 8; ++k) sm_at(sm, ad.at(k, sh)) = x[k];
       }
@@ -395,7 +421,7 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
         }
-        fwd_octet<WIDE>(x, W, m, i, 3, md);
+        fwd_octet<WIDE>(x, W, m << soff, (blk << s) + i, 3, md);
         if (last) {
           emit(g, q, x);
         } else {
@@ -414,7 +440,7 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
 // store(j, v) receives coefficient j, v in [0,4p).
 template <int LOGN, int G, bool WIDE, class Fetch, class Store>
 __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
-                                            Fetch fetch, Store store) {
+                                            Fetch fetch, Store store, u32 soff = 0, u32 blk = 0) {
   const NttGeom<LOGN, G> ge(logn_rt);
   const u32 T = ge.T, tid = threadIdx.x;
   const Mod md(lt);
@@ -440,7 +466,7 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
         }
-        inv_octet<WIDE>(x, IW, m, i, 3, md);
+        inv_octet<WIDE>(x, IW, m << soff, (blk << s) + i, 3, md);
         if (final_round) {
           finish_octet<WIDE>(x, 3, md);
 #pragma unroll
@@ -463,7 +489,7 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
         const OctAddr ad(q, sh);
 #pragma unroll
         for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
-        inv_octet<WIDE>(x, IW, 1, 0, (int)ge.r0, md);
+        inv_octet<WIDE>(x, IW, 1u << soff, blk, (int)ge.r0, md);
         finish_octet<WIDE>(x, (int)ge.r0, md);
 #pragma unroll
         for (int k = 0; k < 8; ++k) store(q + ((u32)k << sh), x[k]);

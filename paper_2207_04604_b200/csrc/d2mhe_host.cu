@@ -649,12 +649,12 @@ d2mhe_status d2mhe_combine_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev,
 static d2mhe_status ntt_common(d2mhe_ctx* c, u64* polys_dev, u32 batch, bool inverse) {
   if (!c || !polys_dev || batch == 0) return D2MHE_ERR_INVALID_ARG;
   if (!aligned16(polys_dev)) return D2MHE_ERR_INVALID_ARG;
-  if (c->params.log2_n > D2MHE_MAX_SMEM_LOGN) return D2MHE_ERR_UNSUPPORTED;
-  if ((u64)batch * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)batch * c->view.L * (c->params.log2_n > D2MHE_MAX_SMEM_LOGN ? 16u : 1u) > 0x7fffffffull)
+    return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
   cudaError_t e = d2mhe_launch::ntt(c->view, c->limb_params, c->stream, polys_dev, batch, inverse);
   if (e != cudaSuccess) return fail_cuda(c, e);
-  c->launches += 1;
+  c->launches += c->params.log2_n > D2MHE_MAX_SMEM_LOGN ? 2 : 1;
   return D2MHE_OK;
 }
 d2mhe_status d2mhe_ntt_forward(d2mhe_ctx* c, uint64_t* polys_dev, u32 batch) {

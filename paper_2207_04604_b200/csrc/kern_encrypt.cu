@@ -8,13 +8,15 @@ namespace {
 // Lambda * m for a plaintext coefficient m < 2^32: exact quotient from two widening
 // products, result in [0, 2p).
 __device__ __forceinline__ u64 shoup_u32(u32 m, u64 w, u64 ws, u64 np) {
-  const u32 sl = (u32)ws, sh = (u32)(ws >> 32);
-  const u32 q = (u32)(madwide(m, sh, ((u64)m * sl) >> 32) >> 32);
-  u64 r = madwide(q, (u32)np, (u64)m * (u32)w);
-  u32 rh = (u32)(r >> 32);
-  rh = madlo(m, (u32)(w >> 32), rh);
-  rh = madlo(q, (u32)(np >> 32), rh);
-  return ((u64)rh << 32) | (u32)r;
+  u32 sl, sh, wl, wh, nl, nh, ql, q, rl, rh;
+  split64(ws, sl, sh);
+  split64(w, wl, wh);
+  split64(np, nl, nh);
+  split64(madwide(m, sh, join64(mulhi32(m, sl), 0u)), ql, q);  // q = floor(m ws / 2^64) exactly
+  split64(madwide(q, nl, mulwide(m, wl)), rl, rh);
+  rh = madlo(m, wh, rh);
+  rh = madlo(q, nh, rh);
+  return join64(rl, rh);
 }
 
 // grid = n_units * L, launched in thread-block clusters of cs CTAs = cs limbs of the same

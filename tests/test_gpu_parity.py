@@ -38,6 +38,7 @@ def _brv(n_bits):
     (3, 30, 1, 2), (4, 36, 2, 3), (5, 54, 3, 2), (6, 60, 2, 5), (7, 50, 2, 2), (8, 54, 1, 3),
     (9, 60, 2, 2), (10, 36, 3, 2), (11, 54, 2, 2), (12, 36, 3, 5), (12, 60, 4, 3),
     (13, 54, 4, 3), (13, 60, 1, 7), (14, 54, 8, 2), (14, 60, 3, 3),
+    (15, 60, 2, 2), (15, 50, 3, 1), (16, 60, 3, 2), (16, 54, 1, 3),
 ])
 def test_ntt_forward_inverse_against_oracle(d2, log2_n, bits, L, batch):
     moduli = wl.ntt_primes(bits, 1 << 17, L) if bits >= 50 else small_moduli(log2_n, bits, L)
