@@ -107,6 +107,36 @@ def algorithmic_bytes(cfg, n_cts):
     }
 
 
+# Integer roofline of the transform-bearing kernels.  The scarce unit is the 32-bit integer
+# multiply-add pipe: 64 lanes per SM per clock (a widening or high-half multiply occupies it
+# for two passes).  Peak = 148 SMs x 64 lanes x 1.965 GHz (the documented SM count and maximum
+# SM clock) = 18.6e12 multiply-add slots per second; a register-only probe of the butterfly
+# reaches 96 % of it.  Algorithmic slots: one lazy Shoup butterfly = 5 widening/high + 4 low
+# multiplies = 14 slots; a transform = (N/2) log2 N butterflies; a pointwise product = 14;
+# one Philox4x32-10 call = 20 widening multiplies = 40 slots (one call serves all L limbs).
+IMAD_LANES_PER_SM = 64
+NUM_SMS = 148
+SM_MAX_HZ = 1.965e9
+IMAD_PEAK = NUM_SMS * IMAD_LANES_PER_SM * SM_MAX_HZ
+
+
+def algorithmic_mad_slots(cfg, n_cts):
+    K, S, L, n = cfg.num_parties, cfg.num_parties, cfg.num_limbs, cfg.n
+    transform = 14 * (n // 2) * cfg.log2_n   # slots per limb-transform
+    units = K * n_cts
+    return {
+        # NTT(u) + 2 inverse transforms, 2 pointwise products, Lambda*m (10 slots) per limb; 3 samples per coefficient
+        "encrypt": units * (L * (3 * transform + n * (2 * 14 + 10)) + 3 * 40 * n),
+        # NTT(c1) once, then per share: pointwise product + inverse transform per limb, one sample per coefficient
+        "partial_decrypt": units * (L * (transform + S * (transform + 14 * n)) + S * 40 * n),
+    }
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures under profiles/
+# (null when the kernel has changed since the capture).
+NCU_TRAFFIC_BYTES = {}
+
+
 # ----------------------------------------------------------------------------------
 # reference arm: the CPU oracle, as it stands
 # ----------------------------------------------------------------------------------
@@ -377,9 +407,24 @@ def run_cuda(args, cfg):
         dur_ms = per_call[dominant] / launches_dom
         bytes_per_launch = ab[dominant] / (n_chunks_total / args.steps)
         achieved = bytes_per_launch / 1e9 / (dur_ms * 1e-3)
-        roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": None,
-                    "avg_launch_ms": dur_ms}
+        traffic = NCU_TRAFFIC_BYTES.get((cfg.name, dominant))
+        slots = algorithmic_mad_slots(cfg, C)
+        if dominant in slots:  # transform-bearing kernel: bound by the integer multiply-add pipe
+            slots_per_launch = slots[dominant] / (n_chunks_total / args.steps)
+            got = slots_per_launch / (dur_ms * 1e-3)
+            roofline = {"bound": "alu", "kernel": dominant, "achieved": got / 1e12, "peak": IMAD_PEAK / 1e12,
+                        "unit": "T int32 multiply-add slots/s", "frac": got / IMAD_PEAK,
+                        "peak_source": "148 SMs x 64 lanes x 1.965 GHz (unit counts and clocks)",
+                        "traffic": traffic, "avg_launch_ms": dur_ms,
+                        "hbm": {"achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                                "peak_source": "of " + peak_kind}}
+        else:
+            roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                        "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": traffic,
+                        "avg_launch_ms": dur_ms}
+        for name in slots:
+            ms = kernels[name]["ms_per_step"]
+            kernels[name]["alu_frac"] = slots[name] / (ms * 1e-3) / IMAD_PEAK if ms else None
         round_bytes = sum(ab.values())
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -406,17 +451,88 @@ def run_cuda(args, cfg):
     parallel.finish()
 
 
+def run_sweep(args):
+    """Kernel sweep (configuration 5): batched forward/inverse transforms and the RNS multiply-add over
+    N in 2^12..2^16, L in {1,4,8,16,24}, batch in {1,64,1024,4096}, uniform residues mod 60-bit primes
+    (50-bit with --sweep-bits 50).  One JSON line with a row per point; GB/s = 16 B (transforms) or 32 B
+    (multiply-add) per residue over the CUDA-event time, against the measured HBM copy bandwidth."""
+    import torch
+
+    from paper_2207_04604_b200 import build, d2mhe
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    build.build()
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.current_stream(dev)
+    peak, peak_kind = measured_peaks()
+    flush = torch.empty(384 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    rows = []
+    for log2_n in wl.SWEEP_LOG2_N:
+        n = 1 << log2_n
+        for L in wl.SWEEP_LIMBS:
+            moduli = wl.sweep_moduli(args.sweep_bits, L)
+            ctx = d2mhe.Context(log2_n, moduli, 1, seed=args.seed)
+            tile = torch.from_numpy(wl.random_polys(moduli, log2_n, 1, args.seed).view(np.int64)).to(dev)
+            for batch in wl.SWEEP_BATCH:
+                nbytes = 8 * n * L * batch
+                row = {"N": n, "L": L, "batch": batch, "GiB": nbytes / 2**30}
+                if nbytes > 0.6 * free_b:
+                    row["skipped"] = "buffer exceeds the memory budget"
+                    rows.append(row)
+                    continue
+                polys = tile.expand(batch, L, n).contiguous()
+
+                def timed(fn, reps=3):
+                    fn()
+                    best = None
+                    for _ in range(reps):
+                        flush.zero_()
+                        a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a_.record(stream)
+                        fn()
+                        b_.record(stream)
+                        torch.cuda.synchronize(dev)
+                        ms = a_.elapsed_time(b_)
+                        best = ms if best is None else min(best, ms)
+                    return best
+
+                f_ms = timed(lambda: ctx.ntt_forward(polys, batch))
+                i_ms = timed(lambda: ctx.ntt_inverse(polys, batch))
+                row.update({"forward_GBps": 2 * nbytes / 1e9 / (f_ms * 1e-3), "inverse_GBps": 2 * nbytes / 1e9 / (i_ms * 1e-3)})
+                if 4 * nbytes <= 0.6 * free_b:
+                    b2, c2, d2_ = polys.clone(), polys.clone(), torch.empty_like(polys)
+                    m_ms = timed(lambda: ctx.poly_muladd(polys, b2, c2, d2_, batch))
+                    row["muladd_GBps"] = 4 * nbytes / 1e9 / (m_ms * 1e-3)
+                    del b2, c2, d2_
+                row["in_l2_or_launch_bound"] = bool(nbytes < 2 * 126e6 or batch * L < NUM_SMS)
+                for k_ in ("forward", "inverse", "muladd"):
+                    if k_ + "_GBps" in row:
+                        row[k_ + "_frac_of_hbm"] = row[k_ + "_GBps"] / peak
+                rows.append(row)
+                del polys
+                torch.cuda.empty_cache()
+            ctx.close()
+    print(json.dumps({"metric": METRIC, "unit": "GB/s", "config": {"workload": "kernel-sweep", "prime_bits": args.sweep_bits},
+                      "hbm_peak_GBps": peak, "peak_source": "of " + peak_kind, "dtype": "u64", "data": "synthetic",
+                      "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--config", type=int, default=2, help="round configuration 1..4 (default: MNIST-shaped)")
+    ap.add_argument("--config", type=int, default=2, help="round configuration 1..4 (default 2: MNIST-shaped); 5 = kernel sweep")
     ap.add_argument("--seed", type=int, default=1)
     ap.add_argument("--chunk", type=int, default=0, help="ciphertext indices per chunk (0: as many as fit)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep-bits", type=int, default=60, choices=[50, 60])
     args = ap.parse_args()
+    if args.config == 5:
+        return run_sweep(args)
     cfg = wl.round_config(args.config)
     if args.impl == "reference":
         run_reference(args, cfg)

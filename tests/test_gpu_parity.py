@@ -86,6 +86,47 @@ def test_poly_muladd_against_oracle(d2, log2_n, bits, L, batch):
     ctx.close()
 
 
+@pytest.mark.parametrize("log2_n", [12, 13, 14, 15, 16])
+def test_sweep_shapes_against_oracle(d2, log2_n):
+    """Kernel-sweep shapes: every L of the sweep at this N (60-bit primes), small batch."""
+    for L in wl.SWEEP_LIMBS:
+        moduli = wl.sweep_moduli(60, L)
+        ctx = d2.Context(log2_n, moduli, 1, seed=1)
+        o = make_oracle(log2_n, moduli, seed=1)
+        a = wl.random_polys(moduli, log2_n, 2, seed=L)
+        psi = [ctx.get_root(l) for l in range(L)]
+        dev = d2.from_u64_numpy(a, ctx.device)
+        ctx.ntt_forward(dev, 2)
+        perm = _brv(log2_n)
+        assert np.array_equal(d2.to_u64_numpy(dev), o.ntt(a, psi)[..., perm])
+        ctx.ntt_inverse(dev, 2)
+        assert np.array_equal(d2.to_u64_numpy(dev), a)
+        b, c = wl.random_polys(moduli, log2_n, 2, seed=50 + L), wl.random_polys(moduli, log2_n, 2, seed=90 + L)
+        db, dc = d2.from_u64_numpy(b, ctx.device), d2.from_u64_numpy(c, ctx.device)
+        ctx.poly_muladd(dev, db, dc, dev, 2)
+        assert np.array_equal(d2.to_u64_numpy(dev), o.poly_muladd(a, b, c))
+        ctx.close()
+
+
+def test_large_batch_transform_sampled_polynomials(d2):
+    """Batch 1024 x L 4 at N = 16384 and batch 256 at N = 65536: sampled polynomials against the oracle."""
+    for log2_n, batch in ((14, 1024), (16, 256)):
+        moduli = wl.sweep_moduli(50, 4)
+        ctx = d2.Context(log2_n, moduli, 1, seed=1)
+        o = make_oracle(log2_n, moduli, seed=1)
+        a = wl.random_polys(moduli, log2_n, batch, seed=3)
+        psi = [ctx.get_root(l) for l in range(4)]
+        dev = d2.from_u64_numpy(a, ctx.device)
+        ctx.ntt_forward(dev, batch)
+        got = d2.to_u64_numpy(dev)
+        perm = _brv(log2_n)
+        for r in (0, 1, batch // 3, batch - 1):
+            assert np.array_equal(got[r], o.ntt(a[r:r + 1], psi)[0][..., perm])
+        ctx.ntt_inverse(dev, batch)
+        assert np.array_equal(d2.to_u64_numpy(dev), a)
+        ctx.close()
+
+
 def test_ring_product_through_transforms_equals_schoolbook(d2):
     """INTT(NTT(a) . NTT(b)) = a*b in Z_p[X]/(X^N+1) for tiny N (definition by brute force)."""
     from oracle import d2mhe_oracle as orc
