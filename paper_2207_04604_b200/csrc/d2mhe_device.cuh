@@ -23,7 +23,8 @@ struct LimbTab {
   u64 half;                     // (q-1)/2 mod q_l
   u64 cq;                       // ceil(2^61 / q_l) * q_l: keeps Garner differences non-negative
   u64 mask;                     // 2^bitlen(q_l) - 1, for the rejection sampler
-  u64 rmod, rmod_sh;            // 2^64 mod q_l: leaves Montgomery form
+  u64 rmod, rmod_sh;            // 2^64 mod q_l: leaves Montgomery form; builds Shoup companions
+  u32 red_shift, red_mul;       // bitlen(q_l) - 1 and floor(2^(bitlen + 15) / q_l): small-quotient reduction
   const ulonglong2* W;          // [N] forward twiddles psi^brv(i) as {w, floor(w 2^64 / q_l)}
   const ulonglong2* IW;         // [N] their inverses
 };
@@ -219,10 +220,21 @@ __device__ __forceinline__ u64 shoup_approx(u64 y, u64 w, u64 ws, u64 np) {
 // are kept below 8p with one conditional subtraction per butterfly.
 struct Mod {
   u64 p, np, twop, fourp;
-  const u64 one_sh;
+  u32 red_shift, red_mul;
   __device__ __forceinline__ explicit Mod(const LimbTab& lt)
-      : p(lt.p), np(lt.np), twop(lt.twop), fourp(2 * lt.twop), one_sh(lt.one_sh) {}
+      : p(lt.p), np(lt.np), twop(lt.twop), fourp(2 * lt.twop), red_shift(lt.red_shift), red_mul(lt.red_mul) {}
 };
+
+// x - q p with q = floor(floor(x / 2^(b-1)) * floor(2^(b+15) / p) / 2^16), b = bitlen(p): q is
+// floor(x/p) or up to 2 below it, so the result is below 3p.  Needs x < 2^(b+8) (true for every
+// lazily grown value here: at most 128p).  One 32-bit, one widening and one low multiply.
+__device__ __forceinline__ u64 reduce_small(u64 x, const Mod& m) {
+  const u32 q = ((u32)(x >> m.red_shift) * m.red_mul) >> 16;
+  u32 nl, nh, rl, rh;
+  split64(m.np, nl, nh);
+  split64(madwide(q, nl, x), rl, rh);
+  return join64(rl, madlo(q, nh, rh));
+}
 
 // forward (Cooley-Tukey): (X, Y) -> (X + wY, X - wY)
 template <bool WIDE>
@@ -291,7 +303,7 @@ __device__ __forceinline__ void inv_octet(u64 (&x)[8], const ulonglong2* __restr
 #pragma unroll
     for (int k = 0; k < 4; ++k) gs_bfly<WIDE>(x[k], x[k + 4], w, md, c64);
   }
-  if (WIDE) x[0] = shoup_approx(x[0], 1, md.one_sh, md.np);
+  if (WIDE) x[0] = reduce_small(x[0], md);
 }
 
 // Brings the outputs of the last inverse round below 4p.  After a full round the bounds are
@@ -303,14 +315,14 @@ __device__ __forceinline__ void finish_octet(u64 (&x)[8], int nst, const Mod& md
     if (nst >= 3) {
       x[1] = csub(csub(x[1], md.fourp << 1), md.fourp);
     } else {
-      x[1] = shoup_approx(x[1], 1, md.one_sh, md.np);
+      x[1] = reduce_small(x[1], md);
     }
     if (nst >= 2) {
       x[2] = csub(x[2], md.fourp);
       x[3] = csub(x[3], md.fourp);
     } else {
-      x[2] = shoup_approx(x[2], 1, md.one_sh, md.np);
-      x[3] = shoup_approx(x[3], 1, md.one_sh, md.np);
+      x[2] = reduce_small(x[2], md);
+      x[3] = reduce_small(x[3], md);
     }
   }
 }

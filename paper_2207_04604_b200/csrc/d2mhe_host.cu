@@ -243,6 +243,8 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
     u32 bits = 0;
     for (u64 x = p; x; x >>= 1) ++bits;
     T.mask = bits >= 64 ? ~(u64)0 : (((u64)1 << bits) - 1);
+    T.red_shift = bits - 1;
+    T.red_mul = (u32)(((u128)1 << (bits + 15)) / p);
 
     const u64 psi = c->roots[l], psi_inv = h_inv(psi, p);
     std::vector<u64> pw(n), ipw(n);
