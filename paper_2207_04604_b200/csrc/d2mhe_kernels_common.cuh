@@ -14,7 +14,7 @@
 #define D2MHE_G13 2
 #endif
 #ifndef D2MHE_G14
-#define D2MHE_G14 4
+#define D2MHE_G14 2
 #endif
 #ifndef D2MHE_MINB12
 #define D2MHE_MINB12 4
