@@ -274,7 +274,13 @@ enum {
   TAG_ENC_U = 4,    /* mu             (Sec. 3.2 item 3)                 */
   TAG_ENC_E0 = 5,   /* e_0            (Sec. 3.2 item 3)                 */
   TAG_ENC_E1 = 6,   /* e_1            (Sec. 3.2 item 3)                 */
-  TAG_DEC_ERR = 7   /* e_{0,k} in a decryption share (Eq. 2)            */
+  TAG_DEC_ERR = 7,  /* e_{0,k} in a decryption share (Eq. 2)            */
+  TAG_USER_SECRET = 8,  /* sk_i of a user's own key pair (Algorithm 2, Require) */
+  TAG_USER_PK_ERR = 9,  /* e_i of pk_i                                   */
+  TAG_USER_P1 = 10,     /* p_{1,i} of pk_i                               */
+  TAG_CONV_MU = 11,     /* mu_k of MBFV.Convert (Eq. 2)                  */
+  TAG_CONV_E0 = 12,     /* e_{0,k} of MBFV.Convert                       */
+  TAG_CONV_E1 = 13      /* e_{1,k} of MBFV.Convert                       */
 };
 
 /*
@@ -321,16 +327,16 @@ static uint32_t bit_length(uint64_t x) {
  * its unmasked draw is reduced mod p.
  */
 static uint64_t uniform_mod(const orc_params* P, uint32_t tag, uint32_t j, uint32_t idx,
-                            uint64_t p) {
+                            uint32_t party, uint64_t p) {
   uint32_t bits = bit_length(p);
   uint64_t mask = bits >= 64 ? ~(uint64_t)0 : (((uint64_t)1 << bits) - 1);
   uint32_t w[4];
   for (uint32_t attempt = 0; attempt < 255; ++attempt) {
-    draw(P, tag, attempt, j, idx, 0, 0, w);
+    draw(P, tag, attempt, j, idx, party, 0, w);
     uint64_t r = (((uint64_t)w[0] << 32) | w[1]) & mask;
     if (r < p) return r;
   }
-  draw(P, tag, 255, j, idx, 0, 0, w);
+  draw(P, tag, 255, j, idx, party, 0, w);
   return (((uint64_t)w[0] << 32) | w[1]) % p;
 }
 
@@ -375,7 +381,7 @@ void orc_common_p1(const orc_params* P, uint64_t* p1 /*[L][N]*/) {
   uint32_t n = 1u << P->log2_n;
   for (uint32_t l = 0; l < P->num_limbs; ++l)
     for (uint32_t j = 0; j < n; ++j)
-      p1[(size_t)l * n + j] = uniform_mod(P, TAG_P1, j, l, P->moduli[l]);
+      p1[(size_t)l * n + j] = uniform_mod(P, TAG_P1, j, l, 0, P->moduli[l]);
 }
 
 static void small_to_limb(const int8_t* v, uint64_t* out, uint32_t n, uint64_t p) {
@@ -785,6 +791,133 @@ int orc_decrypt_single(const orc_params* P, const uint64_t* ct, const int32_t* s
   free(v);
   free(C);
   return status;
+}
+
+/* ------------------------------------------------------------------ */
+/* MBFV.Convert to a recipient's own key (Sec. 4.2 item 3, Eq. 2-3)    */
+/* ------------------------------------------------------------------ */
+
+/* sk_i of user i's own BFV key pair (Algorithm 2, Require): BFV.SecKeyGen. */
+void orc_user_secret(const orc_params* P, uint32_t user, int8_t* s) {
+  orc_sample_ternary(P, TAG_USER_SECRET, 0, user, 0, s);
+}
+
+/* pk_i = (-(sk_i p_{1,i} + e_i), p_{1,i}) (BFV.PubKeyGen, Sec. 3.2 item 2); pk is [2][L][N]. */
+void orc_user_pk(const orc_params* P, uint32_t user, uint64_t* pk) {
+  uint32_t n = 1u << P->log2_n, L = P->num_limbs;
+  size_t poly = (size_t)L * n;
+  int8_t* s = (int8_t*)malloc(n);
+  int8_t* e = (int8_t*)malloc(n);
+  uint64_t* sl = (uint64_t*)malloc(sizeof(uint64_t) * n);
+  uint64_t* prod = (uint64_t*)malloc(sizeof(uint64_t) * n);
+  orc_user_secret(P, user, s);
+  orc_sample_gauss(P, TAG_USER_PK_ERR, 0, user, 0, e);
+  for (uint32_t l = 0; l < L; ++l) {
+    uint64_t p = P->moduli[l];
+    uint64_t* p1 = pk + poly + (size_t)l * n;
+    for (uint32_t j = 0; j < n; ++j) p1[j] = uniform_mod(P, TAG_USER_P1, j, l, user, p);
+    small_to_limb(s, sl, n, p);
+    orc_ring_mul(p1, sl, prod, P->log2_n, p);
+    for (uint32_t j = 0; j < n; ++j)
+      pk[(size_t)l * n + j] = subm(0, addm(prod[j], lift(e[j], p), p), p);
+  }
+  free(s);
+  free(e);
+  free(sl);
+  free(prod);
+}
+
+/*
+ * Conversion share of party k for recipient i (Eq. 2):
+ *   (h_0, h_1) = (s_k c_1 + mu_k p_{0,i} + e_{0,k},  mu_k p_{1,i} + e_{1,k}),
+ * mu_k, e_{0,k}, e_{1,k} from chi on the stream (party, recipient, ct_index).
+ * pk_i is [2][L][N], c1 is [L][N], h is [2][L][N].
+ */
+void orc_convert_share(const orc_params* P, const uint64_t* pk_i, uint32_t party, uint32_t recipient,
+                       uint32_t ct_index, const uint64_t* c1, uint64_t* h) {
+  uint32_t n = 1u << P->log2_n, L = P->num_limbs;
+  size_t poly = (size_t)L * n;
+  int8_t* s = (int8_t*)malloc(n);
+  int8_t* mu = (int8_t*)malloc(n);
+  int8_t* e0 = (int8_t*)malloc(n);
+  int8_t* e1 = (int8_t*)malloc(n);
+  uint64_t* sl = (uint64_t*)malloc(sizeof(uint64_t) * n);
+  uint64_t* ml = (uint64_t*)malloc(sizeof(uint64_t) * n);
+  uint64_t* a = (uint64_t*)malloc(sizeof(uint64_t) * n);
+  uint64_t* b = (uint64_t*)malloc(sizeof(uint64_t) * n);
+  orc_secret_share(P, party, s);
+  orc_sample_gauss(P, TAG_CONV_MU, ct_index, party, recipient, mu);
+  orc_sample_gauss(P, TAG_CONV_E0, ct_index, party, recipient, e0);
+  orc_sample_gauss(P, TAG_CONV_E1, ct_index, party, recipient, e1);
+  for (uint32_t l = 0; l < L; ++l) {
+    uint64_t p = P->moduli[l];
+    small_to_limb(s, sl, n, p);
+    small_to_limb(mu, ml, n, p);
+    orc_ring_mul(sl, c1 + (size_t)l * n, a, P->log2_n, p);
+    orc_ring_mul(ml, pk_i + (size_t)l * n, b, P->log2_n, p);
+    for (uint32_t j = 0; j < n; ++j)
+      h[(size_t)l * n + j] = addm(addm(a[j], b[j], p), lift(e0[j], p), p);
+    orc_ring_mul(ml, pk_i + poly + (size_t)l * n, b, P->log2_n, p);
+    for (uint32_t j = 0; j < n; ++j) h[poly + (size_t)l * n + j] = addm(b[j], lift(e1[j], p), p);
+  }
+  free(s);
+  free(mu);
+  free(e0);
+  free(e1);
+  free(sl);
+  free(ml);
+  free(a);
+  free(b);
+}
+
+/* agg [n_rec][n_cts][2][L][N], pk_users [n_rec][2][L][N] -> shares [n_rec][n_parties][n_cts][2][L][N]. */
+void orc_convert_share_batch(const orc_params* P, const uint64_t* agg, const uint64_t* pk_users,
+                             const uint32_t* recipients, uint32_t n_rec, const uint32_t* parties,
+                             uint32_t n_parties, uint32_t ct_first, uint32_t n_cts, uint64_t* shares) {
+  uint32_t n = 1u << P->log2_n, L = P->num_limbs;
+  size_t poly = (size_t)L * n;
+  int64_t total = (int64_t)n_rec * n_parties * n_cts;
+#pragma omp parallel for schedule(dynamic)
+  for (int64_t u = 0; u < total; ++u) {
+    uint32_t c = (uint32_t)(u % n_cts);
+    uint32_t k = (uint32_t)((u / n_cts) % n_parties);
+    uint32_t i = (uint32_t)(u / ((int64_t)n_cts * n_parties));
+    const uint64_t* c1 = agg + (((size_t)i * n_cts + c) * 2 + 1) * poly;
+    orc_convert_share(P, pk_users + (size_t)i * 2 * poly, parties[k], recipients[i], ct_first + c, c1,
+                      shares + (size_t)u * 2 * poly);
+  }
+}
+
+/* ct' = (c_0 + sum_k h_{0,k}, sum_k h_{1,k}); out [n_rec][n_cts][2][L][N]. */
+void orc_convert_combine_batch(const orc_params* P, const uint64_t* agg, const uint64_t* shares,
+                               uint32_t n_rec, uint32_t n_shares, uint32_t n_cts, uint64_t* out) {
+  uint32_t n = 1u << P->log2_n, L = P->num_limbs;
+  size_t poly = (size_t)L * n;
+#pragma omp parallel for schedule(dynamic)
+  for (int64_t u = 0; u < (int64_t)n_rec * n_cts; ++u) {
+    uint32_t i = (uint32_t)(u / n_cts), c = (uint32_t)(u % n_cts);
+    for (uint32_t comp = 0; comp < 2; ++comp)
+      for (uint32_t l = 0; l < L; ++l)
+        for (uint32_t j = 0; j < n; ++j) {
+          size_t o = ((size_t)comp * L + l) * n + j;
+          uint64_t acc = comp == 0 ? agg[(size_t)u * 2 * poly + o] % P->moduli[l] : 0;
+          for (uint32_t k = 0; k < n_shares; ++k)
+            acc = addm(acc, shares[(((size_t)i * n_shares + k) * n_cts + c) * 2 * poly + o], P->moduli[l]);
+          out[(size_t)u * 2 * poly + o] = acc;
+        }
+  }
+}
+
+/* BFV.Decrypt of ct [n][n_cts][2][L][N] with explicit small secrets [n][N] -> plain [n][n_cts][N]. */
+void orc_decrypt_batch(const orc_params* P, const uint64_t* ct, const int32_t* secrets, uint32_t n_users,
+                       uint32_t n_cts, uint32_t* plain) {
+  uint32_t n = 1u << P->log2_n, L = P->num_limbs;
+  size_t poly = (size_t)L * n;
+#pragma omp parallel for schedule(dynamic)
+  for (int64_t u = 0; u < (int64_t)n_users * n_cts; ++u) {
+    uint32_t i = (uint32_t)(u / n_cts);
+    orc_decrypt_single(P, ct + (size_t)u * 2 * poly, secrets + (size_t)i * n, plain + (size_t)u * n, NULL);
+  }
 }
 
 /* ------------------------------------------------------------------ */

@@ -286,6 +286,44 @@ class Oracle:
                                 ctypes.c_uint32(shares.shape[1]), ctypes.c_uint32(n_cts), _p(plain))
         return plain
 
+    # MBFV.Convert to a recipient's own key (Sec. 4.2 item 3)
+    def user_secret(self, user):
+        out = np.empty(self.n, dtype=np.int8)
+        lib().orc_user_secret(self._ref, ctypes.c_uint32(user), _p(out))
+        return out
+
+    def user_pk(self, user):
+        out = np.empty((2, self.num_limbs, self.n), dtype=np.uint64)
+        lib().orc_user_pk(self._ref, ctypes.c_uint32(user), _p(out))
+        return out
+
+    def convert_share(self, agg, pk_users, recipients, parties, ct_first):
+        """agg [n_rec, n_cts, 2, L, N], pk_users [n_rec, 2, L, N] -> [n_rec, n_parties, n_cts, 2, L, N]."""
+        agg, pk_users = _u64(agg), _u64(pk_users)
+        recipients, parties = _u32(recipients), _u32(parties)
+        n_rec, n_cts = agg.shape[0], agg.shape[1]
+        shares = np.empty((n_rec, parties.size, n_cts, 2, self.num_limbs, self.n), dtype=np.uint64)
+        lib().orc_convert_share_batch(self._ref, _p(agg), _p(pk_users), _p(recipients), ctypes.c_uint32(n_rec),
+                                      _p(parties), ctypes.c_uint32(parties.size), ctypes.c_uint32(ct_first),
+                                      ctypes.c_uint32(n_cts), _p(shares))
+        return shares
+
+    def convert_combine(self, agg, shares):
+        agg, shares = _u64(agg), _u64(shares)
+        out = np.empty_like(agg)
+        lib().orc_convert_combine_batch(self._ref, _p(agg), _p(shares), ctypes.c_uint32(agg.shape[0]),
+                                        ctypes.c_uint32(shares.shape[1]), ctypes.c_uint32(agg.shape[1]), _p(out))
+        return out
+
+    def decrypt(self, ct, secrets):
+        """ct [n, n_cts, 2, L, N], secrets int [n, N] -> plain [n, n_cts, N]."""
+        ct = _u64(ct)
+        secrets = np.ascontiguousarray(secrets, dtype=np.int32)
+        plain = np.empty((ct.shape[0], ct.shape[1], self.n), dtype=np.uint32)
+        lib().orc_decrypt_batch(self._ref, _p(ct), _p(secrets), ctypes.c_uint32(ct.shape[0]),
+                                ctypes.c_uint32(ct.shape[1]), _p(plain))
+        return plain
+
     def decrypt_single(self, ct, s, want_noise=False):
         """BFV.Decrypt of one ciphertext [2, L, N] under an explicit integer secret s[N]."""
         ct = _u64(ct)

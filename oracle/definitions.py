@@ -93,6 +93,15 @@ def decryption_share(c1, s_k, e_k, q):
     return poly_add(negacyclic_mul(c1, [x % q for x in s_k], q), [x % q for x in e_k], q)
 
 
+def convert_share(c1, s_k, mu_k, e0_k, e1_k, p0_i, p1_i, q):
+    """(h_0, h_1) = (s_k c1 + mu_k p_{0,i} + e_{0,k}, mu_k p_{1,i} + e_{1,k})   (Eq. 2)."""
+    mu = [x % q for x in mu_k]
+    h0 = poly_add(poly_add(negacyclic_mul(c1, [x % q for x in s_k], q), negacyclic_mul(mu, p0_i, q), q),
+                  [x % q for x in e0_k], q)
+    h1 = poly_add(negacyclic_mul(mu, p1_i, q), [x % q for x in e1_k], q)
+    return h0, h1
+
+
 def combine(c0, shares, q, t):
     """[ round( t/q * [c0 + sum_k h_k]_q ) ]_t   (Sec. 4.2 item 3, Eq. 3; Sec. 3.2 item 5)."""
     v = list(c0)
