@@ -152,6 +152,37 @@ d2mhe_status d2mhe_combine_decrypt(d2mhe_ctx* ctx, const uint64_t* agg_dev,
                                    uint32_t n_shares, uint32_t n_cts, uint32_t* plain_dev);
 
 /*
+ * MBFV.Convert (Sec. 4.2 item 3, Eq. 2-3; Algorithm 2 lines 8-9): re-encryption of an aggregate
+ * from the collective key to the recipient's OWN key pair, followed by BFV.Decrypt under it.
+ *
+ * d2mhe_user_keygen: every listed user i generates sk_i <- R_3 and
+ *   pk_i = (-(sk_i p_{1,i} + e_i), p_{1,i}), p_{1,i} uniform, e_i from chi (Algorithm 2, Require;
+ *   Sec. 3.2 items 1-2).  pk_out_dev: optional out [n_users, 2, L, N].
+ * d2mhe_convert_share: shares[i, a, c] = (h_0, h_1) =
+ *   (s_k c_1 + mu_k p_{0,i} + e_{0,k},  mu_k p_{1,i} + e_{1,k}),  k = parties[a], i = recipients[i],
+ *   mu_k, e_{0,k}, e_{1,k} from chi (the paper draws mu_k from chi) on the stream
+ *   (party k, recipient i, ciphertext index ct_first + c).  Recipients need own keys, parties key shares.
+ *   agg_dev: [n_rec, n_cts, 2, L, N];  shares_dev: out [n_rec, n_parties, n_cts, 2, L, N].
+ * d2mhe_convert_combine: ct'[i, c] = (c_0 + sum_k h_{0,k}, sum_k h_{1,k}); n_shares must equal the
+ *   size of the collective key's party set.  ct_out_dev: out [n_rec, n_cts, 2, L, N].
+ * d2mhe_decrypt: BFV.Decrypt(sk_i, ct) (Sec. 3.2 item 5) for users[i] on ct_dev [n_users, n_cts, 2, L, N];
+ *   scratch_dev: caller-provided [n_users, n_cts, L, N] uint64 (receives c_1 sk_i);
+ *   plain_dev: out [n_users, n_cts, N] in [0,t).
+ * users, recipients, parties: HOST arrays.
+ */
+d2mhe_status d2mhe_user_keygen(d2mhe_ctx* ctx, const uint32_t* users, uint32_t n_users,
+                               uint64_t* pk_out_dev);
+d2mhe_status d2mhe_convert_share(d2mhe_ctx* ctx, const uint64_t* agg_dev, const uint32_t* recipients,
+                                 uint32_t n_rec, const uint32_t* parties, uint32_t n_parties,
+                                 uint32_t ct_first, uint32_t n_cts, uint64_t* shares_dev);
+d2mhe_status d2mhe_convert_combine(d2mhe_ctx* ctx, const uint64_t* agg_dev, const uint64_t* shares_dev,
+                                   uint32_t n_rec, uint32_t n_shares, uint32_t n_cts,
+                                   uint64_t* ct_out_dev);
+d2mhe_status d2mhe_decrypt(d2mhe_ctx* ctx, const uint32_t* users, uint32_t n_users,
+                           const uint64_t* ct_dev, uint32_t n_cts, uint64_t* scratch_dev,
+                           uint32_t* plain_dev);
+
+/*
  * Batched negacyclic number-theoretic transform of [batch, L, N], in place.
  * Forward: position p of limb l receives a(psi_l^(2 brv(p) + 1)), brv = reversal of
  * the log2_n-bit index, psi_l the root reported by d2mhe_get_root.  Inverse undoes it.
@@ -217,6 +248,8 @@ d2mhe_status d2mhe_round_device_static(d2mhe_ctx* ctx, const int32_t* values_dev
 /* Test hooks. */
 /* s_k as int8 [N] on the HOST (needs a key share for `party`). */
 d2mhe_status d2mhe_debug_export_secret(d2mhe_ctx* ctx, uint32_t party, int8_t* s_host);
+/* sk_i of a user's own key pair as int8 [N] on the HOST (needs d2mhe_user_keygen for `user`). */
+d2mhe_status d2mhe_debug_export_user_secret(d2mhe_ctx* ctx, uint32_t user, int8_t* s_host);
 /* The primitive 2N-th root of unity used for limb `limb`. */
 d2mhe_status d2mhe_get_root(const d2mhe_ctx* ctx, uint32_t limb, uint64_t* psi);
 /* psi_t, the slot root (D2MHE_ERR_UNSUPPORTED if t != 1 mod 2N). */

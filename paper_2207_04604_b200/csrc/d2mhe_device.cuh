@@ -93,7 +93,13 @@ enum : u32 {
   TAG_ENC_U = 4,
   TAG_ENC_E0 = 5,
   TAG_ENC_E1 = 6,
-  TAG_DEC_ERR = 7
+  TAG_DEC_ERR = 7,
+  TAG_USER_SECRET = 8,
+  TAG_USER_PK_ERR = 9,
+  TAG_USER_P1 = 10,
+  TAG_CONV_MU = 11,
+  TAG_CONV_E0 = 12,
+  TAG_CONV_E1 = 13
 };
 
 // One stream: counter = (j, idx, party | recipient << 16, tag | attempt << 8).

@@ -353,6 +353,12 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   if (err != cudaSuccess) return fail_cuda(c, err);
   c->view.pk_coef = dev_alloc<u64>(c, 2 * poly, &err);
   if (err != cudaSuccess) return fail_cuda(c, err);
+  c->view.usk_mont = dev_alloc<u64>(c, (size_t)P.num_parties * poly, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  c->view.upk_mont = dev_alloc<u64>(c, (size_t)P.num_parties * 2 * poly, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  c->view.upk_coef = dev_alloc<u64>(c, (size_t)P.num_parties * 2 * poly, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
   c->view.range_flag = dev_alloc<u32>(c, 4, &err);
   if (err != cudaSuccess) return fail_cuda(c, err);
   err = cudaMemset(c->view.range_flag, 0, 16);
@@ -430,6 +436,7 @@ d2mhe_status d2mhe_create(const d2mhe_params* P, d2mhe_ctx** out) {
   c->device = P->device;
   c->can_pack = (t - 1) % two_n == 0;
   c->has_share.assign(P->num_parties, false);
+  c->has_user_key.assign(P->num_parties, false);
   std::memset(&c->view, 0, sizeof(c->view));
   std::memset(&c->limb_params, 0, sizeof(c->limb_params));
   for (u32 l = 0; l < P->num_limbs; ++l) {
@@ -679,6 +686,104 @@ d2mhe_status d2mhe_poly_muladd(d2mhe_ctx* c, const uint64_t* a, const uint64_t* 
   return D2MHE_OK;
 }
 
+// ---- MBFV.Convert to a recipient's own key ---------------------------------------------
+
+d2mhe_status d2mhe_user_keygen(d2mhe_ctx* c, const u32* users, u32 n_users, uint64_t* pk_out_dev) {
+  if (!c) return D2MHE_ERR_INVALID_ARG;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  d2mhe_status st = check_party_list(c, users, n_users, false, true);
+  if (st != D2MHE_OK) return st;
+  if (!aligned16(pk_out_dev)) return D2MHE_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[1] = {users};
+  const size_t counts[1] = {n_users};
+  if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::user_keygen(c->view, c->limb_params, c->stream, sg.dev[0], n_users);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  const size_t pk_words = 2 * (size_t)c->view.L * c->view.n;
+  if (pk_out_dev) {
+    for (u32 i = 0; i < n_users; ++i) {
+      e = cudaMemcpyAsync(pk_out_dev + (size_t)i * pk_words, c->view.upk_coef + (size_t)users[i] * pk_words,
+                          pk_words * sizeof(u64), cudaMemcpyDeviceToDevice, c->stream);
+      if (e != cudaSuccess) return fail_cuda(c, e);
+    }
+  }
+  for (u32 i = 0; i < n_users; ++i) c->has_user_key[users[i]] = true;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_convert_share(d2mhe_ctx* c, const uint64_t* agg_dev, const u32* recipients, u32 n_rec,
+                                 const u32* parties, u32 n_parties, u32 ct_first, u32 n_cts,
+                                 uint64_t* shares_dev) {
+  if (!c || !agg_dev || !shares_dev || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(agg_dev) || !aligned16(shares_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  d2mhe_status st = check_party_list(c, recipients, n_rec, false, false);
+  if (st != D2MHE_OK) return st;
+  for (u32 i = 0; i < n_rec; ++i)
+    if (!c->has_user_key[recipients[i]]) return D2MHE_ERR_STATE;
+  st = check_party_list(c, parties, n_parties, true, true);
+  if (st != D2MHE_OK) return st;
+  if ((u64)ct_first + n_cts > 0xffffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)n_rec * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[2] = {recipients, parties};
+  const size_t counts[2] = {n_rec, n_parties};
+  if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::convert_share(c->view, c->limb_params, c->stream,
+                                              reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1],
+                                              n_parties, ct_first, n_cts, reinterpret_cast<u64*>(shares_dev));
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_convert_combine(d2mhe_ctx* c, const uint64_t* agg_dev, const uint64_t* shares_dev,
+                                   u32 n_rec, u32 n_shares, u32 n_cts, uint64_t* ct_out_dev) {
+  if (!c || !agg_dev || !shares_dev || !ct_out_dev || n_rec == 0 || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(agg_dev) || !aligned16(shares_dev) || !aligned16(ct_out_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!c->has_pk) return D2MHE_ERR_STATE;
+  if (n_shares != c->pk_parties.size()) return D2MHE_ERR_INVALID_ARG;
+  if ((u64)n_rec * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  cudaError_t e = d2mhe_launch::convert_combine(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
+                                                reinterpret_cast<const u64*>(shares_dev), n_rec, n_shares, n_cts,
+                                                reinterpret_cast<u64*>(ct_out_dev));
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_decrypt(d2mhe_ctx* c, const u32* users, u32 n_users, const uint64_t* ct_dev, u32 n_cts,
+                           uint64_t* scratch_dev, u32* plain_dev) {
+  if (!c || !ct_dev || !scratch_dev || !plain_dev || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(ct_dev) || !aligned16(scratch_dev) || !aligned16(plain_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  d2mhe_status st = check_party_list(c, users, n_users, false, false);
+  if (st != D2MHE_OK) return st;
+  for (u32 i = 0; i < n_users; ++i)
+    if (!c->has_user_key[users[i]]) return D2MHE_ERR_STATE;
+  if ((u64)n_users * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[1] = {users};
+  const size_t counts[1] = {n_users};
+  if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::secret_product(c->view, c->limb_params, c->stream,
+                                               reinterpret_cast<const u64*>(ct_dev), sg.dev[0], n_users, n_cts,
+                                               reinterpret_cast<u64*>(scratch_dev));
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  // [c_0 + c_1 sk_i]_q then the exact scale-and-round: the product plays the role of one share
+  e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(ct_dev),
+                            reinterpret_cast<const u64*>(scratch_dev), n_users, 1, n_cts, plain_dev);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 2;
+  return release_slot(c, sg);
+}
+
 // ---- whole round ---------------------------------------------------------------------
 
 // Per ciphertext index of a chunk: plain K*N u32, ct and agg K*2*L*N u64 each,
@@ -777,6 +882,15 @@ d2mhe_status d2mhe_debug_export_secret(d2mhe_ctx* c, u32 party, int8_t* s_host) 
   if (party >= c->params.num_parties) return D2MHE_ERR_RANGE;
   if (!c->has_share[party]) return D2MHE_ERR_STATE;
   const Stream st(c->params.seed, TAG_SECRET, 0, party, 0);
+  for (u32 j = 0; j < c->view.n; ++j) s_host[j] = (int8_t)st.ternary(j);
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_debug_export_user_secret(d2mhe_ctx* c, u32 user, int8_t* s_host) {
+  if (!c || !s_host) return D2MHE_ERR_INVALID_ARG;
+  if (user >= c->params.num_parties) return D2MHE_ERR_RANGE;
+  if (!c->has_user_key[user]) return D2MHE_ERR_STATE;
+  const Stream st(c->params.seed, TAG_USER_SECRET, 0, user, 0);
   for (u32 j = 0; j < c->view.n; ++j) s_host[j] = (int8_t)st.ternary(j);
   return D2MHE_OK;
 }

@@ -46,6 +46,9 @@ struct DevView {
   u64* s_mont;   // [K][L][N]  NTT(s_k) * N^-1 in Montgomery form
   u64* pk_mont;  // [2][L][N]  NTT(p_0), NTT(p_1) * N^-1 in Montgomery form
   u64* pk_coef;  // [2][L][N]  (p_0, p_1), coefficient domain
+  u64* usk_mont;  // [K][L][N]     NTT(sk_i) * N^-1 (Montgomery form) of the users' own keys
+  u64* upk_mont;  // [K][2][L][N]  NTT(p_{0,i}), NTT(p_{1,i}) * N^-1 (Montgomery form)
+  u64* upk_coef;  // [K][2][L][N]  pk_i, coefficient domain
   u32* range_flag;
 };
 
@@ -69,6 +72,7 @@ struct d2mhe_ctx {
   LimbParams limb_params;
   std::vector<void*> allocs;        // device allocations to free
   std::vector<bool> has_share;
+  std::vector<bool> has_user_key;
   std::vector<u32> pk_parties;      // party set of the last collective_pk
   bool has_pk = false;
   u64 launches = 0;
@@ -97,6 +101,15 @@ cudaError_t partial_decrypt(const DevView& v, const LimbParams& lp, cudaStream_t
 cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
                     u32 n_shares, u32 n_cts, u32* plain);
 cudaError_t ntt(const DevView& v, const LimbParams& lp, cudaStream_t s, u64* polys, u32 batch, bool inverse);
+cudaError_t user_keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* users_dev,
+                        u32 n_users);
+cudaError_t convert_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
+                          const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties,
+                          u32 ct_first, u32 n_cts, u64* shares);
+cudaError_t convert_combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
+                            u32 n_shares, u32 n_cts, u64* out);
+cudaError_t secret_product(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* ct,
+                           const u32* users_dev, u32 n_users, u32 n_cts, u64* prod);
 cudaError_t muladd(const DevView& v, cudaStream_t s, const u64* a, const u64* b, const u64* c,
                    u64* d, u32 batch);
 // number of kernel launches the call above performed (for bookkeeping)

@@ -28,7 +28,8 @@ EXPORTS = [
     "d2mhe_keygen_share", "d2mhe_collective_pk", "d2mhe_encode", "d2mhe_decode", "d2mhe_encrypt",
     "d2mhe_aggregate", "d2mhe_partial_decrypt", "d2mhe_combine_decrypt", "d2mhe_ntt_forward",
     "d2mhe_ntt_inverse", "d2mhe_poly_muladd", "d2mhe_round_workspace_bytes", "d2mhe_round_device",
-    "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_debug_export_secret", "d2mhe_get_root", "d2mhe_get_plain_root",
+    "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_user_keygen", "d2mhe_convert_share",
+    "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_get_root", "d2mhe_get_plain_root",
     "d2mhe_launch_count",
 ]
 
@@ -91,6 +92,11 @@ def load():
         lib.d2mhe_round_host.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp, sz]
         lib.d2mhe_round_device_static.argtypes = [vp, vp, u32, u32, vp, vp, vp]
         lib.d2mhe_debug_export_secret.argtypes = [vp, u32, vp]
+        lib.d2mhe_debug_export_user_secret.argtypes = [vp, u32, vp]
+        lib.d2mhe_user_keygen.argtypes = [vp, vp, u32, vp]
+        lib.d2mhe_convert_share.argtypes = [vp, vp, vp, u32, vp, u32, u32, u32, vp]
+        lib.d2mhe_convert_combine.argtypes = [vp, vp, vp, u32, u32, u32, vp]
+        lib.d2mhe_decrypt.argtypes = [vp, vp, u32, vp, u32, vp, vp]
         lib.d2mhe_get_root.argtypes = [vp, u32, ctypes.POINTER(u64)]
         lib.d2mhe_get_plain_root.argtypes = [vp, ctypes.POINTER(u64)]
         lib.d2mhe_launch_count.argtypes = [vp]
@@ -258,6 +264,32 @@ class Context:
         self._check(load().d2mhe_round_host(self._h, ctypes.c_void_p(values_host.data_ptr()), ct_first, n_cts, offp,
                                             rowsp, ctypes.c_void_p(sums_host.data_ptr()), _dev(workspace),
                                             workspace.numel() * workspace.element_size()), "d2mhe_round_host")
+
+    # ---- conversion to the recipient's own key ----
+    def user_keygen(self, users, pk_out=None):
+        arr, ptr = _host_u32(users)
+        self._check(load().d2mhe_user_keygen(self._h, ptr, arr.size, _dev(pk_out, U64)), "d2mhe_user_keygen")
+
+    def convert_share(self, agg, recipients, parties, ct_first, n_cts, shares):
+        rec, recp = _host_u32(recipients)
+        par, parp = _host_u32(parties)
+        self._check(load().d2mhe_convert_share(self._h, _dev(agg, U64), recp, rec.size, parp, par.size, ct_first,
+                                               n_cts, _dev(shares, U64)), "d2mhe_convert_share")
+
+    def convert_combine(self, agg, shares, n_rec, n_shares, n_cts, ct_out):
+        self._check(load().d2mhe_convert_combine(self._h, _dev(agg, U64), _dev(shares, U64), n_rec, n_shares, n_cts,
+                                                 _dev(ct_out, U64)), "d2mhe_convert_combine")
+
+    def decrypt(self, users, ct, n_cts, scratch, plain):
+        arr, ptr = _host_u32(users)
+        self._check(load().d2mhe_decrypt(self._h, ptr, arr.size, _dev(ct, U64), n_cts, _dev(scratch, U64),
+                                         _dev(plain, U32)), "d2mhe_decrypt")
+
+    def debug_export_user_secret(self, user):
+        out = np.empty(self.n, dtype=np.int8)
+        self._check(load().d2mhe_debug_export_user_secret(self._h, user, out.ctypes.data_as(ctypes.c_void_p)),
+                    "d2mhe_debug_export_user_secret")
+        return out
 
     # ---- test hooks ----
     def debug_export_secret(self, party):

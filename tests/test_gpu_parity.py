@@ -349,6 +349,74 @@ def test_large_configs_on_sampled_ciphertext_indices(d2, index, sample):
 
 
 # ----------------------------------------------------------------------------------
+# conversion to the recipient's own key (MBFV.Convert) and decryption under it
+# ----------------------------------------------------------------------------------
+
+
+@pytest.mark.parametrize("log2_n,moduli_spec,K,n_cts", [
+    (4, (30, 2), 3, 2), (6, (54, 3), 2, 1), (9, (60, 2), 3, 2), (12, None, 4, 2), (13, (54, 4), 3, 1), (14, (54, 5), 2, 1),
+])
+def test_convert_every_message(d2, log2_n, moduli_spec, K, n_cts):
+    if moduli_spec is None:
+        moduli = wl.round_config(1).moduli
+    else:
+        moduli = small_moduli(log2_n, *moduli_spec)
+    seed = 31 + log2_n
+    L, n = len(moduli), 1 << log2_n
+    ctx = d2.Context(log2_n, moduli, K, seed=seed)
+    o = make_oracle(log2_n, moduli, seed=seed)
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    pk = o.collective_pk(parties)
+    rng = np.random.default_rng(seed)
+    values = rng.integers(-4000, 4001, size=(K, n_cts, n)).astype(np.int32)
+    offsets = np.array([0, K, K + 1], dtype=np.uint32)
+    rows = np.array(parties + [0], dtype=np.uint32)
+    want_ct = o.encrypt(pk, parties, 7, o.encode(values))
+    want_agg = o.aggregate(want_ct, offsets, rows)
+    agg = d2.from_u64_numpy(want_agg, ctx.device)
+    recipients = [K - 1, 0]
+    # own key pairs
+    pk_users = ctx.empty_u64(2, 2, L, n)
+    ctx.user_keygen(recipients, pk_users)
+    ctx.sync()
+    want_pk_users = np.stack([o.user_pk(i) for i in recipients])
+    assert np.array_equal(d2.to_u64_numpy(pk_users), want_pk_users)
+    for i in recipients:
+        assert np.array_equal(ctx.debug_export_user_secret(i), o.user_secret(i))
+    # shares
+    shares = ctx.empty_u64(2, K, n_cts, 2, L, n)
+    ctx.convert_share(agg, recipients, parties, 7, n_cts, shares)
+    want_shares = o.convert_share(want_agg, want_pk_users, recipients, parties, 7)
+    assert np.array_equal(d2.to_u64_numpy(shares), want_shares)
+    # combination
+    conv = ctx.empty_u64(2, n_cts, 2, L, n)
+    ctx.convert_combine(agg, shares, 2, K, n_cts, conv)
+    want_conv = o.convert_combine(want_agg, want_shares)
+    assert np.array_equal(d2.to_u64_numpy(conv), want_conv)
+    # decryption under the recipients' own keys
+    scratch = ctx.empty_u64(2, n_cts, L, n)
+    plain = ctx.empty_u32(2, n_cts, n)
+    ctx.decrypt(recipients, conv, n_cts, scratch, plain)
+    secrets = np.stack([o.user_secret(i).astype(np.int32) for i in recipients])
+    want_plain = o.decrypt(want_conv, secrets)
+    assert np.array_equal(d2.to_u32_numpy(plain), want_plain)
+    sums = torch.empty((2, n_cts, n), dtype=torch.int32, device=ctx.device)
+    ctx.decode(plain, 2 * n_cts, sums)
+    ctx.sync()
+    got = sums.cpu().numpy()
+    assert np.array_equal(got[0], values.astype(np.int64).sum(axis=0))
+    assert np.array_equal(got[1], values[0])
+    # a recipient without an own key pair is refused
+    if K > 2:
+        with pytest.raises(d2.D2mheError) as e:
+            ctx.convert_share(agg, [1, 0], parties, 7, n_cts, shares)
+        assert e.value.status == d2.ERR_STATE
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------------
 # whole-round driver, chunking, determinism, error paths
 # ----------------------------------------------------------------------------------
 
