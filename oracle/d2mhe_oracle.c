@@ -280,7 +280,11 @@ enum {
   TAG_USER_P1 = 10,     /* p_{1,i} of pk_i                               */
   TAG_CONV_MU = 11,     /* mu_k of MBFV.Convert (Eq. 2)                  */
   TAG_CONV_E0 = 12,     /* e_{0,k} of MBFV.Convert                       */
-  TAG_CONV_E1 = 13      /* e_{1,k} of MBFV.Convert                       */
+  TAG_CONV_E1 = 13,     /* e_{1,k} of MBFV.Convert                       */
+  TAG_BOOT_ALPHA = 14,  /* common polynomial alpha of MBFV.Bootstrap      */
+  TAG_BOOT_MASK = 15,   /* M_k over R_t (Eq. 4)                          */
+  TAG_BOOT_E0 = 16,     /* e_{0,k} of MBFV.Bootstrap                     */
+  TAG_BOOT_E1 = 17      /* e_{1,k} of MBFV.Bootstrap                     */
 };
 
 /*
@@ -917,6 +921,164 @@ void orc_decrypt_batch(const orc_params* P, const uint64_t* ct, const int32_t* s
   for (int64_t u = 0; u < (int64_t)n_users * n_cts; ++u) {
     uint32_t i = (uint32_t)(u / n_cts);
     orc_decrypt_single(P, ct + (size_t)u * 2 * poly, secrets + (size_t)i * n, plain + (size_t)u * n, NULL);
+  }
+}
+
+/* ------------------------------------------------------------------ */
+/* MBFV.Bootstrap (Sec. 4.2 item 4, Eq. 4)                             */
+/* ------------------------------------------------------------------ */
+
+/* The common random polynomial alpha for (recipient, ct_index): uniform on R_q, limb by limb.
+ * Counter: (j, ct_index, limb | recipient << 16, tag | attempt << 8). */
+void orc_boot_alpha(const orc_params* P, uint32_t recipient, uint32_t ct_index, uint64_t* alpha) {
+  uint32_t n = 1u << P->log2_n;
+  for (uint32_t l = 0; l < P->num_limbs; ++l) {
+    uint64_t p = P->moduli[l];
+    uint32_t bits = bit_length(p);
+    uint64_t mask = (((uint64_t)1 << bits) - 1);
+    for (uint32_t j = 0; j < n; ++j) {
+      uint32_t w[4];
+      uint64_t val = 0;
+      int done = 0;
+      for (uint32_t attempt = 0; attempt < 255 && !done; ++attempt) {
+        draw(P, TAG_BOOT_ALPHA, attempt, j, ct_index, l, recipient, w);
+        uint64_t r = (((uint64_t)w[0] << 32) | w[1]) & mask;
+        if (r < p) {
+          val = r;
+          done = 1;
+        }
+      }
+      if (!done) {
+        draw(P, TAG_BOOT_ALPHA, 255, j, ct_index, l, recipient, w);
+        val = (((uint64_t)w[0] << 32) | w[1]) % p;
+      }
+      alpha[(size_t)l * n + j] = val;
+    }
+  }
+}
+
+/* M_k uniform over R_t: rejection on bitlen(t)-bit draws, stream (party, recipient, ct_index). */
+void orc_boot_mask(const orc_params* P, uint32_t party, uint32_t recipient, uint32_t ct_index,
+                   uint32_t* mask_out) {
+  uint32_t n = 1u << P->log2_n;
+  uint64_t t = P->plain_modulus;
+  uint64_t m = (((uint64_t)1 << bit_length(t)) - 1);
+  for (uint32_t j = 0; j < n; ++j) {
+    uint32_t w[4];
+    uint64_t val = 0;
+    int done = 0;
+    for (uint32_t attempt = 0; attempt < 255 && !done; ++attempt) {
+      draw(P, TAG_BOOT_MASK, attempt, j, ct_index, party, recipient, w);
+      uint64_t r = (((uint64_t)w[0] << 32) | w[1]) & m;
+      if (r < t) {
+        val = r;
+        done = 1;
+      }
+    }
+    if (!done) {
+      draw(P, TAG_BOOT_MASK, 255, j, ct_index, party, recipient, w);
+      val = (((uint64_t)w[0] << 32) | w[1]) % t;
+    }
+    mask_out[j] = (uint32_t)val;
+  }
+}
+
+/*
+ * Bootstrap share of party k (Eq. 4):
+ *   (eta_0, eta_1) = (s_k c_1 - Lambda M_k + e_{0,k},  -s_k alpha + Lambda M_k + e_{1,k}).
+ * c1, alpha are [L][N]; eta is [2][L][N].
+ */
+void orc_boot_share(const orc_params* P, uint32_t party, uint32_t recipient, uint32_t ct_index,
+                    const uint64_t* c1, const uint64_t* alpha, uint64_t* eta) {
+  uint32_t n = 1u << P->log2_n, L = P->num_limbs;
+  size_t poly = (size_t)L * n;
+  int8_t* s = (int8_t*)malloc(n);
+  int8_t* e0 = (int8_t*)malloc(n);
+  int8_t* e1 = (int8_t*)malloc(n);
+  uint32_t* mk = (uint32_t*)malloc(sizeof(uint32_t) * n);
+  uint64_t* sl = (uint64_t*)malloc(sizeof(uint64_t) * n);
+  uint64_t* a = (uint64_t*)malloc(sizeof(uint64_t) * n);
+  uint64_t delta[ORC_MAX_LIMBS];
+  orc_delta(P, delta);
+  orc_secret_share(P, party, s);
+  orc_boot_mask(P, party, recipient, ct_index, mk);
+  orc_sample_gauss(P, TAG_BOOT_E0, ct_index, party, recipient, e0);
+  orc_sample_gauss(P, TAG_BOOT_E1, ct_index, party, recipient, e1);
+  for (uint32_t l = 0; l < L; ++l) {
+    uint64_t p = P->moduli[l];
+    small_to_limb(s, sl, n, p);
+    orc_ring_mul(sl, c1 + (size_t)l * n, a, P->log2_n, p);
+    for (uint32_t j = 0; j < n; ++j) {
+      uint64_t dm = mulm(delta[l], mk[j] % p, p);
+      eta[(size_t)l * n + j] = addm(subm(a[j], dm, p), lift(e0[j], p), p);
+    }
+    orc_ring_mul(sl, alpha + (size_t)l * n, a, P->log2_n, p);
+    for (uint32_t j = 0; j < n; ++j) {
+      uint64_t dm = mulm(delta[l], mk[j] % p, p);
+      eta[poly + (size_t)l * n + j] = addm(addm(subm(0, a[j], p), dm, p), lift(e1[j], p), p);
+    }
+  }
+  free(s);
+  free(e0);
+  free(e1);
+  free(mk);
+  free(sl);
+  free(a);
+}
+
+/* agg [n_rec][n_cts][2][L][N] -> shares [n_rec][n_parties][n_cts][2][L][N]. */
+void orc_boot_share_batch(const orc_params* P, const uint64_t* agg, const uint32_t* recipients,
+                          uint32_t n_rec, const uint32_t* parties, uint32_t n_parties,
+                          uint32_t ct_first, uint32_t n_cts, uint64_t* shares) {
+  uint32_t n = 1u << P->log2_n, L = P->num_limbs;
+  size_t poly = (size_t)L * n;
+  int64_t total = (int64_t)n_rec * n_parties * n_cts;
+#pragma omp parallel for schedule(dynamic)
+  for (int64_t u = 0; u < total; ++u) {
+    uint32_t c = (uint32_t)(u % n_cts);
+    uint32_t k = (uint32_t)((u / n_cts) % n_parties);
+    uint32_t i = (uint32_t)(u / ((int64_t)n_cts * n_parties));
+    uint64_t* alpha = (uint64_t*)malloc(sizeof(uint64_t) * poly);
+    orc_boot_alpha(P, recipients[i], ct_first + c, alpha);
+    const uint64_t* c1 = agg + (((size_t)i * n_cts + c) * 2 + 1) * poly;
+    orc_boot_share(P, parties[k], recipients[i], ct_first + c, c1, alpha, shares + (size_t)u * 2 * poly);
+    free(alpha);
+  }
+}
+
+/*
+ * ct' = ( [round(t/q [c_0 + eta_0]_q)]_t Lambda + eta_1,  alpha ),  eta_d = sum_k eta_{d,k}.
+ * agg [n_rec][n_cts][2][L][N], shares [n_rec][n_shares][n_cts][2][L][N] -> out [n_rec][n_cts][2][L][N].
+ */
+void orc_boot_combine_batch(const orc_params* P, const uint64_t* agg, const uint64_t* shares,
+                            const uint32_t* recipients, uint32_t n_rec, uint32_t n_shares,
+                            uint32_t ct_first, uint32_t n_cts, uint64_t* out) {
+  uint32_t n = 1u << P->log2_n, L = P->num_limbs;
+  size_t poly = (size_t)L * n;
+  uint64_t delta[ORC_MAX_LIMBS];
+  orc_delta(P, delta);
+#pragma omp parallel for schedule(dynamic)
+  for (int64_t u = 0; u < (int64_t)n_rec * n_cts; ++u) {
+    uint32_t i = (uint32_t)(u / n_cts), c = (uint32_t)(u % n_cts);
+    uint64_t* eta0 = (uint64_t*)malloc(sizeof(uint64_t) * poly * n_shares);
+    uint32_t* x = (uint32_t*)malloc(sizeof(uint32_t) * n);
+    for (uint32_t k = 0; k < n_shares; ++k)
+      memcpy(eta0 + (size_t)k * poly, shares + ((((size_t)i * n_shares + k) * n_cts + c) * 2) * poly,
+             sizeof(uint64_t) * poly);
+    orc_combine(P, agg + (size_t)u * 2 * poly, eta0, n_shares, x);
+    uint64_t* o = out + (size_t)u * 2 * poly;
+    for (uint32_t l = 0; l < L; ++l) {
+      uint64_t p = P->moduli[l];
+      for (uint32_t j = 0; j < n; ++j) {
+        uint64_t acc = mulm(delta[l], x[j] % p, p);
+        for (uint32_t k = 0; k < n_shares; ++k)
+          acc = addm(acc, shares[((((size_t)i * n_shares + k) * n_cts + c) * 2 + 1) * poly + (size_t)l * n + j], p);
+        o[(size_t)l * n + j] = acc;
+      }
+    }
+    orc_boot_alpha(P, recipients[i], ct_first + c, o + poly);
+    free(eta0);
+    free(x);
   }
 }
 

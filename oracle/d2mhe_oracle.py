@@ -324,6 +324,36 @@ class Oracle:
                                 ctypes.c_uint32(ct.shape[1]), _p(plain))
         return plain
 
+    # MBFV.Bootstrap (Sec. 4.2 item 4)
+    def boot_alpha(self, recipient, ct_index):
+        out = np.empty((self.num_limbs, self.n), dtype=np.uint64)
+        lib().orc_boot_alpha(self._ref, ctypes.c_uint32(recipient), ctypes.c_uint32(ct_index), _p(out))
+        return out
+
+    def boot_mask(self, party, recipient, ct_index):
+        out = np.empty(self.n, dtype=np.uint32)
+        lib().orc_boot_mask(self._ref, ctypes.c_uint32(party), ctypes.c_uint32(recipient), ctypes.c_uint32(ct_index), _p(out))
+        return out
+
+    def boot_share(self, agg, recipients, parties, ct_first):
+        agg = _u64(agg)
+        recipients, parties = _u32(recipients), _u32(parties)
+        n_rec, n_cts = agg.shape[0], agg.shape[1]
+        shares = np.empty((n_rec, parties.size, n_cts, 2, self.num_limbs, self.n), dtype=np.uint64)
+        lib().orc_boot_share_batch(self._ref, _p(agg), _p(recipients), ctypes.c_uint32(n_rec), _p(parties),
+                                   ctypes.c_uint32(parties.size), ctypes.c_uint32(ct_first), ctypes.c_uint32(n_cts),
+                                   _p(shares))
+        return shares
+
+    def boot_combine(self, agg, shares, recipients, ct_first):
+        agg, shares = _u64(agg), _u64(shares)
+        recipients = _u32(recipients)
+        out = np.empty_like(agg)
+        lib().orc_boot_combine_batch(self._ref, _p(agg), _p(shares), _p(recipients), ctypes.c_uint32(agg.shape[0]),
+                                     ctypes.c_uint32(shares.shape[1]), ctypes.c_uint32(ct_first),
+                                     ctypes.c_uint32(agg.shape[1]), _p(out))
+        return out
+
     def decrypt_single(self, ct, s, want_noise=False):
         """BFV.Decrypt of one ciphertext [2, L, N] under an explicit integer secret s[N]."""
         ct = _u64(ct)

@@ -102,6 +102,26 @@ def convert_share(c1, s_k, mu_k, e0_k, e1_k, p0_i, p1_i, q):
     return h0, h1
 
 
+def bootstrap_share(c1, alpha, s_k, m_k, e0_k, e1_k, q, t):
+    """(eta_0, eta_1) = (s_k c1 - Lambda M_k + e_{0,k}, -s_k alpha + Lambda M_k + e_{1,k})   (Eq. 4)."""
+    lam = q // t
+    s = [x % q for x in s_k]
+    lm = [lam * x % q for x in m_k]
+    eta0 = poly_add(poly_add(negacyclic_mul(c1, s, q), poly_neg(lm, q), q), [x % q for x in e0_k], q)
+    eta1 = poly_add(poly_add(poly_neg(negacyclic_mul(alpha, s, q), q), lm, q), [x % q for x in e1_k], q)
+    return eta0, eta1
+
+
+def bootstrap_combine(c0, eta0_list, eta1_list, alpha, q, t):
+    """ct' = ([round(t/q [c0 + eta_0]_q)]_t Lambda + eta_1, alpha)   (Sec. 4.2 item 4)."""
+    x = combine(c0, eta0_list, q, t)
+    lam = q // t
+    c0n = [lam * v % q for v in x]
+    for e in eta1_list:
+        c0n = poly_add(c0n, e, q)
+    return c0n, list(alpha)
+
+
 def combine(c0, shares, q, t):
     """[ round( t/q * [c0 + sum_k h_k]_q ) ]_t   (Sec. 4.2 item 3, Eq. 3; Sec. 3.2 item 5)."""
     v = list(c0)
