@@ -183,6 +183,26 @@ d2mhe_status d2mhe_decrypt(d2mhe_ctx* ctx, const uint32_t* users, uint32_t n_use
                            uint32_t* plain_dev);
 
 /*
+ * MBFV.Bootstrap (Sec. 4.2 item 4, Eq. 4): collective noise refresh of agg[i, c].
+ * d2mhe_bootstrap_share: shares[i, a, c] = (eta_0, eta_1) =
+ *   (s_k c_1 - Lambda M_k + e_{0,k},  -s_k alpha + Lambda M_k + e_{1,k}),  k = parties[a],
+ *   M_k uniform over R_t, e_{0,k}, e_{1,k} from chi on the stream (party k, recipient, ciphertext
+ *   index ct_first + c); alpha is the common polynomial, uniform on R_q, derived from
+ *   (recipient, ciphertext index).  shares_dev: out [n_rec, n_parties, n_cts, 2, L, N].
+ * d2mhe_bootstrap_combine: ct'[i, c] = ([round(t/q [c_0 + sum_k eta_{0,k}]_q)]_t Lambda + sum_k eta_{1,k}, alpha).
+ *   n_shares must equal the size of the collective key's party set; recipients and ct_first as in
+ *   the share call (they select alpha).  plain_scratch_dev: caller-provided uint32 [n_rec, n_cts, N]
+ *   (receives the masked plaintext); ct_out_dev: out [n_rec, n_cts, 2, L, N].
+ */
+d2mhe_status d2mhe_bootstrap_share(d2mhe_ctx* ctx, const uint64_t* agg_dev, const uint32_t* recipients,
+                                   uint32_t n_rec, const uint32_t* parties, uint32_t n_parties,
+                                   uint32_t ct_first, uint32_t n_cts, uint64_t* shares_dev);
+d2mhe_status d2mhe_bootstrap_combine(d2mhe_ctx* ctx, const uint64_t* agg_dev, const uint64_t* shares_dev,
+                                     const uint32_t* recipients, uint32_t n_rec, uint32_t n_shares,
+                                     uint32_t ct_first, uint32_t n_cts, uint32_t* plain_scratch_dev,
+                                     uint64_t* ct_out_dev);
+
+/*
  * Batched negacyclic number-theoretic transform of [batch, L, N], in place.
  * Forward: position p of limb l receives a(psi_l^(2 brv(p) + 1)), brv = reversal of
  * the log2_n-bit index, psi_l the root reported by d2mhe_get_root.  Inverse undoes it.

@@ -99,7 +99,11 @@ enum : u32 {
   TAG_USER_P1 = 10,
   TAG_CONV_MU = 11,
   TAG_CONV_E0 = 12,
-  TAG_CONV_E1 = 13
+  TAG_CONV_E1 = 13,
+  TAG_BOOT_ALPHA = 14,
+  TAG_BOOT_MASK = 15,
+  TAG_BOOT_E0 = 16,
+  TAG_BOOT_E1 = 17
 };
 
 // One stream: counter = (j, idx, party | recipient << 16, tag | attempt << 8).

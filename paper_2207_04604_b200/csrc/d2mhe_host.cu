@@ -648,7 +648,7 @@ d2mhe_status d2mhe_combine_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev,
   if ((u64)n_rec * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
   cudaError_t e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
-                                        reinterpret_cast<const u64*>(shares_dev), n_rec, n_shares, n_cts,
+                                        reinterpret_cast<const u64*>(shares_dev), n_rec, n_shares, 1, n_cts,
                                         plain_dev);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
@@ -778,7 +778,62 @@ d2mhe_status d2mhe_decrypt(d2mhe_ctx* c, const u32* users, u32 n_users, const ui
   if (e != cudaSuccess) return fail_cuda(c, e);
   // [c_0 + c_1 sk_i]_q then the exact scale-and-round: the product plays the role of one share
   e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(ct_dev),
-                            reinterpret_cast<const u64*>(scratch_dev), n_users, 1, n_cts, plain_dev);
+                            reinterpret_cast<const u64*>(scratch_dev), n_users, 1, 1, n_cts, plain_dev);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 2;
+  return release_slot(c, sg);
+}
+
+// ---- MBFV.Bootstrap ---------------------------------------------------------------------
+
+d2mhe_status d2mhe_bootstrap_share(d2mhe_ctx* c, const uint64_t* agg_dev, const u32* recipients, u32 n_rec,
+                                   const u32* parties, u32 n_parties, u32 ct_first, u32 n_cts,
+                                   uint64_t* shares_dev) {
+  if (!c || !agg_dev || !shares_dev || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(agg_dev) || !aligned16(shares_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  d2mhe_status st = check_party_list(c, recipients, n_rec, false, false);
+  if (st != D2MHE_OK) return st;
+  st = check_party_list(c, parties, n_parties, true, true);
+  if (st != D2MHE_OK) return st;
+  if ((u64)ct_first + n_cts > 0xffffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)n_rec * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[2] = {recipients, parties};
+  const size_t counts[2] = {n_rec, n_parties};
+  if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::boot_share(c->view, c->limb_params, c->stream,
+                                           reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1],
+                                           n_parties, ct_first, n_cts, reinterpret_cast<u64*>(shares_dev));
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_bootstrap_combine(d2mhe_ctx* c, const uint64_t* agg_dev, const uint64_t* shares_dev,
+                                     const u32* recipients, u32 n_rec, u32 n_shares, u32 ct_first,
+                                     u32 n_cts, u32* plain_scratch_dev, uint64_t* ct_out_dev) {
+  if (!c || !agg_dev || !shares_dev || !plain_scratch_dev || !ct_out_dev || n_cts == 0)
+    return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(agg_dev) || !aligned16(shares_dev) || !aligned16(plain_scratch_dev) || !aligned16(ct_out_dev))
+    return D2MHE_ERR_INVALID_ARG;
+  if (!c->has_pk) return D2MHE_ERR_STATE;
+  if (n_shares != c->pk_parties.size()) return D2MHE_ERR_INVALID_ARG;
+  d2mhe_status st = check_party_list(c, recipients, n_rec, false, false);
+  if (st != D2MHE_OK) return st;
+  if ((u64)ct_first + n_cts > 0xffffffffull || (u64)n_rec * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[1] = {recipients};
+  const size_t counts[1] = {n_rec};
+  if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
+  cudaError_t e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
+                                        reinterpret_cast<const u64*>(shares_dev), n_rec, n_shares, 2, n_cts,
+                                        plain_scratch_dev);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  e = d2mhe_launch::boot_finish(c->view, c->stream, plain_scratch_dev, reinterpret_cast<const u64*>(shares_dev),
+                                sg.dev[0], n_rec, n_shares, ct_first, n_cts, reinterpret_cast<u64*>(ct_out_dev));
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 2;
   return release_slot(c, sg);

@@ -98,8 +98,14 @@ cudaError_t aggregate(const DevView& v, cudaStream_t s, const u64* ct, u32 n_cts
 cudaError_t partial_decrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
                             const u32* recipients_dev, u32 n_rec, const u32* parties_dev,
                             u32 n_parties, u32 ct_first, u32 n_cts, u64* shares);
+// shares hold share_comps polynomials per (recipient, party, ciphertext); the first one is summed
 cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
-                    u32 n_shares, u32 n_cts, u32* plain);
+                    u32 n_shares, u32 share_comps, u32 n_cts, u32* plain);
+cudaError_t boot_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
+                       const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties,
+                       u32 ct_first, u32 n_cts, u64* shares);
+cudaError_t boot_finish(const DevView& v, cudaStream_t s, const u32* x, const u64* shares,
+                        const u32* recipients_dev, u32 n_rec, u32 n_shares, u32 ct_first, u32 n_cts, u64* out);
 cudaError_t ntt(const DevView& v, const LimbParams& lp, cudaStream_t s, u64* polys, u32 batch, bool inverse);
 cudaError_t user_keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* users_dev,
                         u32 n_users);

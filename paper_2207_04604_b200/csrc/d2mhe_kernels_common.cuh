@@ -78,6 +78,20 @@ __device__ __forceinline__ void load_octet_rw(const u64* src, u64 (&x)[8]) {
   }
 }
 
+// Lambda * m for a plaintext coefficient m < 2^32: exact quotient from two widening
+// products, result in [0, 2p).
+__device__ __forceinline__ u64 shoup_u32(u32 m, u64 w, u64 ws, u64 np) {
+  u32 sl, sh, wl, wh, nl, nh, ql, q, rl, rh;
+  split64(ws, sl, sh);
+  split64(w, wl, wh);
+  split64(np, nl, nh);
+  split64(madwide(m, sh, join64(mulhi32(m, sl), 0u)), ql, q);  // q = floor(m ws / 2^64) exactly
+  split64(madwide(q, nl, mulwide(m, wl)), rl, rh);
+  rh = madlo(m, wh, rh);
+  rh = madlo(q, nh, rh);
+  return join64(rl, rh);
+}
+
 // v (below 4p) + small signed e, canonical in [0, p)
 __device__ __forceinline__ u64 add_small_canon(u64 v, int e, const LimbTab& lt) {
   const u64 s = v + lt.p + (u64)(long long)e;  // below 5p + 19

@@ -1,0 +1,143 @@
+// MBFV.Bootstrap (Sec. 4.2 item 4, Eq. 4): collective noise refresh.
+#include "d2mhe_kernels_common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace {
+
+// Shares (eta_0, eta_1) = (s_k c_1 - Lambda M_k + e_{0,k}, -s_k alpha + Lambda M_k + e_{1,k}).
+// grid = n_rec * n_cts * L in clusters over limbs: e_0, e_1 (bytes) and the mask M_k (32-bit words,
+// uniform mod t) are sampled once per cluster and pushed through distributed shared memory.
+// NTT(c_1) is parked in the eta_0 row and NTT(alpha) in the eta_1 row of the last share.
+// Iterations -2 and -1 run the two forward transforms, iteration a >= 0 produces share a, so that
+// one forward and one inverse call site serve the whole kernel.
+template <int LOGN, int G, bool WIDE>
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+    k_boot_share(DevView v, const __grid_constant__ LimbParams lp, const u64* __restrict__ agg,
+                 const u32* __restrict__ recipients, const u32* __restrict__ parties, u32 n_parties,
+                 u32 ct_first, u32 n_cts, u64* shares) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const u32 cs = cluster.num_blocks(), rank = cluster.block_rank();
+  const u32 l = blockIdx.x % v.L, unit = blockIdx.x / v.L;
+  const u32 irec = unit / n_cts, cl = unit % n_cts, c = ct_first + cl;
+  const u32 recipient = recipients[irec];
+  const LimbTab& lt = lp.limbs[l];
+  GaussTab* gt = gauss_smem();
+  load_gauss(gt, v.gauss);
+  signed char* small = bytes_smem();                        // e_0, e_1: N bytes each
+  u32* mask = reinterpret_cast<u32*>(small + 2 * v.n);      // M_k: N words
+  u64* sm = poly_smem(6 * v.n);
+  const size_t row = (size_t)l * v.n, poly = (size_t)v.L * v.n;
+  const u64* c1 = agg + ((size_t)unit * 2 + 1) * poly + row;
+  u64* park = shares + ((((size_t)irec * n_parties + (n_parties - 1)) * n_cts + cl) * 2) * poly + row;
+  const Stream sa(v.seed, TAG_BOOT_ALPHA, c, l, recipient);
+  const u64 t = v.round.t;
+  u64 tmask = 1;
+  while (tmask <= t) tmask <<= 1;
+  tmask -= 1;
+#pragma unroll 1
+  for (int a = -2; a < (int)n_parties; ++a) {
+    const u32 party = a < 0 ? 0u : parties[a];
+    if (a >= 0) {
+      cluster.sync();  // every CTA is done with the previous share's samples
+      const Stream s0(v.seed, TAG_BOOT_E0, c, party, recipient);
+      const Stream s1(v.seed, TAG_BOOT_E1, c, party, recipient);
+      const Stream sk_(v.seed, TAG_BOOT_MASK, c, party, recipient);
+      const u32 quarter = v.n >> 2;
+      // words 0..N/4-1: e_0 and N/4..N/2-1: e_1 (four samples per word), then N words of M_k
+#pragma unroll 1
+      for (u32 w = rank + cs * threadIdx.x; w < 2 * quarter + v.n; w += cs * blockDim.x) {
+        u32 word;
+        if (w < 2 * quarter) {
+          const Stream& st = w < quarter ? s0 : s1;
+          const u32 j0 = 4 * (w < quarter ? w : w - quarter);
+          word = 0;
+#pragma unroll
+          for (u32 b = 0; b < 4; ++b) word |= ((u32)gauss_from_r(*gt, st.draw64(j0 + b)) & 0xffu) << (8 * b);
+        } else {
+          word = (u32)uniform_mod(sk_, w - 2 * quarter, t, tmask);
+        }
+        for (u32 r = 0; r < cs; ++r) cluster.map_shared_rank(reinterpret_cast<u32*>(small), r)[w] = word;
+      }
+      cluster.sync();  // all samples of this share have landed everywhere
+    }
+    u64* h0 = a < 0 ? park : shares + ((((size_t)irec * n_parties + a) * n_cts + cl) * 2) * poly + row;
+    u64* h1 = h0 + poly;
+    if (a < 0) {
+      u64* dst = a == -2 ? park : park + poly;
+      ntt_forward<LOGN, G, WIDE>(
+          sm, lt, v.logn,
+          [&](u32 j) { return a == -2 ? __ldg(c1 + j) : uniform_mod(sa, j, lt.p, lt.mask); },
+          [&](int, u32 q, u64(&x)[8]) { store_octet(dst + 8 * (size_t)q, x); });
+      continue;
+    }
+    const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
+#pragma unroll 1
+    for (u32 comp = 0; comp < 2; ++comp) {
+      const u64* src = comp ? park + poly : park;
+      u64* out = comp ? h1 : h0;
+      const signed char* e = small + comp * v.n;
+      ntt_inverse<LOGN, G, WIDE>(
+          sm, lt, v.logn,
+          [&](int, u32 q, u64(&x)[8]) {
+            u64 a8[8];
+            load_octet_rw(src + 8 * (size_t)q, a8);
+            load_octet(sk + 8 * (size_t)q, x);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) x[k] = mont_lazy(a8[k], x[k], lt.p, lt.pinv);
+          },
+          [&](u32 j, u64 val) {
+            const u64 dm = shoup_u32(mask[j], lt.delta, lt.delta_sh, lt.np);  // Lambda M_k, below 2p
+            // eta_0 = val - dm + e,  eta_1 = -val + dm + e; both sums below 8p
+            const u64 s = (comp ? (2 * lt.twop - val) + dm : val + (lt.twop - dm)) + lt.p + (u64)(long long)e[j];
+            out[j] = csub(csub(csub(s, 2 * lt.twop), lt.twop), lt.p);
+          });
+    }
+  }
+  cluster.sync();
+}
+
+// ct' = (Lambda x + sum_k eta_{1,k}, alpha) with x the rounded plaintext of c_0 + eta_0.
+// grid = (n_rec * n_cts, chunks); one residue per thread and iteration.
+__global__ void __launch_bounds__(256)
+    k_boot_finish(DevView v, const u32* __restrict__ x, const u64* __restrict__ shares,
+                  const u32* __restrict__ recipients, u32 n_shares, u32 ct_first, u32 n_cts,
+                  u64* __restrict__ out) {
+  const u32 unit = blockIdx.x, irec = unit / n_cts, cl = unit % n_cts;
+  const u32 recipient = recipients[irec];
+  const size_t poly = (size_t)v.L * v.n;
+  for (size_t e = (size_t)blockIdx.y * blockDim.x + threadIdx.x; e < poly; e += (size_t)gridDim.y * blockDim.x) {
+    const u32 l = (u32)(e >> v.logn), j = (u32)(e & (v.n - 1));
+    const LimbTab* lt = v.limbs + l;
+    const u64 p = lt->p;
+    u64 acc = csub(shoup_u32(x[(size_t)unit * v.n + j], lt->delta, lt->delta_sh, lt->np), p);
+    for (u32 k = 0; k < n_shares; ++k)
+      acc = addmod(acc, __ldg(shares + ((((size_t)irec * n_shares + k) * n_cts + cl) * 2 + 1) * poly + e), p);
+    out[(size_t)unit * 2 * poly + e] = acc;
+    const Stream sa(v.seed, TAG_BOOT_ALPHA, ct_first + cl, l, recipient);
+    out[(size_t)unit * 2 * poly + poly + e] = uniform_mod(sa, j, p, lt->mask);
+  }
+}
+
+}  // namespace
+
+namespace d2mhe_launch {
+
+cudaError_t boot_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
+                       const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties,
+                       u32 ct_first, u32 n_cts, u64* shares) {
+  D2MHE_DISPATCH_EX(k_boot_share, v, n_rec * n_cts * v.L, s, 6 * (size_t)v.n, cluster_size_for(v.L), v, lp,
+                    agg, recipients_dev, parties_dev, n_parties, ct_first, n_cts, shares);
+}
+
+cudaError_t boot_finish(const DevView& v, cudaStream_t s, const u32* x, const u64* shares,
+                        const u32* recipients_dev, u32 n_rec, u32 n_shares, u32 ct_first, u32 n_cts, u64* out) {
+  const size_t poly = (size_t)v.L * v.n;
+  u32 by = (u32)((poly + 255) / 256);
+  if (by > 32768) by = 32768;
+  dim3 grid(n_rec * n_cts, by);
+  k_boot_finish<<<grid, 256, 0, s>>>(v, x, shares, recipients_dev, n_shares, ct_first, n_cts, out);
+  return cudaGetLastError();
+}
+
+}  // namespace d2mhe_launch

@@ -5,20 +5,6 @@ namespace cg = cooperative_groups;
 
 namespace {
 
-// Lambda * m for a plaintext coefficient m < 2^32: exact quotient from two widening
-// products, result in [0, 2p).
-__device__ __forceinline__ u64 shoup_u32(u32 m, u64 w, u64 ws, u64 np) {
-  u32 sl, sh, wl, wh, nl, nh, ql, q, rl, rh;
-  split64(ws, sl, sh);
-  split64(w, wl, wh);
-  split64(np, nl, nh);
-  split64(madwide(m, sh, join64(mulhi32(m, sl), 0u)), ql, q);  // q = floor(m ws / 2^64) exactly
-  split64(madwide(q, nl, mulwide(m, wl)), rl, rh);
-  rh = madlo(m, wh, rh);
-  rh = madlo(q, nh, rh);
-  return join64(rl, rh);
-}
-
 // grid = n_units * L, launched in thread-block clusters of cs CTAs = cs limbs of the same
 // (party, ciphertext).  u, e_0 and e_1 do not depend on the limb: each CTA samples 1/cs of
 // their coefficients and pushes them (four to a word) into the shared memory of all cs CTAs.

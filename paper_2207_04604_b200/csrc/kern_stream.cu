@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(256)
 template <int LMAX>
 __global__ void __launch_bounds__(256)
     k_combine(DevView v, const u64* __restrict__ agg, const u64* __restrict__ shares, u32 n_shares,
-              u32 n_cts, u32* __restrict__ plain) {
+              u32 share_comps, u32 n_cts, u32* __restrict__ plain) {
   const u32 unit = blockIdx.x, irec = unit / n_cts, cl = unit % n_cts;
   const u32 j = blockIdx.y * blockDim.x + threadIdx.x;
   if (j >= v.n) return;
@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(256)
       const u64 p = lt->p;
       u64 acc = __ldg(c0 + (size_t)l * v.n + j);
       for (u32 k = 0; k < n_shares; ++k)
-        acc = addmod(acc, __ldg(shares + (((size_t)irec * n_shares + k) * n_cts + cl) * poly +
+        acc = addmod(acc, __ldg(shares + (((size_t)irec * n_shares + k) * n_cts + cl) * share_comps * poly +
                                 (size_t)l * v.n + j), p);
       d[l] = addmod(shoup_full(acc, lt->tmod, lt->tmod_sh, p), lt->half, p);
     }
@@ -200,14 +200,14 @@ cudaError_t aggregate(const DevView& v, cudaStream_t s, const u64* ct, u32 n_cts
 }
 
 cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
-                    u32 n_shares, u32 n_cts, u32* plain) {
+                    u32 n_shares, u32 share_comps, u32 n_cts, u32* plain) {
   dim3 grid(n_rec * n_cts, (v.n + 255) / 256);
   if (v.L <= 4)
-    k_combine<4><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, n_cts, plain);
+    k_combine<4><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, share_comps, n_cts, plain);
   else if (v.L <= 8)
-    k_combine<8><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, n_cts, plain);
+    k_combine<8><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, share_comps, n_cts, plain);
   else
-    k_combine<D2MHE_MAX_LIMBS><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, n_cts, plain);
+    k_combine<D2MHE_MAX_LIMBS><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, share_comps, n_cts, plain);
   return cudaGetLastError();
 }
 

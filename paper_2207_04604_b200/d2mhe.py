@@ -29,7 +29,7 @@ EXPORTS = [
     "d2mhe_aggregate", "d2mhe_partial_decrypt", "d2mhe_combine_decrypt", "d2mhe_ntt_forward",
     "d2mhe_ntt_inverse", "d2mhe_poly_muladd", "d2mhe_round_workspace_bytes", "d2mhe_round_device",
     "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_user_keygen", "d2mhe_convert_share",
-    "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_get_root", "d2mhe_get_plain_root",
+    "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_bootstrap_share", "d2mhe_bootstrap_combine", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_get_root", "d2mhe_get_plain_root",
     "d2mhe_launch_count",
 ]
 
@@ -97,6 +97,8 @@ def load():
         lib.d2mhe_convert_share.argtypes = [vp, vp, vp, u32, vp, u32, u32, u32, vp]
         lib.d2mhe_convert_combine.argtypes = [vp, vp, vp, u32, u32, u32, vp]
         lib.d2mhe_decrypt.argtypes = [vp, vp, u32, vp, u32, vp, vp]
+        lib.d2mhe_bootstrap_share.argtypes = [vp, vp, vp, u32, vp, u32, u32, u32, vp]
+        lib.d2mhe_bootstrap_combine.argtypes = [vp, vp, vp, vp, u32, u32, u32, u32, vp, vp]
         lib.d2mhe_get_root.argtypes = [vp, u32, ctypes.POINTER(u64)]
         lib.d2mhe_get_plain_root.argtypes = [vp, ctypes.POINTER(u64)]
         lib.d2mhe_launch_count.argtypes = [vp]
@@ -284,6 +286,19 @@ class Context:
         arr, ptr = _host_u32(users)
         self._check(load().d2mhe_decrypt(self._h, ptr, arr.size, _dev(ct, U64), n_cts, _dev(scratch, U64),
                                          _dev(plain, U32)), "d2mhe_decrypt")
+
+    # ---- collective noise refresh ----
+    def bootstrap_share(self, agg, recipients, parties, ct_first, n_cts, shares):
+        rec, recp = _host_u32(recipients)
+        par, parp = _host_u32(parties)
+        self._check(load().d2mhe_bootstrap_share(self._h, _dev(agg, U64), recp, rec.size, parp, par.size, ct_first,
+                                                 n_cts, _dev(shares, U64)), "d2mhe_bootstrap_share")
+
+    def bootstrap_combine(self, agg, shares, recipients, n_shares, ct_first, n_cts, plain_scratch, ct_out):
+        rec, recp = _host_u32(recipients)
+        self._check(load().d2mhe_bootstrap_combine(self._h, _dev(agg, U64), _dev(shares, U64), recp, rec.size,
+                                                   n_shares, ct_first, n_cts, _dev(plain_scratch, U32),
+                                                   _dev(ct_out, U64)), "d2mhe_bootstrap_combine")
 
     def debug_export_user_secret(self, user):
         out = np.empty(self.n, dtype=np.int8)

@@ -416,6 +416,50 @@ def test_convert_every_message(d2, log2_n, moduli_spec, K, n_cts):
     ctx.close()
 
 
+@pytest.mark.parametrize("log2_n,moduli_spec,K,n_cts", [
+    (4, (30, 2), 3, 2), (7, (54, 3), 2, 1), (12, None, 4, 2), (13, (54, 4), 3, 1), (14, (60, 2), 2, 1),
+])
+def test_bootstrap_every_message(d2, log2_n, moduli_spec, K, n_cts):
+    """MBFV.Bootstrap: shares, refreshed ciphertext, and that the refreshed ciphertext goes through
+    the ordinary collective decryption to the same sums."""
+    moduli = wl.round_config(1).moduli if moduli_spec is None else small_moduli(log2_n, *moduli_spec)
+    seed = 51 + log2_n
+    L, n = len(moduli), 1 << log2_n
+    ctx = d2.Context(log2_n, moduli, K, seed=seed)
+    o = make_oracle(log2_n, moduli, seed=seed)
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    pk = o.collective_pk(parties)
+    values = np.random.default_rng(seed).integers(-4000, 4001, size=(K, n_cts, n)).astype(np.int32)
+    offsets = np.array([0, K, K + 1], dtype=np.uint32)
+    rows = np.array(parties + [K - 1], dtype=np.uint32)
+    want_agg = o.aggregate(o.encrypt(pk, parties, 9, o.encode(values)), offsets, rows)
+    agg = d2.from_u64_numpy(want_agg, ctx.device)
+    recipients = [1, 0]
+    shares = ctx.empty_u64(2, K, n_cts, 2, L, n)
+    ctx.bootstrap_share(agg, recipients, parties, 9, n_cts, shares)
+    want_shares = o.boot_share(want_agg, recipients, parties, 9)
+    assert np.array_equal(d2.to_u64_numpy(shares), want_shares)
+    fresh = ctx.empty_u64(2, n_cts, 2, L, n)
+    scratch = ctx.empty_u32(2, n_cts, n)
+    ctx.bootstrap_combine(agg, shares, recipients, K, 9, n_cts, scratch, fresh)
+    want_fresh = o.boot_combine(want_agg, want_shares, recipients, 9)
+    assert np.array_equal(d2.to_u64_numpy(fresh), want_fresh)
+    # the refreshed ciphertexts decrypt collectively to the same sums
+    dshares = ctx.empty_u64(2, K, n_cts, L, n)
+    ctx.partial_decrypt(fresh, recipients, parties, 9, n_cts, dshares)
+    plain = ctx.empty_u32(2, n_cts, n)
+    ctx.combine_decrypt(fresh, dshares, 2, K, n_cts, plain)
+    sums = torch.empty((2, n_cts, n), dtype=torch.int32, device=ctx.device)
+    ctx.decode(plain, 2 * n_cts, sums)
+    ctx.sync()
+    got = sums.cpu().numpy()
+    assert np.array_equal(got[0], values.astype(np.int64).sum(axis=0))
+    assert np.array_equal(got[1], values[K - 1])
+    ctx.close()
+
+
 # ----------------------------------------------------------------------------------
 # whole-round driver, chunking, determinism, error paths
 # ----------------------------------------------------------------------------------
