@@ -460,6 +460,72 @@ def test_bootstrap_every_message(d2, log2_n, moduli_spec, K, n_cts):
     ctx.close()
 
 
+def test_private_dpsgd_equals_plaintext_dpsgd(d2):
+    """Algorithm 2 on synthetic quadratic objectives L_i(W) = |W - a_i|^2 / 2: the encrypted loop gives
+    bit for bit what plaintext D-PSGD gives on the same fixed-point values, and it converges."""
+    from paper_2207_04604_b200 import dpsgd
+
+    K, H, lr = 6, 10000, 0.5
+    moduli = wl.round_config(1).moduli
+    ctx = d2.Context(12, moduli, K, seed=8)
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    offsets, rows = wl.regular_graph(K, 2, 8)
+    rng = np.random.default_rng(8)
+    targets = rng.uniform(-1.0, 1.0, size=(K, H))
+    w_enc = np.zeros((K, H))
+    w_ref = np.zeros((K, H))
+    loop = dpsgd.PrivateDPSGD(ctx, offsets, rows, H, chunk_cts=2)
+    assert loop.C == 3
+    losses = []
+    for _ in range(6):
+        w_enc = loop.step(w_enc, w_enc - targets, lr)
+        w_ref = dpsgd.plaintext_mix(w_ref, offsets, rows, loop.clip) - lr * (w_ref - targets)
+        assert np.array_equal(w_enc, w_ref)
+        losses.append(float(((w_enc.mean(axis=0) - targets.mean(axis=0)) ** 2).mean()))
+    assert losses[-1] < 0.05 * losses[0]
+    ctx.close()
+
+
+def test_per_neighbourhood_keys(d2):
+    """The literal reading of Sec. 4.2 item 1: one collective key per closed neighbourhood U_i, shares
+    only from U_i.  Expressed with the same calls by passing the neighbourhood as the party set."""
+    cfg = wl.round_config(1)
+    K, L, n = cfg.num_parties, cfg.num_limbs, cfg.n
+    seed = 12
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, K, seed=seed)
+    o = make_oracle(cfg.log2_n, cfg.moduli, seed=seed)
+    offsets, rows = wl.regular_graph(K, cfg.degree, seed)
+    values = wl.gradients(cfg, seed)[:, :1]
+    ctx.keygen_share(list(range(K)))
+    dv = torch.from_numpy(values).to(ctx.device)
+    plain = ctx.empty_u32(K, 1, n)
+    ctx.encode(dv, K, plain)
+    for i in range(K):
+        U = [int(x) for x in rows[offsets[i]:offsets[i + 1]]]
+        S = len(U)
+        pk = ctx.empty_u64(2, L, n)
+        ctx.collective_pk(U, None, pk)  # key of this neighbourhood: s = sum_{k in U_i} s_k
+        want_pk = o.collective_pk(U)
+        assert np.array_equal(d2.to_u64_numpy(pk), want_pk)
+        ct = ctx.empty_u64(S, 1, 2, L, n)
+        ctx.encrypt(U, 0, 1, plain[U].contiguous(), ct)
+        agg = ctx.empty_u64(1, 1, 2, L, n)
+        ctx.aggregate(ct, S, 1, [0, S], list(range(S)), agg)
+        shares = ctx.empty_u64(1, S, 1, L, n)
+        ctx.partial_decrypt(agg, [i], U, 0, 1, shares)
+        out = ctx.empty_u32(1, 1, n)
+        ctx.combine_decrypt(agg, shares, 1, S, 1, out)
+        sums = torch.empty((1, 1, n), dtype=torch.int32, device=ctx.device)
+        ctx.decode(out, 1, sums)
+        ctx.sync()
+        assert np.array_equal(sums.cpu().numpy()[0, 0], values[U, 0].astype(np.int64).sum(axis=0))
+        want_ct = o.encrypt(want_pk, U, 0, o.encode(values[U]))
+        assert np.array_equal(d2.to_u64_numpy(ct), want_ct)
+    ctx.close()
+
+
 # ----------------------------------------------------------------------------------
 # whole-round driver, chunking, determinism, error paths
 # ----------------------------------------------------------------------------------
