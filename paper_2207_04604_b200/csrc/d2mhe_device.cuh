@@ -460,9 +460,14 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
 // Inverse transform (without the N^-1 scaling: fold it into an operand).
 // fetch(g, q, x) fills the octet of positions 8q..8q+7 with values below 4p (below 16p when WIDE);
 // store(j, v) receives coefficient j, v in [0,4p).
-template <int LOGN, int G, bool WIDE, class Fetch, class Store>
+struct NoHook {
+  __device__ __forceinline__ void operator()() const {}
+};
+// before_final() is called by every thread just before the round that calls store().
+template <int LOGN, int G, bool WIDE, class Fetch, class Store, class Hook = NoHook>
 __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
-                                            Fetch fetch, Store store, u32 soff = 0, u32 blk = 0) {
+                                            Fetch fetch, Store store, u32 soff = 0, u32 blk = 0,
+                                            Hook before_final = Hook()) {
   const NttGeom<LOGN, G> ge(logn_rt);
   const u32 T = ge.T, tid = threadIdx.x;
   const Mod md(lt);
@@ -475,6 +480,7 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
     const u32 sh = ge.logn - (u32)s - 3;
     const u32 m = 1u << s;
     const bool final_round = (s == 0);
+    if (final_round) before_final();
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       const u32 q = tid + g * T;
@@ -504,6 +510,7 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
   }
   if (ge.r0) {
     const u32 sh = ge.logn - 3;
+    before_final();
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       const u32 q = tid + g * T;

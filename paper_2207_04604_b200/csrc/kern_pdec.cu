@@ -9,7 +9,8 @@ namespace {
 // (recipient, ciphertext).  The noise polynomial e of a share is the same for every limb, so
 // each CTA of the cluster samples 1/cs of its coefficients (Philox + table inversion) and
 // pushes them, four to a word, into the shared memory of all cs CTAs (distributed shared
-// memory); two noise buffers alternate so that one cluster barrier per share suffices.
+// memory); two noise buffers alternate so that one cluster barrier per share suffices, and
+// that barrier is split: arrive after the push, wait just before the last inverse round.
 // NTT(c_1) is computed once per CTA and parked in the output row of the LAST share
 // (L2-resident, re-read for every share, overwritten by that share at the very end), so no
 // registers are held across the party loop.  Each share costs one pointwise product, one
@@ -49,7 +50,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
         for (u32 r = 0; r < cs; ++r) cluster.map_shared_rank(reinterpret_cast<u32*>(buf), r)[w] = pack;
       }
     }
-    cluster.sync();  // every CTA's part of e has landed in every CTA's buffer
+    cluster.barrier_arrive();  // waited for just before the last round, the only reader of the noise
     const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
     u64* out = shares + (((size_t)irec * n_parties + a) * n_cts + cl) * poly + row;
     ntt_inverse<LOGN, G, WIDE>(
@@ -61,7 +62,8 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = mont_lazy(ch[k], x[k], lt.p, lt.pinv);
         },
-        [&](u32 j, u64 val) { out[j] = add_small_canon(val, (int)buf[j], lt); });
+        [&](u32 j, u64 val) { out[j] = add_small_canon(val, (int)buf[j], lt); }, 0, 0,
+        [&]() { cluster.barrier_wait(); });  // every CTA's part of e has landed in every CTA's buffer
   }
   cluster.sync();  // no CTA leaves while a peer may still write into its buffers
 }

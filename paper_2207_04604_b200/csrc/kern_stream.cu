@@ -65,6 +65,7 @@ __global__ void __launch_bounds__(256)
   const u32 L = v.L;
   const size_t poly = (size_t)L * v.n;
   const u64* c0 = agg + (size_t)unit * 2 * poly;
+  const bool lazy = v.wide != 0 && n_shares < 120;
   u64 d[LMAX];
 #pragma unroll
   for (int l = 0; l < LMAX; ++l) {
@@ -72,9 +73,16 @@ __global__ void __launch_bounds__(256)
       const LimbTab* lt = v.limbs + l;
       const u64 p = lt->p;
       u64 acc = __ldg(c0 + (size_t)l * v.n + j);
-      for (u32 k = 0; k < n_shares; ++k)
-        acc = addmod(acc, __ldg(shares + (((size_t)irec * n_shares + k) * n_cts + cl) * share_comps * poly +
-                                (size_t)l * v.n + j), p);
+      const u64* sh = shares + ((size_t)irec * n_shares * n_cts + cl) * share_comps * poly + (size_t)l * v.n + j;
+      const size_t kstride = (size_t)n_cts * share_comps * poly;
+      if (lazy) {
+        // primes below 2^57 and fewer than 120 shares: the plain 64-bit sum cannot overflow and the
+        // multiplication by t below reduces any 64-bit value, so the loads are all independent
+#pragma unroll 8
+        for (u32 k = 0; k < n_shares; ++k) acc += __ldg(sh + k * kstride);
+      } else {
+        for (u32 k = 0; k < n_shares; ++k) acc = addmod(acc, __ldg(sh + k * kstride), p);
+      }
       d[l] = addmod(shoup_full(acc, lt->tmod, lt->tmod_sh, p), lt->half, p);
     }
   }
