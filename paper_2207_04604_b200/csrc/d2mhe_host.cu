@@ -567,7 +567,7 @@ d2mhe_status d2mhe_encrypt(d2mhe_ctx* c, const u32* parties, u32 n_parties, u32 
   if (!c->has_pk) return D2MHE_ERR_STATE;
   d2mhe_status st = check_party_list(c, parties, n_parties, false, false);
   if (st != D2MHE_OK) return st;
-  if ((u64)ct_first + n_cts > 0xffffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)ct_first + n_cts > 0x100000000ull) return D2MHE_ERR_RANGE;
   if ((u64)n_parties * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
   Staged sg;
@@ -621,7 +621,7 @@ d2mhe_status d2mhe_partial_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev, const 
   if (st != D2MHE_OK) return st;
   st = check_party_list(c, parties, n_parties, true, true);
   if (st != D2MHE_OK) return st;
-  if ((u64)ct_first + n_cts > 0xffffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)ct_first + n_cts > 0x100000000ull) return D2MHE_ERR_RANGE;
   if ((u64)n_rec * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
   Staged sg;
@@ -726,7 +726,7 @@ d2mhe_status d2mhe_convert_share(d2mhe_ctx* c, const uint64_t* agg_dev, const u3
     if (!c->has_user_key[recipients[i]]) return D2MHE_ERR_STATE;
   st = check_party_list(c, parties, n_parties, true, true);
   if (st != D2MHE_OK) return st;
-  if ((u64)ct_first + n_cts > 0xffffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)ct_first + n_cts > 0x100000000ull) return D2MHE_ERR_RANGE;
   if ((u64)n_rec * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
   Staged sg;
@@ -796,7 +796,7 @@ d2mhe_status d2mhe_bootstrap_share(d2mhe_ctx* c, const uint64_t* agg_dev, const 
   if (st != D2MHE_OK) return st;
   st = check_party_list(c, parties, n_parties, true, true);
   if (st != D2MHE_OK) return st;
-  if ((u64)ct_first + n_cts > 0xffffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)ct_first + n_cts > 0x100000000ull) return D2MHE_ERR_RANGE;
   if ((u64)n_rec * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
   Staged sg;
@@ -822,7 +822,7 @@ d2mhe_status d2mhe_bootstrap_combine(d2mhe_ctx* c, const uint64_t* agg_dev, cons
   if (n_shares != c->pk_parties.size()) return D2MHE_ERR_INVALID_ARG;
   d2mhe_status st = check_party_list(c, recipients, n_rec, false, false);
   if (st != D2MHE_OK) return st;
-  if ((u64)ct_first + n_cts > 0xffffffffull || (u64)n_rec * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  if ((u64)ct_first + n_cts > 0x100000000ull || (u64)n_rec * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
   Staged sg;
   const u32* arrays[1] = {recipients};

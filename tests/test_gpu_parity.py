@@ -275,6 +275,26 @@ def test_small_rings_every_message(d2, log2_n, bits, L, K):
     ctx.close()
 
 
+@pytest.mark.parametrize("log2_n,bits,L,K,ct_first", [
+    (5, 54, 1, 1, 0),             # one party, one limb: plain BFV
+    (6, 60, 24, 2, 5),            # the maximum number of limbs, 60-bit primes
+    (12, 54, 6, 3, 2**32 - 2),    # cluster of 6 limbs; ciphertext indices up to 2^32 - 1
+    (11, 36, 7, 2, 1),            # 7 limbs: a prime cluster size
+])
+def test_degenerate_and_extreme_parameter_sets(d2, log2_n, bits, L, K, ct_first):
+    moduli = wl.ntt_primes(bits, 1 << 17, L) if bits >= 50 else small_moduli(log2_n, bits, L)
+    ctx = d2.Context(log2_n, moduli, K, seed=99)
+    o = make_oracle(log2_n, moduli, seed=99)
+    n = 1 << log2_n
+    half = (T - 1) // 2 // K
+    values = np.random.default_rng(1).integers(-half, half + 1, size=(K, 2, n)).astype(np.int32)
+    values[0, 0, :2] = [half, -half]  # extreme slot values
+    offsets = np.array([0, K], dtype=np.uint32)
+    rows = np.arange(K, dtype=np.uint32)
+    _run_round(d2, ctx, o, K, list(range(K)), offsets, rows, values, ct_first)
+    ctx.close()
+
+
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_config1_every_message(d2, seed):
     cfg = wl.round_config(1)
