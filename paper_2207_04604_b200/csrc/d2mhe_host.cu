@@ -883,11 +883,10 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
     u64* shares = agg + (size_t)K * cc * 2 * polyw;
     // values are [K, n_cts, N]: gather the chunk's columns party by party
     int32_t* vals_dev = reinterpret_cast<int32_t*>(plain);  // encode runs in place
-    for (u32 k = 0; k < K; ++k) {
-      const int32_t* src = values + ((size_t)k * n_cts + done) * n;
-      cudaError_t e = cudaMemcpyAsync(vals_dev + (size_t)k * cc * n, src, (size_t)cc * n * sizeof(int32_t),
-                                      host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice,
-                                      c->stream);
+    {  // one strided copy: K rows of cc*N values, source rows n_cts*N apart
+      cudaError_t e = cudaMemcpy2DAsync(vals_dev, (size_t)cc * n * sizeof(int32_t), values + (size_t)done * n,
+                                        (size_t)n_cts * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
+                                        host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, c->stream);
       if (e != cudaSuccess) return fail_cuda(c, e);
     }
     d2mhe_status st;
@@ -902,11 +901,10 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
     if ((st = d2mhe_combine_decrypt(c, reinterpret_cast<uint64_t*>(agg), reinterpret_cast<uint64_t*>(shares),
                                     K, S, cc, plain)) != D2MHE_OK) return st;
     if ((st = d2mhe_decode(c, plain, K * cc, vals_dev)) != D2MHE_OK) return st;
-    for (u32 k = 0; k < K; ++k) {
-      int32_t* dst = sums + ((size_t)k * n_cts + done) * n;
-      cudaError_t e = cudaMemcpyAsync(dst, vals_dev + (size_t)k * cc * n, (size_t)cc * n * sizeof(int32_t),
-                                      host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice,
-                                      c->stream);
+    {
+      cudaError_t e = cudaMemcpy2DAsync(sums + (size_t)done * n, (size_t)n_cts * n * sizeof(int32_t), vals_dev,
+                                        (size_t)cc * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
+                                        host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, c->stream);
       if (e != cudaSuccess) return fail_cuda(c, e);
     }
   }

@@ -123,6 +123,19 @@ __device__ __forceinline__ u32 shoup32_lazy(u32 x, uint2 w, u32 t) {
 }
 __device__ __forceinline__ u32 csub32(u32 x, u32 t) { return x >= t ? x - t : x; }
 
+// Gentleman-Sande / Cooley-Tukey butterflies mod t on lazily reduced 32-bit values (below 2t)
+__device__ __forceinline__ void gs32(u32& X, u32& Y, uint2 w, u32 t, u32 twot) {
+  const u32 s = X + Y, d = X - Y + twot;
+  X = csub32(s, twot);
+  Y = shoup32_lazy(d, w, t);
+}
+__device__ __forceinline__ void ct32(u32& X, u32& Y, uint2 w, u32 t, u32 twot) {
+  const u32 x = csub32(X, twot), T = shoup32_lazy(Y, w, t);
+  X = x + T;
+  Y = x - T + twot;
+}
+
+// encode: values -> slots at bit-reversed positions -> inverse transform, two stages per barrier
 __global__ void __launch_bounds__(1024)
     k_encode(DevView v, const int32_t* __restrict__ values, u32* __restrict__ plain) {
   u32* sm = reinterpret_cast<u32*>(smem_raw);
@@ -140,15 +153,33 @@ __global__ void __launch_bounds__(1024)
   }
   if (bad) atomicOr(v.range_flag, 1u);
   __syncthreads();
-  u32 lt = 0;  // log2 of the butterfly span
-  for (u32 m = n >> 1; m >= 1; m >>= 1, ++lt) {
+  u32 lt = 0;  // log2 of the butterfly span of the next stage
+  for (; lt + 1 < logn; lt += 2) {
+    const u32 span = 1u << lt, m = n >> (lt + 1);
+    for (u32 b = threadIdx.x; b < (n >> 2); b += blockDim.x) {
+      const u32 i2 = b >> lt, jj = b & (span - 1);
+      const u32 base = (i2 << (lt + 2)) + jj;
+      u32 x0 = sm[base], x1 = sm[base + span], x2 = sm[base + 2 * span], x3 = sm[base + 3 * span];
+      gs32(x0, x1, __ldg(pt.IW + m + 2 * i2), t, twot);
+      gs32(x2, x3, __ldg(pt.IW + m + 2 * i2 + 1), t, twot);
+      const uint2 w = __ldg(pt.IW + (m >> 1) + i2);
+      gs32(x0, x2, w, t, twot);
+      gs32(x1, x3, w, t, twot);
+      sm[base] = x0;
+      sm[base + span] = x1;
+      sm[base + 2 * span] = x2;
+      sm[base + 3 * span] = x3;
+    }
+    __syncthreads();
+  }
+  if (lt < logn) {  // odd number of stages: the last one (m = 1)
+    const u32 span = 1u << lt;
+    const uint2 w = __ldg(pt.IW + 1);
     for (u32 b = threadIdx.x; b < (n >> 1); b += blockDim.x) {
-      const u32 i = b >> lt, jj = b & ((1u << lt) - 1);
-      const u32 idx = (i << (lt + 1)) + jj;
-      const u32 X = sm[idx], Y = sm[idx + (1u << lt)];
-      const uint2 w = __ldg(pt.IW + m + i);
-      sm[idx] = csub32(X + Y, twot);
-      sm[idx + (1u << lt)] = shoup32_lazy(X - Y + twot, w, t);
+      u32 x0 = sm[b], x1 = sm[b + span];
+      gs32(x0, x1, w, t, twot);
+      sm[b] = x0;
+      sm[b + span] = x1;
     }
     __syncthreads();
   }
@@ -156,6 +187,7 @@ __global__ void __launch_bounds__(1024)
   for (u32 j = threadIdx.x; j < n; j += blockDim.x) out[j] = csub32(shoup32_lazy(sm[j], ninv, t), t);
 }
 
+// decode: forward transform (two stages per barrier), slots read back from bit-reversed positions
 __global__ void __launch_bounds__(1024)
     k_decode(DevView v, const u32* __restrict__ plain, int32_t* __restrict__ values) {
   u32* sm = reinterpret_cast<u32*>(smem_raw);
@@ -165,16 +197,35 @@ __global__ void __launch_bounds__(1024)
   int32_t* out = values + (size_t)blockIdx.x * n;
   for (u32 j = threadIdx.x; j < n; j += blockDim.x) sm[j] = in[j];
   __syncthreads();
-  u32 lt = logn - 1;
-  for (u32 m = 1; m < n; m <<= 1, --lt) {
+  int lt = (int)logn - 1;  // log2 span of the next stage (m = n >> (lt + 1) groups)
+  if (logn & 1u) {  // odd number of stages: do the first one (m = 1) alone
+    const u32 span = 1u << lt;
+    const uint2 w = __ldg(pt.W + 1);
     for (u32 b = threadIdx.x; b < (n >> 1); b += blockDim.x) {
-      const u32 i = b >> lt, jj = b & ((1u << lt) - 1);
-      const u32 idx = (i << (lt + 1)) + jj;
-      const u32 X = csub32(sm[idx], twot);
-      const uint2 w = __ldg(pt.W + m + i);
-      const u32 T = shoup32_lazy(sm[idx + (1u << lt)], w, t);
-      sm[idx] = X + T;
-      sm[idx + (1u << lt)] = X - T + twot;
+      u32 x0 = sm[b], x1 = sm[b + span];
+      ct32(x0, x1, w, t, twot);
+      sm[b] = x0;
+      sm[b + span] = x1;
+    }
+    __syncthreads();
+    --lt;
+  }
+  for (; lt >= 1; lt -= 2) {
+    // stages with spans 2^lt (m2 groups) then 2^(lt-1) (2 m2 groups)
+    const u32 span = 1u << (lt - 1), m2 = n >> (lt + 1);
+    for (u32 b = threadIdx.x; b < (n >> 2); b += blockDim.x) {
+      const u32 i2 = b >> (lt - 1), jj = b & (span - 1);
+      const u32 base = (i2 << (lt + 1)) + jj;
+      u32 x0 = sm[base], x1 = sm[base + span], x2 = sm[base + 2 * span], x3 = sm[base + 3 * span];
+      const uint2 w = __ldg(pt.W + m2 + i2);
+      ct32(x0, x2, w, t, twot);
+      ct32(x1, x3, w, t, twot);
+      ct32(x0, x1, __ldg(pt.W + 2 * m2 + 2 * i2), t, twot);
+      ct32(x2, x3, __ldg(pt.W + 2 * m2 + 2 * i2 + 1), t, twot);
+      sm[base] = x0;
+      sm[base + span] = x1;
+      sm[base + 2 * span] = x2;
+      sm[base + 3 * span] = x3;
     }
     __syncthreads();
   }
@@ -223,7 +274,7 @@ cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 
   const size_t smem = (size_t)v.n * 4;
   cudaError_t e = set_smem(k_encode, smem);
   if (e != cudaSuccess) return e;
-  u32 threads = v.n / 2 < 1024 ? (v.n / 2 < 32 ? 32 : v.n / 2) : 1024;
+  u32 threads = v.n / 4 < 1024 ? (v.n / 4 < 32 ? 32 : v.n / 4) : 1024;
   k_encode<<<n_cts, threads, smem, s>>>(v, values, plain);
   return cudaGetLastError();
 }
@@ -232,7 +283,7 @@ cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts
   const size_t smem = (size_t)v.n * 4;
   cudaError_t e = set_smem(k_decode, smem);
   if (e != cudaSuccess) return e;
-  u32 threads = v.n / 2 < 1024 ? (v.n / 2 < 32 ? 32 : v.n / 2) : 1024;
+  u32 threads = v.n / 4 < 1024 ? (v.n / 4 < 32 ? 32 : v.n / 4) : 1024;
   k_decode<<<n_cts, threads, smem, s>>>(v, plain, values);
   return cudaGetLastError();
 }
