@@ -35,7 +35,10 @@ __global__ void __launch_bounds__(256)
   ulonglong2* out = reinterpret_cast<ulonglong2*>(agg) + (size_t)unit * ct_pairs;
   for (size_t e = (size_t)blockIdx.y * blockDim.x + threadIdx.x; e < ct_pairs;
        e += (size_t)gridDim.y * blockDim.x) {
-    const u32 l = (u32)(((e * 2) >> v.logn) % v.L);
+    // a block of 256 pairs lies inside one limb row whenever N >= 512: take the row from a
+    // block-uniform index so that the division runs on the uniform datapath
+    const size_t e_row = v.n >= 512 ? e - threadIdx.x : e;
+    const u32 l = (u32)(((e_row * 2) >> v.logn) % v.L);
     const u64 p = v.limbs[l].p;
     ulonglong2 acc = make_ulonglong2(0, 0);
     for (u32 a = beg; a < end; ++a) {
