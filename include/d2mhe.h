@@ -221,16 +221,22 @@ d2mhe_status d2mhe_poly_muladd(d2mhe_ctx* ctx, const uint64_t* a_dev, const uint
  * One whole private gradient update for ciphertext indices ct_first .. ct_first+n_cts-1
  * of all K parties (Algorithm 2 lines 6-9 and 11 without the model update): encode,
  * encrypt, neighbour sums, shares from every share holder, combine, decode.  Ciphertext
- * indices are processed in chunks so that all protocol messages of a chunk
- * (ciphertexts, aggregates, shares) live in the caller's workspace.
+ * indices are processed in sub-chunks so that all protocol messages of the sub-chunks in
+ * flight (ciphertexts, aggregates, shares) live in the caller's workspace.  Up to three
+ * sub-chunks are in flight at a time on internal streams, so that one sub-chunk's copies
+ * and memory-bound kernels overlap another's arithmetic; the internal streams start after
+ * the work already queued on the context's stream, and the context's stream continues
+ * after they have finished (so the call behaves like one operation on that stream).
  *   values:  int32 [K, n_cts, N]   in
  *   sums:    int32 [K, n_cts, N]   out: sums[i] = sum over list(i) of the values
  *   nbr_offsets / nbr_rows: HOST CSR lists over parties, K lists.
  *   workspace_dev / workspace_bytes: device scratch, at least
- *   d2mhe_round_workspace_bytes(ctx, 1); larger workspaces allow larger chunks.
+ *   d2mhe_round_workspace_bytes(ctx, 1); d2mhe_round_workspace_bytes(ctx, n_cts) holds
+ *   the whole range at once (the fastest choice when it fits); anything in between makes
+ *   more, smaller sub-chunks.  The contents left in the workspace are unspecified.
  * d2mhe_round_device takes device values/sums.  d2mhe_round_host takes HOST values/sums
- * (pinned memory recommended), copies them in and out on the context's stream and
- * returns after the stream has drained.
+ * (pinned memory recommended), copies each sub-chunk in and out on the stream that
+ * computes it and returns after all of it has finished.
  */
 size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* ctx, uint32_t chunk_cts);
 d2mhe_status d2mhe_round_device(d2mhe_ctx* ctx, const int32_t* values_dev, uint32_t ct_first,

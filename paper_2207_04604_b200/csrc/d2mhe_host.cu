@@ -383,6 +383,15 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
     if (err != cudaSuccess) return fail_cuda(c, err);
     c->idx_event_valid[i] = false;
   }
+  // lanes of the whole-round entry points
+  for (int i = 0; i < kRoundLanes; ++i) {
+    err = cudaStreamCreateWithFlags(&c->lane_stream[i], cudaStreamNonBlocking);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    err = cudaEventCreateWithFlags(&c->lane_event[i], cudaEventDisableTiming);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+  }
+  err = cudaEventCreateWithFlags(&c->fork_event, cudaEventDisableTiming);
+  if (err != cudaSuccess) return fail_cuda(c, err);
   return D2MHE_OK;
 }
 
@@ -469,6 +478,11 @@ void d2mhe_destroy(d2mhe_ctx* c) {
   if (c->idx_host) cudaFreeHost(c->idx_host);
   for (int i = 0; i < kIdxSlots; ++i)
     if (c->idx_event[i]) cudaEventDestroy(c->idx_event[i]);
+  for (int i = 0; i < kRoundLanes; ++i) {
+    if (c->lane_event[i]) cudaEventDestroy(c->lane_event[i]);
+    if (c->lane_stream[i]) cudaStreamDestroy(c->lane_stream[i]);
+  }
+  if (c->fork_event) cudaEventDestroy(c->fork_event);
   delete c;
 }
 
@@ -854,62 +868,112 @@ size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* c, u32 chunk_cts) {
   return round_bytes_per_ct(c) * chunk_cts + 256;
 }
 
+// The ciphertext-index range is cut into sub-chunks that are issued in turn on a few
+// internal streams ("lanes"), each with its own part of the workspace: one lane's copies,
+// memory-bound kernels and partial last waves overlap the other lane's arithmetic.  The
+// lanes start after everything queued on the context's stream so far and the context's
+// stream continues after all of them have finished.
 static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io, u32 ct_first,
                                u32 n_cts, const u32* nbr_offsets, const u32* nbr_rows,
                                int32_t* sums, void* ws, size_t ws_bytes) {
-  if (!c || !values || !sums || !nbr_offsets || !nbr_rows || !ws || n_cts == 0)
-    return D2MHE_ERR_INVALID_ARG;
+  if (!c || !values || !sums || !nbr_offsets || !ws || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
   if (!aligned16(ws) || (!host_io && (!aligned16(values) || !aligned16(sums))))
     return D2MHE_ERR_INVALID_ARG;
   if (!protocol_ok(c) || !c->can_pack) return D2MHE_ERR_UNSUPPORTED;
   if (!c->has_pk) return D2MHE_ERR_STATE;
-  const u32 K = c->params.num_parties, S = (u32)c->pk_parties.size();
-  const size_t n = c->view.n, polyw = (size_t)c->view.L * n;
+  const u32 K = c->params.num_parties, S = (u32)c->pk_parties.size(), L = c->view.L;
+  if ((u64)ct_first + n_cts > 0x100000000ull) return D2MHE_ERR_RANGE;
+  if (nbr_offsets[0] != 0) return D2MHE_ERR_INVALID_ARG;
+  for (u32 i = 0; i < K; ++i)
+    if (nbr_offsets[i + 1] < nbr_offsets[i]) return D2MHE_ERR_INVALID_ARG;
+  const u32 nnz = nbr_offsets[K];
+  if (nnz > 1048576) return D2MHE_ERR_RANGE;
+  if (nnz && !nbr_rows) return D2MHE_ERR_INVALID_ARG;
+  for (u32 a = 0; a < nnz; ++a)
+    if (nbr_rows[a] >= K) return D2MHE_ERR_RANGE;
+  const size_t n = c->view.n, polyw = (size_t)L * n;
   const size_t per_ct = round_bytes_per_ct(c);
   if (ws_bytes < per_ct + 256) return D2MHE_ERR_WORKSPACE;
-  u32 chunk = (u32)std::min<size_t>((ws_bytes - 256) / per_ct, n_cts);
-  // The in/out staging of the host variant lives in the plain/decoded area of the chunk.
-  std::vector<u32> all(K);
-  for (u32 i = 0; i < K; ++i) all[i] = i;
+  const size_t cap = (ws_bytes - 256) / per_ct;  // ciphertext indices the workspace holds
+  const u32 lanes = (u32)std::min<size_t>(std::min<size_t>(kRoundLanes, cap), n_cts);
+  const size_t grid_cap = 0x7fffffffull / ((u64)K * std::max(L, 2u));  // launch-grid limit of the kernels
+  // Fewest sub-chunks (a whole number of passes over the lanes, sizes differing by at most one,
+  // larger ones first) such that the first pass, which holds the largest ones, fits the workspace.
+  u32 n_sub = lanes;
+  for (;; n_sub += lanes) {
+    if (n_sub >= n_cts) {
+      n_sub = n_cts;
+      break;
+    }
+    const u32 small = n_cts / n_sub, n_big = n_cts % n_sub;
+    size_t first_pass = 0;
+    for (u32 l = 0; l < lanes; ++l) first_pass += small + (l < n_big ? 1u : 0u);
+    if (first_pass <= cap && small + (n_big ? 1u : 0u) <= grid_cap) break;
+  }
+  const u32 sub_small = n_cts / n_sub, n_large = n_cts % n_sub;  // the first n_large get one more
+  size_t lane_first[kRoundLanes + 1] = {};                       // lane l starts this many indices into the workspace
+  for (u32 l = 0; l < lanes; ++l) lane_first[l + 1] = lane_first[l] + sub_small + (l < n_large ? 1u : 0u);
 
   DeviceGuard guard(c->device);
+  std::vector<u32> all(K);
+  for (u32 i = 0; i < K; ++i) all[i] = i;
+  const u32 dummy = 0;
+  Staged sg;  // the four index lists of every sub-chunk, staged once
+  const u32* arrays[4] = {all.data(), c->pk_parties.data(), nbr_offsets, nnz ? nbr_rows : &dummy};
+  const size_t counts[4] = {K, S, (size_t)K + 1, nnz ? (size_t)nnz : 1};
+  d2mhe_status st = stage_indices(c, arrays, counts, 4, &sg);
+  if (st != D2MHE_OK) return st;
+  cudaError_t e;
+  if (lanes > 1) {
+    if ((e = cudaEventRecord(c->fork_event, c->stream)) != cudaSuccess) return fail_cuda(c, e);
+    for (u32 l = 0; l < lanes; ++l)
+      if ((e = cudaStreamWaitEvent(c->lane_stream[l], c->fork_event, 0)) != cudaSuccess) return fail_cuda(c, e);
+  }
   unsigned char* base = reinterpret_cast<unsigned char*>(ws);
-  for (u32 done = 0; done < n_cts; done += chunk) {
-    const u32 cc = std::min(chunk, n_cts - done);
-    // layout for this chunk (all 16-byte aligned: every block is a multiple of 16 bytes)
-    u32* plain = reinterpret_cast<u32*>(base);
-    u64* ct = reinterpret_cast<u64*>(base + (size_t)K * cc * n * sizeof(u32));
+  u32 done = 0;
+  for (u32 i = 0; i < n_sub; ++i) {
+    const u32 cc = sub_small + (i < n_large ? 1u : 0u), lane = i % lanes;
+    cudaStream_t s = lanes > 1 ? c->lane_stream[lane] : c->stream;
+    // layout of the lane's part (all 16-byte aligned: every block is a multiple of 16 bytes)
+    unsigned char* lane_base = base + lane_first[lane] * per_ct;
+    u32* plain = reinterpret_cast<u32*>(lane_base);
+    u64* ct = reinterpret_cast<u64*>(lane_base + (size_t)K * cc * n * sizeof(u32));
     u64* agg = ct + (size_t)K * cc * 2 * polyw;
     u64* shares = agg + (size_t)K * cc * 2 * polyw;
-    // values are [K, n_cts, N]: gather the chunk's columns party by party
-    int32_t* vals_dev = reinterpret_cast<int32_t*>(plain);  // encode runs in place
-    {  // one strided copy: K rows of cc*N values, source rows n_cts*N apart
-      cudaError_t e = cudaMemcpy2DAsync(vals_dev, (size_t)cc * n * sizeof(int32_t), values + (size_t)done * n,
-                                        (size_t)n_cts * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
-                                        host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, c->stream);
-      if (e != cudaSuccess) return fail_cuda(c, e);
-    }
-    d2mhe_status st;
-    if ((st = d2mhe_encode(c, vals_dev, K * cc, plain)) != D2MHE_OK) return st;
-    if ((st = d2mhe_encrypt(c, all.data(), K, ct_first + done, cc, plain, reinterpret_cast<uint64_t*>(ct))) != D2MHE_OK) return st;
-    if ((st = d2mhe_aggregate(c, reinterpret_cast<uint64_t*>(ct), K, cc, nbr_offsets, nbr_rows, K,
-                              reinterpret_cast<uint64_t*>(agg))) != D2MHE_OK) return st;
-    if ((st = d2mhe_partial_decrypt(c, reinterpret_cast<uint64_t*>(agg), all.data(), K,
-                                    c->pk_parties.data(), S, ct_first + done, cc,
-                                    reinterpret_cast<uint64_t*>(shares))) != D2MHE_OK)
-      return st;
-    if ((st = d2mhe_combine_decrypt(c, reinterpret_cast<uint64_t*>(agg), reinterpret_cast<uint64_t*>(shares),
-                                    K, S, cc, plain)) != D2MHE_OK) return st;
-    if ((st = d2mhe_decode(c, plain, K * cc, vals_dev)) != D2MHE_OK) return st;
-    {
-      cudaError_t e = cudaMemcpy2DAsync(sums + (size_t)done * n, (size_t)n_cts * n * sizeof(int32_t), vals_dev,
-                                        (size_t)cc * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
-                                        host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, c->stream);
-      if (e != cudaSuccess) return fail_cuda(c, e);
+    int32_t* vals_dev = reinterpret_cast<int32_t*>(plain);  // encode and decode run in place
+    // values are [K, n_cts, N]: one strided copy, K rows of cc*N values, rows n_cts*N apart
+    e = cudaMemcpy2DAsync(vals_dev, (size_t)cc * n * sizeof(int32_t), values + (size_t)done * n,
+                          (size_t)n_cts * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
+                          host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    if ((e = d2mhe_launch::encode(c->view, s, vals_dev, K * cc, plain)) != cudaSuccess) return fail_cuda(c, e);
+    if ((e = d2mhe_launch::encrypt(c->view, c->limb_params, s, sg.dev[0], K, ct_first + done, cc, plain, ct)) !=
+        cudaSuccess)
+      return fail_cuda(c, e);
+    if ((e = d2mhe_launch::aggregate(c->view, s, ct, cc, sg.dev[2], sg.dev[3], K, agg)) != cudaSuccess)
+      return fail_cuda(c, e);
+    if ((e = d2mhe_launch::partial_decrypt(c->view, c->limb_params, s, agg, sg.dev[0], K, sg.dev[1], S,
+                                           ct_first + done, cc, shares)) != cudaSuccess)
+      return fail_cuda(c, e);
+    if ((e = d2mhe_launch::combine(c->view, s, agg, shares, K, S, 1, cc, plain)) != cudaSuccess)
+      return fail_cuda(c, e);
+    if ((e = d2mhe_launch::decode(c->view, s, plain, K * cc, vals_dev)) != cudaSuccess) return fail_cuda(c, e);
+    c->launches += 6;
+    e = cudaMemcpy2DAsync(sums + (size_t)done * n, (size_t)n_cts * n * sizeof(int32_t), vals_dev,
+                          (size_t)cc * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
+                          host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    done += cc;
+  }
+  if (lanes > 1) {
+    for (u32 l = 0; l < lanes; ++l) {
+      if ((e = cudaEventRecord(c->lane_event[l], c->lane_stream[l])) != cudaSuccess) return fail_cuda(c, e);
+      if ((e = cudaStreamWaitEvent(c->stream, c->lane_event[l], 0)) != cudaSuccess) return fail_cuda(c, e);
     }
   }
+  if ((st = release_slot(c, sg)) != D2MHE_OK) return st;
   if (host_io) {
-    cudaError_t e = cudaStreamSynchronize(c->stream);
+    e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) return fail_cuda(c, e);
   }
   return D2MHE_OK;

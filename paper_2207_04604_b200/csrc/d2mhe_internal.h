@@ -59,6 +59,10 @@ struct DevView {
 
 static const size_t kIdxSlotWords = (size_t)1 << 21;  // u32 words per staging slot (8 MiB)
 static const int kIdxSlots = 4;
+#ifndef D2MHE_ROUND_LANES
+#define D2MHE_ROUND_LANES 3
+#endif
+static const int kRoundLanes = D2MHE_ROUND_LANES;  // internal streams of the whole-round entry points
 
 struct d2mhe_ctx {
   d2mhe_params params;
@@ -82,6 +86,9 @@ struct d2mhe_ctx {
   cudaEvent_t idx_event[kIdxSlots] = {};
   bool idx_event_valid[kIdxSlots] = {};
   int idx_next = 0;
+  cudaStream_t lane_stream[kRoundLanes] = {};
+  cudaEvent_t lane_event[kRoundLanes] = {};
+  cudaEvent_t fork_event = nullptr;
   cudaError_t last_cuda = cudaSuccess;
 };
 

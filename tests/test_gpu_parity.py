@@ -563,12 +563,40 @@ def test_round_driver_matches_stepwise_and_plain_sums(d2):
     values = wl.gradients(cfg, seed)
     want = np.stack([values[rows[offsets[i]:offsets[i + 1]]].astype(np.int64).sum(axis=0) for i in range(K)])
     dv = torch.from_numpy(values).to(ctx.device)
-    for chunk in (1, 5, C):
+    for chunk in (1, 2, 5, C, C + 3):
         ws = torch.empty(ctx.round_workspace_bytes(chunk), dtype=torch.uint8, device=ctx.device)
         sums = torch.zeros((K, C, n), dtype=torch.int32, device=ctx.device)
         ctx.round_device(dv, 0, C, offsets, rows, sums, ws)
         ctx.sync()
         assert np.array_equal(sums.cpu().numpy(), want)
+    # The messages themselves, not only the sums: a workspace for three indices makes thirteen
+    # one-index sub-chunks that rotate over three parts of it, so that at the end the parts hold
+    # indices 12, 10 and 11, each as [plain | ciphertexts | aggregates | shares].  They must be
+    # the messages the step-by-step calls produce for those indices.
+    L = cfg.num_limbs
+    ws = torch.empty(ctx.round_workspace_bytes(3), dtype=torch.uint8, device=ctx.device)
+    sums = torch.zeros((K, C, n), dtype=torch.int32, device=ctx.device)
+    ctx.round_device(dv, 0, C, offsets, rows, sums, ws)
+    ctx.sync()
+    assert np.array_equal(sums.cpu().numpy(), want)
+    per_ct = ctx.round_workspace_bytes(1) - 256
+    ct_words, share_words = K * 2 * L * n, K * K * L * n
+    assert per_ct == 4 * K * n + 8 * (2 * ct_words + share_words)
+    held = ws.cpu().numpy()
+    for part, index in enumerate((12, 10, 11)):
+        plain = ctx.empty_u32(K, 1, n)
+        ct = ctx.empty_u64(K, 1, 2, L, n)
+        agg = ctx.empty_u64(K, 1, 2, L, n)
+        shares = ctx.empty_u64(K, K, 1, L, n)
+        ctx.encode(dv[:, index:index + 1].contiguous(), K, plain)
+        ctx.encrypt(parties, index, 1, plain, ct)
+        ctx.aggregate(ct, K, 1, offsets, rows, agg)
+        ctx.partial_decrypt(agg, parties, parties, index, 1, shares)
+        ctx.sync()
+        words = held[part * per_ct + 4 * K * n:(part + 1) * per_ct].view(np.uint64)
+        assert np.array_equal(words[:ct_words], d2.to_u64_numpy(ct).ravel())
+        assert np.array_equal(words[ct_words:2 * ct_words], d2.to_u64_numpy(agg).ravel())
+        assert np.array_equal(words[2 * ct_words:], d2.to_u64_numpy(shares).ravel())
     # host variant, pinned buffers
     hv = torch.from_numpy(values).pin_memory()
     hs = torch.zeros((K, C, n), dtype=torch.int32).pin_memory()
