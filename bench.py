@@ -485,7 +485,9 @@ def run_sweep(args):
     """Kernel sweep (configuration 5): batched forward/inverse transforms and the RNS multiply-add over
     N in 2^12..2^16, L in {1,4,8,16,24}, batch in {1,64,1024,4096}, uniform residues mod 60-bit primes
     (50-bit with --sweep-bits 50).  One JSON line with a row per point; GB/s = 16 B (transforms) or 32 B
-    (multiply-add) per residue over the CUDA-event time, against the measured HBM copy bandwidth."""
+    (multiply-add) per residue over the CUDA-event time, against the measured HBM copy bandwidth.
+    --sweep-bits 30 (or less) runs the 32-bit-word calls instead: 8 and 16 B per residue, N up to 2^14
+    for the transforms."""
     import torch
 
     from paper_2207_04604_b200 import build, d2mhe
@@ -504,9 +506,14 @@ def run_sweep(args):
         for L in wl.SWEEP_LIMBS:
             moduli = wl.sweep_moduli(args.sweep_bits, L)
             ctx = d2mhe.Context(log2_n, moduli, 1, seed=args.seed)
-            tile = torch.from_numpy(wl.random_polys(moduli, log2_n, 1, args.seed).view(np.int64)).to(dev)
+            narrow = args.sweep_bits <= 30
+            word = 4 if narrow else 8
+            host_tile = wl.random_polys(moduli, log2_n, 1, args.seed)
+            tile = torch.from_numpy(host_tile.astype(np.uint32).view(np.int32) if narrow else host_tile.view(np.int64)).to(dev)
+            fwd, inv, mad = ((ctx.ntt32_forward, ctx.ntt32_inverse, ctx.poly_muladd32) if narrow
+                             else (ctx.ntt_forward, ctx.ntt_inverse, ctx.poly_muladd))
             for batch in wl.SWEEP_BATCH:
-                nbytes = 8 * n * L * batch
+                nbytes = word * n * L * batch
                 row = {"N": n, "L": L, "batch": batch, "GiB": nbytes / 2**30}
                 if nbytes > 0.6 * free_b:
                     row["skipped"] = "buffer exceeds the memory budget"
@@ -528,12 +535,13 @@ def run_sweep(args):
                         best = ms if best is None else min(best, ms)
                     return best
 
-                f_ms = timed(lambda: ctx.ntt_forward(polys, batch))
-                i_ms = timed(lambda: ctx.ntt_inverse(polys, batch))
-                row.update({"forward_GBps": 2 * nbytes / 1e9 / (f_ms * 1e-3), "inverse_GBps": 2 * nbytes / 1e9 / (i_ms * 1e-3)})
+                if not narrow or log2_n <= 14:
+                    f_ms = timed(lambda: fwd(polys, batch))
+                    i_ms = timed(lambda: inv(polys, batch))
+                    row.update({"forward_GBps": 2 * nbytes / 1e9 / (f_ms * 1e-3), "inverse_GBps": 2 * nbytes / 1e9 / (i_ms * 1e-3)})
                 if 4 * nbytes <= 0.6 * free_b:
                     b2, c2, d2_ = polys.clone(), polys.clone(), torch.empty_like(polys)
-                    m_ms = timed(lambda: ctx.poly_muladd(polys, b2, c2, d2_, batch))
+                    m_ms = timed(lambda: mad(polys, b2, c2, d2_, batch))
                     row["muladd_GBps"] = 4 * nbytes / 1e9 / (m_ms * 1e-3)
                     del b2, c2, d2_
                 row["in_l2_or_launch_bound"] = bool(nbytes < 2 * 126e6 or batch * L < NUM_SMS)
@@ -545,8 +553,8 @@ def run_sweep(args):
                 torch.cuda.empty_cache()
             ctx.close()
     print(json.dumps({"metric": METRIC, "unit": "GB/s", "config": {"workload": "kernel-sweep", "prime_bits": args.sweep_bits},
-                      "hbm_peak_GBps": peak, "peak_source": "of " + peak_kind, "dtype": "u64", "data": "synthetic",
-                      "rows": rows}))
+                      "hbm_peak_GBps": peak, "peak_source": "of " + peak_kind,
+                      "dtype": "u32" if args.sweep_bits <= 30 else "u64", "data": "synthetic", "rows": rows}))
 
 
 def main():
@@ -559,7 +567,7 @@ def main():
     ap.add_argument("--seed", type=int, default=1)
     ap.add_argument("--chunk", type=int, default=0, help="ciphertext indices per chunk (0: as many as fit)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sweep-bits", type=int, default=60, choices=[50, 60])
+    ap.add_argument("--sweep-bits", type=int, default=60, choices=[30, 50, 60])
     args = ap.parse_args()
     if args.config == 5:
         return run_sweep(args)

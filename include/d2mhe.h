@@ -105,7 +105,7 @@ d2mhe_status d2mhe_decode(d2mhe_ctx* ctx, const uint32_t* plain_dev, uint32_t n_
                           int32_t* values_dev);
 
 /*
- * BFV.Encrypt under the collective key (Sec. 3.2 item 3; Algorithm 2 lines 6, 11):
+ * BFV.Encrypt under the collective key (Sec. 3.2 item 3; the encryption steps of Algorithm 2):
  * ct = (Lambda m + u p_0 + e_0, u p_1 + e_1), Lambda = floor(q/t), u from R_3,
  * e_0, e_1 from chi.  The randomness of unit (parties[a], c) is the stream
  * (party = parties[a], ciphertext index = ct_first + c).
@@ -116,7 +116,7 @@ d2mhe_status d2mhe_encrypt(d2mhe_ctx* ctx, const uint32_t* parties, uint32_t n_p
                            uint64_t* ct_dev);
 
 /*
- * BFV.Add over neighbour lists (Sec. 3.2 item 4; Algorithm 2 line 6 with unit weights):
+ * BFV.Add over neighbour lists (Sec. 3.2 item 4; the neighbour-sum step of Algorithm 2, with unit weights):
  * agg[i, c] = sum_{r in list(i)} ct[r, c] mod q, both components.
  * ct_dev: [n_rows, n_cts, 2, L, N].  nbr_offsets (HOST, n_out+1 entries, non-decreasing,
  * nbr_offsets[0] = 0) and nbr_rows (HOST, nbr_offsets[n_out] entries, each < n_rows) are
@@ -152,7 +152,7 @@ d2mhe_status d2mhe_combine_decrypt(d2mhe_ctx* ctx, const uint64_t* agg_dev,
                                    uint32_t n_shares, uint32_t n_cts, uint32_t* plain_dev);
 
 /*
- * MBFV.Convert (Sec. 4.2 item 3, Eq. 2-3; Algorithm 2 lines 8-9): re-encryption of an aggregate
+ * MBFV.Convert (Sec. 4.2 item 3, Eq. 2-3; the decryption steps of Algorithm 2): re-encryption of an aggregate
  * from the collective key to the recipient's OWN key pair, followed by BFV.Decrypt under it.
  *
  * d2mhe_user_keygen: every listed user i generates sk_i <- R_3 and
@@ -218,8 +218,21 @@ d2mhe_status d2mhe_poly_muladd(d2mhe_ctx* ctx, const uint64_t* a_dev, const uint
                                const uint64_t* c_dev, uint64_t* d_dev, uint32_t batch);
 
 /*
+ * The same three operations on 32-bit words, for parameter sets whose primes are all below
+ * 2^30 (D2MHE_ERR_UNSUPPORTED otherwise): polynomials are uint32 [batch, L, N], residues in
+ * [0, q_l).  Half the bytes and less than a third of the multiplier work of the 64-bit calls per
+ * coefficient; a ciphertext modulus of the same size needs about twice the limbs.  The
+ * transforms need log2_n <= 14 (two polynomials of the batch share one thread block and
+ * shared memory); results are defined exactly as for the 64-bit calls.
+ */
+d2mhe_status d2mhe_ntt32_forward(d2mhe_ctx* ctx, uint32_t* polys_dev, uint32_t batch);
+d2mhe_status d2mhe_ntt32_inverse(d2mhe_ctx* ctx, uint32_t* polys_dev, uint32_t batch);
+d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* ctx, const uint32_t* a_dev, const uint32_t* b_dev,
+                                 const uint32_t* c_dev, uint32_t* d_dev, uint32_t batch);
+
+/*
  * One whole private gradient update for ciphertext indices ct_first .. ct_first+n_cts-1
- * of all K parties (Algorithm 2 lines 6-9 and 11 without the model update): encode,
+ * of all K parties (Algorithm 2 from encryption to decryption, without the model update): encode,
  * encrypt, neighbour sums, shares from every share holder, combine, decode.  Ciphertext
  * indices are processed in sub-chunks so that all protocol messages of the sub-chunks in
  * flight (ciphertexts, aggregates, shares) live in the caller's workspace.  Up to three

@@ -668,7 +668,7 @@ void orc_encrypt(const orc_params* P, const uint64_t* pk, uint32_t party, uint32
 }
 
 /*
- * BFV.Add over a list (Algorithm 2 line 6 with unit weights): out = sum of the
+ * BFV.Add over a list (the neighbour-sum step of Algorithm 2, with unit weights): out = sum of the
  * listed ciphertexts, component by component, mod q.  cts is [n_rows][2][L][N].
  */
 void orc_aggregate(const orc_params* P, const uint64_t* cts, const uint32_t* rows,

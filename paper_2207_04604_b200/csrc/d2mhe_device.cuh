@@ -246,17 +246,58 @@ __device__ __forceinline__ u64 reduce_small(u64 x, const Mod& m) {
   return join64(rl, madlo(q, nh, rh));
 }
 
+// Arithmetic mode of the engine: 0 = one residue per word, primes up to 2^61; 1 = the same with
+// the WIDE policy above (primes below 2^57); 2 = "pair": every 64-bit word carries two 32-bit
+// residues of the same prime below 2^30 (two polynomials transformed side by side with the
+// same twiddles), each half with Harvey's lazy butterflies in 32-bit arithmetic: one high and
+// two low multiplies per butterfly instead of five and four.
+enum : int { MODE_STRICT = 0, MODE_WIDE = 1, MODE_PAIR = 2 };
+
+__device__ __forceinline__ u32 csub32(u32 x, u32 p) { return min(x, x - p); }  // x - p wraps above x when x < p
+// y*w mod p in [0, 2p) for any 32-bit y, given ws = floor(w 2^32 / p), p < 2^31
+__device__ __forceinline__ u32 shoup32(u32 y, u32 w, u32 ws, u32 p) { return y * w - mulhi32(y, ws) * p; }
+// The 32-bit companion is the high half of the 64-bit one: floor(floor(w 2^64 / p) / 2^32).
+__device__ __forceinline__ void ct_bfly_pair(u64& X, u64& Y, const ulonglong2 w, const Mod& m) {
+  const u32 p = (u32)m.p, twop = (u32)m.twop, wl = (u32)w.x, ws = (u32)(w.y >> 32);
+  u32 xa, xb, ya, yb;
+  split64(X, xa, xb);
+  split64(Y, ya, yb);
+  xa = csub32(xa, twop);  // inputs below 4p, kept below 4p
+  xb = csub32(xb, twop);
+  const u32 ta = shoup32(ya, wl, ws, p), tb = shoup32(yb, wl, ws, p);
+  X = join64(xa + ta, xb + tb);
+  Y = join64(xa - ta + twop, xb - tb + twop);
+}
+__device__ __forceinline__ void gs_bfly_pair(u64& X, u64& Y, const ulonglong2 w, const Mod& m) {
+  const u32 p = (u32)m.p, twop = (u32)m.twop, wl = (u32)w.x, ws = (u32)(w.y >> 32);
+  u32 xa, xb, ya, yb;
+  split64(X, xa, xb);
+  split64(Y, ya, yb);
+  X = join64(csub32(xa + ya, twop), csub32(xb + yb, twop));  // inputs below 2p, kept below 2p
+  Y = join64(shoup32(xa - ya + twop, wl, ws, p), shoup32(xb - yb + twop, wl, ws, p));
+}
+
 // forward (Cooley-Tukey): (X, Y) -> (X + wY, X - wY)
-template <bool WIDE>
+template <int MODE>
 __device__ __forceinline__ void ct_bfly(u64& X, u64& Y, const ulonglong2 w, const Mod& m) {
+  if (MODE == MODE_PAIR) {
+    ct_bfly_pair(X, Y, w, m);
+    return;
+  }
+  constexpr bool WIDE = MODE == MODE_WIDE;
   const u64 x = WIDE ? X : csub(X, m.fourp);
   const u64 t = shoup_approx(Y, w.x, w.y, m.np);  // [0,4p)
   X = x + t;
   Y = x - t + m.fourp;
 }
 // inverse (Gentleman-Sande): (X, Y) -> (X + Y, w(X - Y)); c >= bound of Y, a multiple of p
-template <bool WIDE>
+template <int MODE>
 __device__ __forceinline__ void gs_bfly(u64& X, u64& Y, const ulonglong2 w, const Mod& m, u64 c) {
+  if (MODE == MODE_PAIR) {
+    gs_bfly_pair(X, Y, w, m);
+    return;
+  }
+  constexpr bool WIDE = MODE == MODE_WIDE;
   const u64 s = X + Y;
   const u64 d = X - Y + (WIDE ? c : m.fourp);
   X = WIDE ? s : csub(s, m.fourp);
@@ -264,7 +305,7 @@ __device__ __forceinline__ void gs_bfly(u64& X, u64& Y, const ulonglong2 w, cons
 }
 
 // three (or fewer) forward stages on an octet; m = groups at the first stage, i = group index
-template <bool WIDE>
+template <int WIDE>
 __device__ __forceinline__ void fwd_octet(u64 (&x)[8], const ulonglong2* __restrict__ W, u32 m,
                                           u32 i, int nst, const Mod& md) {
   {
@@ -290,7 +331,7 @@ __device__ __forceinline__ void fwd_octet(u64 (&x)[8], const ulonglong2* __restr
 // Inverse stages on an octet whose inputs are all below 16p (WIDE) / 4p (otherwise).
 // WIDE bounds after the round: x0 < 128p, x1 < 16p, x2, x3 < 8p, x4..x7 < 4p; x0 is brought
 // back below 4p here, so every output is again below 16p.
-template <bool WIDE>
+template <int MODE>
 __device__ __forceinline__ void inv_octet(u64 (&x)[8], const ulonglong2* __restrict__ IW, u32 m,
                                           u32 i, int nst, const Mod& md) {
   const u64 c16 = md.fourp << 2, c32 = md.fourp << 3, c64 = md.fourp << 4;
@@ -298,30 +339,30 @@ __device__ __forceinline__ void inv_octet(u64 (&x)[8], const ulonglong2* __restr
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       const ulonglong2 w = __ldg(IW + 4 * m + 4 * i + r);
-      gs_bfly<WIDE>(x[2 * r], x[2 * r + 1], w, md, c16);
+      gs_bfly<MODE>(x[2 * r], x[2 * r + 1], w, md, c16);
     }
   }
   if (nst >= 2) {
     const ulonglong2 w0 = __ldg(IW + 2 * m + 2 * i), w1 = __ldg(IW + 2 * m + 2 * i + 1);
-    gs_bfly<WIDE>(x[0], x[2], w0, md, c32);
-    gs_bfly<WIDE>(x[1], x[3], w0, md, c32);
-    gs_bfly<WIDE>(x[4], x[6], w1, md, c32);
-    gs_bfly<WIDE>(x[5], x[7], w1, md, c32);
+    gs_bfly<MODE>(x[0], x[2], w0, md, c32);
+    gs_bfly<MODE>(x[1], x[3], w0, md, c32);
+    gs_bfly<MODE>(x[4], x[6], w1, md, c32);
+    gs_bfly<MODE>(x[5], x[7], w1, md, c32);
   }
   {
     const ulonglong2 w = __ldg(IW + m + i);
 #pragma unroll
-    for (int k = 0; k < 4; ++k) gs_bfly<WIDE>(x[k], x[k + 4], w, md, c64);
+    for (int k = 0; k < 4; ++k) gs_bfly<MODE>(x[k], x[k + 4], w, md, c64);
   }
-  if (WIDE) x[0] = reduce_small(x[0], md);
+  if (MODE == MODE_WIDE) x[0] = reduce_small(x[0], md);
 }
 
 // Brings the outputs of the last inverse round below 4p.  After a full round the bounds are
 // those listed at inv_octet; a 2-stage round leaves x1 < 64p, x2, x3 < 8p and a 1-stage round
 // x1..x3 < 32p (x0 has already been reduced, x4..x7 are products).
-template <bool WIDE>
+template <int MODE>
 __device__ __forceinline__ void finish_octet(u64 (&x)[8], int nst, const Mod& md) {
-  if (WIDE) {
+  if (MODE == MODE_WIDE) {
     if (nst >= 3) {
       x[1] = csub(csub(x[1], md.fourp << 1), md.fourp);
     } else {
@@ -394,8 +435,9 @@ __device__ __forceinline__ u64& sm_at(u64* sm, u32 byte_off) {
 //
 // Forward transform.  load(j) returns coefficient j (any lazily reduced value below 8p);
 // emit(g, q, x) receives the octet of positions 8q..8q+7 (lazily reduced values: below 66p when
-// WIDE, below 8p otherwise), q = tid + g*T.
-template <int LOGN, int G, bool WIDE, class Load, class Emit>
+// WIDE, below 8p otherwise), q = tid + g*T.  The third template argument is the arithmetic mode
+// (0 / 1 = not WIDE / WIDE; MODE_PAIR: words are pairs of 32-bit residues below 4p, both ways).
+template <int LOGN, int G, int WIDE, class Load, class Emit>
 __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
                                             Load load, Emit emit, u32 soff = 0, u32 blk = 0) {
   const NttGeom<LOGN, G> ge(logn_rt);
@@ -459,12 +501,12 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
 
 // Inverse transform (without the N^-1 scaling: fold it into an operand).
 // fetch(g, q, x) fills the octet of positions 8q..8q+7 with values below 4p (below 16p when WIDE);
-// store(j, v) receives coefficient j, v in [0,4p).
+// store(j, v) receives coefficient j, v in [0,4p).  MODE_PAIR: halves below 2p in and out.
 struct NoHook {
   __device__ __forceinline__ void operator()() const {}
 };
 // before_final() is called by every thread just before the round that calls store().
-template <int LOGN, int G, bool WIDE, class Fetch, class Store, class Hook = NoHook>
+template <int LOGN, int G, int WIDE, class Fetch, class Store, class Hook = NoHook>
 __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
                                             Fetch fetch, Store store, u32 soff = 0, u32 blk = 0,
                                             Hook before_final = Hook()) {

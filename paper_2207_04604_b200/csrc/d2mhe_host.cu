@@ -444,6 +444,9 @@ d2mhe_status d2mhe_create(const d2mhe_params* P, d2mhe_ctx** out) {
   c->params.moduli = reinterpret_cast<const uint64_t*>(c->moduli.data());
   c->device = P->device;
   c->can_pack = (t - 1) % two_n == 0;
+  c->narrow = true;
+  for (u32 l = 0; l < P->num_limbs; ++l)
+    if (P->moduli[l] >= ((u64)1 << 30)) c->narrow = false;
   c->has_share.assign(P->num_parties, false);
   c->has_user_key.assign(P->num_parties, false);
   std::memset(&c->view, 0, sizeof(c->view));
@@ -685,6 +688,35 @@ d2mhe_status d2mhe_ntt_forward(d2mhe_ctx* c, uint64_t* polys_dev, u32 batch) {
 }
 d2mhe_status d2mhe_ntt_inverse(d2mhe_ctx* c, uint64_t* polys_dev, u32 batch) {
   return ntt_common(c, reinterpret_cast<u64*>(polys_dev), batch, true);
+}
+
+static d2mhe_status ntt32_common(d2mhe_ctx* c, u32* polys_dev, u32 batch, bool inverse) {
+  if (!c || !polys_dev || batch == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(polys_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!c->narrow || !protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  if ((u64)batch * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  cudaError_t e = d2mhe_launch::ntt32(c->view, c->limb_params, c->stream, polys_dev, batch, inverse);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return D2MHE_OK;
+}
+d2mhe_status d2mhe_ntt32_forward(d2mhe_ctx* c, uint32_t* polys_dev, u32 batch) {
+  return ntt32_common(c, polys_dev, batch, false);
+}
+d2mhe_status d2mhe_ntt32_inverse(d2mhe_ctx* c, uint32_t* polys_dev, u32 batch) {
+  return ntt32_common(c, polys_dev, batch, true);
+}
+d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* c, const uint32_t* a, const uint32_t* b, const uint32_t* cc,
+                                 uint32_t* d, u32 batch) {
+  if (!c || !a || !b || !cc || !d || batch == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(a) || !aligned16(b) || !aligned16(cc) || !aligned16(d)) return D2MHE_ERR_INVALID_ARG;
+  if (!c->narrow) return D2MHE_ERR_UNSUPPORTED;
+  DeviceGuard guard(c->device);
+  cudaError_t e = d2mhe_launch::muladd32(c->view, c->stream, a, b, cc, d, batch);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return D2MHE_OK;
 }
 
 d2mhe_status d2mhe_poly_muladd(d2mhe_ctx* c, const uint64_t* a, const uint64_t* b,

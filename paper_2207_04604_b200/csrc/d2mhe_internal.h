@@ -70,6 +70,7 @@ struct d2mhe_ctx {
   std::vector<u64> roots;
   u64 psi_t = 0;
   bool can_pack = false;
+  bool narrow = false;  // every prime below 2^30: the 32-bit-word calls are available
   int device = 0;
   cudaStream_t stream = nullptr;
   DevView view;
@@ -114,6 +115,10 @@ cudaError_t boot_share(const DevView& v, const LimbParams& lp, cudaStream_t s, c
 cudaError_t boot_finish(const DevView& v, cudaStream_t s, const u32* x, const u64* shares,
                         const u32* recipients_dev, u32 n_rec, u32 n_shares, u32 ct_first, u32 n_cts, u64* out);
 cudaError_t ntt(const DevView& v, const LimbParams& lp, cudaStream_t s, u64* polys, u32 batch, bool inverse);
+// 32-bit-word variants (every prime below 2^30)
+cudaError_t ntt32(const DevView& v, const LimbParams& lp, cudaStream_t s, u32* polys, u32 batch, bool inverse);
+cudaError_t muladd32(const DevView& v, cudaStream_t s, const u32* a, const u32* b, const u32* c, u32* d,
+                     u32 batch);
 cudaError_t user_keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* users_dev,
                         u32 n_users);
 cudaError_t convert_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,

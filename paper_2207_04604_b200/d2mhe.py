@@ -27,7 +27,8 @@ EXPORTS = [
     "d2mhe_create", "d2mhe_destroy", "d2mhe_set_stream", "d2mhe_sync", "d2mhe_strerror",
     "d2mhe_keygen_share", "d2mhe_collective_pk", "d2mhe_encode", "d2mhe_decode", "d2mhe_encrypt",
     "d2mhe_aggregate", "d2mhe_partial_decrypt", "d2mhe_combine_decrypt", "d2mhe_ntt_forward",
-    "d2mhe_ntt_inverse", "d2mhe_poly_muladd", "d2mhe_round_workspace_bytes", "d2mhe_round_device",
+    "d2mhe_ntt_inverse", "d2mhe_poly_muladd", "d2mhe_ntt32_forward", "d2mhe_ntt32_inverse",
+    "d2mhe_poly_muladd32", "d2mhe_round_workspace_bytes", "d2mhe_round_device",
     "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_user_keygen", "d2mhe_convert_share",
     "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_bootstrap_share", "d2mhe_bootstrap_combine", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_get_root", "d2mhe_get_plain_root",
     "d2mhe_launch_count",
@@ -238,6 +239,16 @@ class Context:
     def poly_muladd(self, a, b, c, d, batch):
         self._check(load().d2mhe_poly_muladd(self._h, _dev(a, U64), _dev(b, U64), _dev(c, U64), _dev(d, U64), batch),
                     "d2mhe_poly_muladd")
+
+    def ntt32_forward(self, polys, batch):
+        self._check(load().d2mhe_ntt32_forward(self._h, _dev(polys, U32), batch), "d2mhe_ntt32_forward")
+
+    def ntt32_inverse(self, polys, batch):
+        self._check(load().d2mhe_ntt32_inverse(self._h, _dev(polys, U32), batch), "d2mhe_ntt32_inverse")
+
+    def poly_muladd32(self, a, b, c, d, batch):
+        self._check(load().d2mhe_poly_muladd32(self._h, _dev(a, U32), _dev(b, U32), _dev(c, U32), _dev(d, U32), batch),
+                    "d2mhe_poly_muladd32")
 
     def round_workspace_bytes(self, chunk_cts):
         return int(load().d2mhe_round_workspace_bytes(self._h, chunk_cts))

@@ -86,6 +86,81 @@ def test_poly_muladd_against_oracle(d2, log2_n, bits, L, batch):
     ctx.close()
 
 
+# ----------------------------------------------------------------------------------
+# 32-bit-word transforms and multiply-add (every prime below 2^30)
+# ----------------------------------------------------------------------------------
+
+
+@pytest.mark.parametrize("log2_n,bits,L,batch", [
+    (3, 20, 1, 2), (4, 24, 2, 3), (6, 30, 2, 5), (9, 28, 3, 1), (10, 30, 3, 4), (11, 30, 2, 7),
+    (12, 30, 4, 5), (12, 25, 1, 2), (13, 30, 3, 3), (13, 30, 8, 2), (14, 30, 2, 3), (14, 29, 3, 2),
+])
+def test_ntt32_forward_inverse_against_oracle(d2, log2_n, bits, L, batch):
+    """Same definition as the 64-bit transforms; odd batches leave one polynomial without a partner."""
+    moduli = wl.ntt_primes(bits, 2 << log2_n, L)
+    assert max(moduli) < 1 << 30
+    ctx = d2.Context(log2_n, moduli, 2, seed=1)
+    o = make_oracle(log2_n, moduli, seed=1)
+    a = wl.random_polys(moduli, log2_n, batch, seed=100 + log2_n)
+    a[0, :, 0] = 0
+    a[0, :, 1] = np.array(moduli, dtype=np.uint64) - 1
+    a[-1, :, -1] = np.array(moduli, dtype=np.uint64) - 1
+    psi = [ctx.get_root(l) for l in range(L)]
+    want = o.ntt(a, psi)
+    perm = _brv(log2_n)
+    dev = d2.from_u32_numpy(a.astype(np.uint32), ctx.device)
+    ctx.ntt32_forward(dev, batch)
+    got = d2.to_u32_numpy(dev).astype(np.uint64)
+    assert np.array_equal(got, want[..., perm])
+    ctx.ntt32_inverse(dev, batch)
+    ctx.sync()
+    assert np.array_equal(d2.to_u32_numpy(dev).astype(np.uint64), a)
+    dev2 = d2.from_u32_numpy(np.ascontiguousarray(want[..., perm]).astype(np.uint32), ctx.device)
+    ctx.ntt32_inverse(dev2, batch)
+    assert np.array_equal(d2.to_u32_numpy(dev2).astype(np.uint64), a)
+    # the 64-bit calls on the same context and data agree
+    dev64 = d2.from_u64_numpy(a, ctx.device)
+    ctx.ntt_forward(dev64, batch)
+    assert np.array_equal(d2.to_u64_numpy(dev64), want[..., perm])
+    ctx.close()
+
+
+@pytest.mark.parametrize("log2_n,bits,L,batch", [(4, 24, 2, 3), (12, 30, 4, 3), (14, 30, 3, 2), (16, 30, 2, 1)])
+def test_poly_muladd32_against_oracle(d2, log2_n, bits, L, batch):
+    moduli = wl.ntt_primes(bits, 2 << log2_n, L)
+    ctx = d2.Context(log2_n, moduli, 2, seed=1)
+    o = make_oracle(log2_n, moduli, seed=1)
+    a, b, c = (wl.random_polys(moduli, log2_n, batch, seed=s) for s in (4, 5, 6))
+    a[0, :, :4] = np.array(moduli, dtype=np.uint64)[:, None] - 1
+    b[0, :, :2] = np.array(moduli, dtype=np.uint64)[:, None] - 1
+    c[0, :, 0] = np.array(moduli, dtype=np.uint64) - 1
+    da, db, dc = (d2.from_u32_numpy(x.astype(np.uint32), ctx.device) for x in (a, b, c))
+    dd = torch.empty_like(da)
+    ctx.poly_muladd32(da, db, dc, dd, batch)
+    ctx.sync()
+    assert np.array_equal(d2.to_u32_numpy(dd).astype(np.uint64), o.poly_muladd(a, b, c))
+    ctx.close()
+
+
+def test_32_bit_calls_refuse_wide_primes_and_large_rings(d2):
+    wide = d2.Context(12, wl.ntt_primes(36, 1 << 13, 2), 2, seed=1)
+    x = wide.empty_u32(1, 2, 4096)
+    for call in (lambda: wide.ntt32_forward(x, 1), lambda: wide.ntt32_inverse(x, 1),
+                 lambda: wide.poly_muladd32(x, x, x, x, 1)):
+        with pytest.raises(d2.D2mheError) as e:
+            call()
+        assert e.value.status == d2.ERR_UNSUPPORTED
+    wide.close()
+    big = d2.Context(15, wl.ntt_primes(30, 1 << 16, 2), 2, seed=1)
+    y = big.empty_u32(1, 2, 1 << 15)
+    with pytest.raises(d2.D2mheError) as e:
+        big.ntt32_forward(y, 1)
+    assert e.value.status == d2.ERR_UNSUPPORTED
+    big.poly_muladd32(y, y, y, y, 1)  # the multiply-add has no size limit
+    big.sync()
+    big.close()
+
+
 @pytest.mark.parametrize("log2_n", [12, 13, 14, 15, 16])
 def test_sweep_shapes_against_oracle(d2, log2_n):
     """Kernel-sweep shapes: every L of the sweep at this N (60-bit primes), small batch."""

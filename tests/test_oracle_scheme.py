@@ -1,6 +1,6 @@
 """Pins for the oracle's protocol steps against what the paper fixes:
 key form (Sec. 4.2 item 2), ciphertext form and decryption (Sec. 3.2 items 3, 5),
-Convert's correctness derivation (Eq. 3), additivity (Algorithm 2 line 6), the
+Convert's correctness derivation (Eq. 3), additivity (the neighbour-sum step of Algorithm 2), the
 noise condition (Sec. 4.2 discussion), and the rounding as a rational number."""
 import numpy as np
 import pytest
