@@ -27,6 +27,11 @@ struct LimbTab {
   u32 red_shift, red_mul;       // bitlen(q_l) - 1 and floor(2^(bitlen + 15) / q_l): small-quotient reduction
   const ulonglong2* W;          // [N] forward twiddles psi^brv(i) as {w, floor(w 2^64 / q_l)}
   const ulonglong2* IW;         // [N] their inverses
+  // The seven twiddles of octet i in the stride-1 round (last forward, first inverse), regrouped
+  // as seven arrays over i so that the threads of a warp load consecutive entries:
+  // [0][i] = W[N/8 + i], [1 + b][i] = W[N/4 + 2i + b], [3 + r][i] = W[N/2 + 4i + r].
+  const ulonglong2* WL;         // [7][N/8]
+  const ulonglong2* IWL;        // [7][N/8]
 };
 
 // ---------------------------------------------------------------------------
@@ -328,6 +333,52 @@ __device__ __forceinline__ void fwd_octet(u64 (&x)[8], const ulonglong2* __restr
     }
   }
 }
+// The three stages of the stride-1 round on octet i, twiddles from the regrouped table.
+template <int MODE>
+__device__ __forceinline__ void fwd_octet_last(u64 (&x)[8], const ulonglong2* __restrict__ WL, u32 oc,
+                                               u32 i, const Mod& md) {
+  {
+    const ulonglong2 w = __ldg(WL + i);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) ct_bfly<MODE>(x[k], x[k + 4], w, md);
+  }
+  {
+    const ulonglong2 w0 = __ldg(WL + oc + i), w1 = __ldg(WL + 2 * oc + i);
+    ct_bfly<MODE>(x[0], x[2], w0, md);
+    ct_bfly<MODE>(x[1], x[3], w0, md);
+    ct_bfly<MODE>(x[4], x[6], w1, md);
+    ct_bfly<MODE>(x[5], x[7], w1, md);
+  }
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const ulonglong2 w = __ldg(WL + (3 + r) * oc + i);
+    ct_bfly<MODE>(x[2 * r], x[2 * r + 1], w, md);
+  }
+}
+template <int MODE>
+__device__ __forceinline__ void inv_octet_first(u64 (&x)[8], const ulonglong2* __restrict__ IWL, u32 oc,
+                                                u32 i, const Mod& md) {
+  const u64 c16 = md.fourp << 2, c32 = md.fourp << 3, c64 = md.fourp << 4;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const ulonglong2 w = __ldg(IWL + (3 + r) * oc + i);
+    gs_bfly<MODE>(x[2 * r], x[2 * r + 1], w, md, c16);
+  }
+  {
+    const ulonglong2 w0 = __ldg(IWL + oc + i), w1 = __ldg(IWL + 2 * oc + i);
+    gs_bfly<MODE>(x[0], x[2], w0, md, c32);
+    gs_bfly<MODE>(x[1], x[3], w0, md, c32);
+    gs_bfly<MODE>(x[4], x[6], w1, md, c32);
+    gs_bfly<MODE>(x[5], x[7], w1, md, c32);
+  }
+  {
+    const ulonglong2 w = __ldg(IWL + i);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) gs_bfly<MODE>(x[k], x[k + 4], w, md, c64);
+  }
+  if (MODE == MODE_WIDE) x[0] = reduce_small(x[0], md);
+}
+
 // Inverse stages on an octet whose inputs are all below 16p (WIDE) / 4p (otherwise).
 // WIDE bounds after the round: x0 < 128p, x1 < 16p, x2, x3 < 8p, x4..x7 < 4p; x0 is brought
 // back below 4p here, so every output is again below 16p.
@@ -485,7 +536,10 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
         }
-        fwd_octet<WIDE>(x, W, m << soff, (blk << s) + i, 3, md);
+        if (WIDE == MODE_PAIR && last && soff == 0)  // pays only where shared-memory wavefronts bind
+          fwd_octet_last<WIDE>(x, lt.WL, ge.octets, i, md);
+        else
+          fwd_octet<WIDE>(x, W, m << soff, (blk << s) + i, 3, md);
         if (last) {
           emit(g, q, x);
         } else {
@@ -536,7 +590,10 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
         }
-        inv_octet<WIDE>(x, IW, m << soff, (blk << s) + i, 3, md);
+        if (WIDE == MODE_PAIR && from_fetch && soff == 0)
+          inv_octet_first<WIDE>(x, lt.IWL, ge.octets, i, md);
+        else
+          inv_octet<WIDE>(x, IW, m << soff, (blk << s) + i, 3, md);
         if (final_round) {
           finish_octet<WIDE>(x, 3, md);
 #pragma unroll

@@ -263,6 +263,21 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
     if (err != cudaSuccess) return fail_cuda(c, err);
     T.IW = dev_upload(c, IW, &err);
     if (err != cudaSuccess) return fail_cuda(c, err);
+    // stride-1 round: the seven twiddles of every octet, one array per twiddle
+    const u32 oc = n / 8;
+    std::vector<ulonglong2> WL(7 * (size_t)oc), IWL(7 * (size_t)oc);
+    for (u32 i = 0; i < oc; ++i) {
+      const u32 src[7] = {oc + i, 2 * oc + 2 * i, 2 * oc + 2 * i + 1, 4 * oc + 4 * i, 4 * oc + 4 * i + 1,
+                          4 * oc + 4 * i + 2, 4 * oc + 4 * i + 3};
+      for (u32 k = 0; k < 7; ++k) {
+        WL[(size_t)k * oc + i] = W[src[k]];
+        IWL[(size_t)k * oc + i] = IW[src[k]];
+      }
+    }
+    T.WL = dev_upload(c, WL, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    T.IWL = dev_upload(c, IWL, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
   }
   for (u32 l = 0; l < L; ++l) c->limb_params.limbs[l] = limbs[l];
   c->view.limbs = dev_upload(c, limbs, &err);
