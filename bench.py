@@ -501,9 +501,14 @@ def run_sweep(args):
     flush = torch.empty(384 * 1024 * 1024, dtype=torch.uint8, device=dev)
     free_b, _ = torch.cuda.mem_get_info(dev)
     rows = []
+    only = [int(x) for x in args.sweep_point.split(",")] if args.sweep_point else None  # N, L, batch
     for log2_n in wl.SWEEP_LOG2_N:
         n = 1 << log2_n
+        if only and n != only[0]:
+            continue
         for L in wl.SWEEP_LIMBS:
+            if only and L != only[1]:
+                continue
             moduli = wl.sweep_moduli(args.sweep_bits, L)
             ctx = d2mhe.Context(log2_n, moduli, 1, seed=args.seed)
             narrow = args.sweep_bits <= 30
@@ -512,7 +517,7 @@ def run_sweep(args):
             tile = torch.from_numpy(host_tile.astype(np.uint32).view(np.int32) if narrow else host_tile.view(np.int64)).to(dev)
             fwd, inv, mad = ((ctx.ntt32_forward, ctx.ntt32_inverse, ctx.poly_muladd32) if narrow
                              else (ctx.ntt_forward, ctx.ntt_inverse, ctx.poly_muladd))
-            for batch in wl.SWEEP_BATCH:
+            for batch in ([only[2]] if only else wl.SWEEP_BATCH):
                 nbytes = word * n * L * batch
                 row = {"N": n, "L": L, "batch": batch, "GiB": nbytes / 2**30}
                 if nbytes > 0.6 * free_b:
@@ -568,6 +573,7 @@ def main():
     ap.add_argument("--chunk", type=int, default=0, help="ciphertext indices per chunk (0: as many as fit)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep-bits", type=int, default=60, choices=[30, 50, 60])
+    ap.add_argument("--sweep-point", default="", help="N,L,batch: run this one point of the sweep (any batch)")
     args = ap.parse_args()
     if args.config == 5:
         return run_sweep(args)
