@@ -252,6 +252,16 @@ d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* ctx, const uint32_t* a_dev, const ui
  * computes it and returns after all of it has finished.
  */
 size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* ctx, uint32_t chunk_cts);
+/*
+ * Host-only (touches no device): how a whole-round call cuts n_cts ciphertext indices when its
+ * workspace holds cap_cts of them.  Writes the sizes of the first max_out sub-chunks to sizes
+ * (may be NULL) and the number of internal streams used to *lanes_out (may be NULL); returns the
+ * number of sub-chunks, 0 for n_cts == 0 or cap_cts == 0.  Sub-chunk i runs on stream i mod
+ * lanes; sizes differ by at most one, larger ones first; the sizes of the first `lanes`
+ * sub-chunks add up to at most cap_cts.
+ */
+uint32_t d2mhe_round_plan(uint32_t n_cts, uint64_t cap_cts, uint32_t* sizes, uint32_t max_out,
+                          uint32_t* lanes_out);
 d2mhe_status d2mhe_round_device(d2mhe_ctx* ctx, const int32_t* values_dev, uint32_t ct_first,
                                 uint32_t n_cts, const uint32_t* nbr_offsets,
                                 const uint32_t* nbr_rows, int32_t* sums_dev,

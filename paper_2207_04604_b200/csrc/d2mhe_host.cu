@@ -915,6 +915,40 @@ size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* c, u32 chunk_cts) {
   return round_bytes_per_ct(c) * chunk_cts + 256;
 }
 
+// Fewest sub-chunks (a whole number of passes over the lanes, sizes differing by at most one,
+// larger ones first) such that the first pass, which holds the largest ones, fits a workspace
+// for `cap` ciphertext indices and no sub-chunk exceeds `max_sub`.
+struct RoundPlan {
+  u32 lanes, n_sub, sub_small, n_large;  // the first n_large sub-chunks hold sub_small + 1 indices
+};
+static RoundPlan plan_round(u32 n_cts, size_t cap, size_t max_sub) {
+  RoundPlan pl;
+  pl.lanes = (u32)std::min<size_t>(std::min<size_t>(kRoundLanes, cap), n_cts);
+  u32 n_sub = pl.lanes;
+  for (;; n_sub += pl.lanes) {
+    if (n_sub >= n_cts) {
+      n_sub = n_cts;
+      break;
+    }
+    const u32 small = n_cts / n_sub, n_big = n_cts % n_sub;
+    size_t first_pass = 0;
+    for (u32 l = 0; l < pl.lanes; ++l) first_pass += small + (l < n_big ? 1u : 0u);
+    if (first_pass <= cap && small + (n_big ? 1u : 0u) <= max_sub) break;
+  }
+  pl.n_sub = n_sub;
+  pl.sub_small = n_cts / n_sub;
+  pl.n_large = n_cts % n_sub;
+  return pl;
+}
+
+uint32_t d2mhe_round_plan(u32 n_cts, uint64_t cap_cts, u32* sizes, u32 max_out, u32* lanes_out) {
+  if (n_cts == 0 || cap_cts == 0) return 0;
+  const RoundPlan pl = plan_round(n_cts, (size_t)cap_cts, 0x7fffffffu);
+  if (lanes_out) *lanes_out = pl.lanes;
+  for (u32 i = 0; sizes && i < pl.n_sub && i < max_out; ++i) sizes[i] = pl.sub_small + (i < pl.n_large ? 1u : 0u);
+  return pl.n_sub;
+}
+
 // The ciphertext-index range is cut into sub-chunks that are issued in turn on a few
 // internal streams ("lanes"), each with its own part of the workspace: one lane's copies,
 // memory-bound kernels and partial last waves overlap the other lane's arithmetic.  The
@@ -942,22 +976,9 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
   const size_t per_ct = round_bytes_per_ct(c);
   if (ws_bytes < per_ct + 256) return D2MHE_ERR_WORKSPACE;
   const size_t cap = (ws_bytes - 256) / per_ct;  // ciphertext indices the workspace holds
-  const u32 lanes = (u32)std::min<size_t>(std::min<size_t>(kRoundLanes, cap), n_cts);
   const size_t grid_cap = 0x7fffffffull / ((u64)K * std::max(L, 2u));  // launch-grid limit of the kernels
-  // Fewest sub-chunks (a whole number of passes over the lanes, sizes differing by at most one,
-  // larger ones first) such that the first pass, which holds the largest ones, fits the workspace.
-  u32 n_sub = lanes;
-  for (;; n_sub += lanes) {
-    if (n_sub >= n_cts) {
-      n_sub = n_cts;
-      break;
-    }
-    const u32 small = n_cts / n_sub, n_big = n_cts % n_sub;
-    size_t first_pass = 0;
-    for (u32 l = 0; l < lanes; ++l) first_pass += small + (l < n_big ? 1u : 0u);
-    if (first_pass <= cap && small + (n_big ? 1u : 0u) <= grid_cap) break;
-  }
-  const u32 sub_small = n_cts / n_sub, n_large = n_cts % n_sub;  // the first n_large get one more
+  const RoundPlan plan = plan_round(n_cts, cap, grid_cap);
+  const u32 lanes = plan.lanes, n_sub = plan.n_sub, sub_small = plan.sub_small, n_large = plan.n_large;
   size_t lane_first[kRoundLanes + 1] = {};                       // lane l starts this many indices into the workspace
   for (u32 l = 0; l < lanes; ++l) lane_first[l + 1] = lane_first[l] + sub_small + (l < n_large ? 1u : 0u);
 

@@ -28,7 +28,7 @@ EXPORTS = [
     "d2mhe_keygen_share", "d2mhe_collective_pk", "d2mhe_encode", "d2mhe_decode", "d2mhe_encrypt",
     "d2mhe_aggregate", "d2mhe_partial_decrypt", "d2mhe_combine_decrypt", "d2mhe_ntt_forward",
     "d2mhe_ntt_inverse", "d2mhe_poly_muladd", "d2mhe_ntt32_forward", "d2mhe_ntt32_inverse",
-    "d2mhe_poly_muladd32", "d2mhe_round_workspace_bytes", "d2mhe_round_device",
+    "d2mhe_poly_muladd32", "d2mhe_round_workspace_bytes", "d2mhe_round_plan", "d2mhe_round_device",
     "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_user_keygen", "d2mhe_convert_share",
     "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_bootstrap_share", "d2mhe_bootstrap_combine", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_get_root", "d2mhe_get_plain_root",
     "d2mhe_launch_count",
@@ -87,6 +87,11 @@ def load():
         lib.d2mhe_ntt_forward.argtypes = [vp, vp, u32]
         lib.d2mhe_ntt_inverse.argtypes = [vp, vp, u32]
         lib.d2mhe_poly_muladd.argtypes = [vp, vp, vp, vp, vp, u32]
+        lib.d2mhe_ntt32_forward.argtypes = [vp, vp, u32]
+        lib.d2mhe_ntt32_inverse.argtypes = [vp, vp, u32]
+        lib.d2mhe_poly_muladd32.argtypes = [vp, vp, vp, vp, vp, u32]
+        lib.d2mhe_round_plan.argtypes = [u32, ctypes.c_uint64, vp, u32, vp]
+        lib.d2mhe_round_plan.restype = ctypes.c_uint32
         lib.d2mhe_round_workspace_bytes.argtypes = [vp, u32]
         lib.d2mhe_round_workspace_bytes.restype = sz
         lib.d2mhe_round_device.argtypes = [vp, vp, u32, u32, vp, vp, vp, vp, sz]
@@ -110,6 +115,16 @@ def load():
                 fn.restype = ctypes.c_int32
         _lib = lib
     return _lib
+
+
+def round_plan(n_cts, cap_cts):
+    """(sub-chunk sizes, internal streams used) of a whole-round call: d2mhe_round_plan."""
+    lib = load()
+    lanes = ctypes.c_uint32(0)
+    n_sub = int(lib.d2mhe_round_plan(n_cts, cap_cts, None, 0, ctypes.byref(lanes)))
+    sizes = (ctypes.c_uint32 * max(n_sub, 1))()
+    lib.d2mhe_round_plan(n_cts, cap_cts, sizes, n_sub, ctypes.byref(lanes))
+    return [int(x) for x in sizes[:n_sub]], int(lanes.value)
 
 
 def strerror(status):

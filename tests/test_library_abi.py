@@ -59,3 +59,33 @@ def test_create_rejects_bad_arguments_before_touching_the_device():
     p.plain_modulus = 65536
     assert lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h)) == d2mhe.ERR_BAD_PARAMS
     assert not h.value
+
+
+def test_round_plan_invariants():
+    """How a whole-round call cuts its index range (host logic, no device): every index once, sizes
+    within one of each other and non-increasing, whole passes over the streams unless every sub-chunk
+    is a single index, and the sub-chunks in flight at the start (the largest) fit the workspace."""
+    from paper_2207_04604_b200 import d2mhe
+
+    assert d2mhe.round_plan(0, 5) == ([], 0)
+    assert d2mhe.round_plan(5, 0) == ([], 0)
+    for n_cts in list(range(1, 40)) + [66, 683, 1000]:
+        for cap in list(range(1, 12)) + [13, 23, 66, 100, 5000]:
+            sizes, lanes = d2mhe.round_plan(n_cts, cap)
+            assert lanes == min(3, cap, n_cts)
+            assert sum(sizes) == n_cts and min(sizes) >= 1
+            assert max(sizes) - min(sizes) <= 1
+            assert sizes == sorted(sizes, reverse=True)
+            assert len(sizes) % lanes == 0 or len(sizes) == n_cts
+            assert sum(sizes[:lanes]) <= cap
+            # no coarser cut with whole passes would have fitted
+            fewer = len(sizes) - lanes
+            if fewer >= lanes and len(sizes) % lanes == 0:
+                small, big = divmod(n_cts, fewer)
+                first = sum(small + (1 if l < big else 0) for l in range(lanes))
+                assert first > cap
+    # the benchmark configurations: 13 indices in a workspace for 13 -> 5 + 4 + 4 on three streams
+    assert d2mhe.round_plan(13, 13) == ([5, 4, 4], 3)
+    assert d2mhe.round_plan(13, 3) == ([1] * 13, 3)
+    assert d2mhe.round_plan(13, 1) == ([1] * 13, 1)
+    assert d2mhe.round_plan(2, 100) == ([1, 1], 2)
