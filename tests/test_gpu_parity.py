@@ -277,8 +277,9 @@ def test_encode_flags_out_of_range_values(d2):
 # ----------------------------------------------------------------------------------
 
 
-def _run_round(d2, ctx, o, cfg_k, parties, offsets, rows, values, ct_first):
-    """Runs every step on the GPU and on the oracle and compares all messages."""
+def _run_round(d2, ctx, o, cfg_k, parties, offsets, rows, values, ct_first, keep=None):
+    """Runs every step on the GPU and on the oracle and compares all messages
+    (keep, if given, receives the oracle's messages)."""
     n_cts = values.shape[1]
     K = len(parties)
     L, n = o.num_limbs, o.n
@@ -331,6 +332,8 @@ def _run_round(d2, ctx, o, cfg_k, parties, offsets, rows, values, ct_first):
     for i in range(n_out):
         lst = rows[offsets[i]:offsets[i + 1]]
         assert np.array_equal(got[i], values[lst].astype(np.int64).sum(axis=0))
+    if keep is not None:
+        keep.update(ct=want_ct, agg=want_agg, shares=want_shares, sums=got)
     return got
 
 
@@ -377,7 +380,31 @@ def test_config1_every_message(d2, seed):
     o = make_oracle(cfg.log2_n, cfg.moduli, seed=seed)
     offsets, rows = wl.regular_graph(cfg.num_parties, cfg.degree, seed)
     values = wl.gradients(cfg, seed)
-    _run_round(d2, ctx, o, cfg.num_parties, list(range(cfg.num_parties)), offsets, rows, values, 0)
+    want = {}
+    _run_round(d2, ctx, o, cfg.num_parties, list(range(cfg.num_parties)), offsets, rows, values, 0, keep=want)
+    # The same round in the launch configuration the benchmark times: one whole-round call with a
+    # workspace for all 13 indices, i.e. sub-chunks of 5 + 4 + 4 indices on three streams.  Each part
+    # of the workspace is [plain | ciphertexts | aggregates | shares] of its sub-chunk; all of it must
+    # be the oracle's messages.
+    K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, cfg.num_cts
+    assert d2.round_plan(C, C) == ([5, 4, 4], 3)
+    ws = torch.empty(ctx.round_workspace_bytes(C), dtype=torch.uint8, device=ctx.device)
+    sums = torch.zeros((K, C, n), dtype=torch.int32, device=ctx.device)
+    ctx.round_device(torch.from_numpy(values).to(ctx.device), 0, C, offsets, rows, sums, ws)
+    ctx.sync()
+    assert np.array_equal(sums.cpu().numpy(), want["sums"])
+    held = ws.cpu().numpy()
+    per_ct = ctx.round_workspace_bytes(1) - 256
+    first = 0
+    for cc in (5, 4, 4):
+        part = held[first * per_ct:(first + cc) * per_ct]
+        words = part[4 * K * cc * n:].view(np.uint64)
+        n_ct, n_sh = K * cc * 2 * L * n, K * K * cc * L * n
+        sl = slice(first, first + cc)
+        assert np.array_equal(words[:n_ct].reshape(K, cc, 2, L, n), want["ct"][:, sl])
+        assert np.array_equal(words[n_ct:2 * n_ct].reshape(K, cc, 2, L, n), want["agg"][:, sl])
+        assert np.array_equal(words[2 * n_ct:2 * n_ct + n_sh].reshape(K, K, cc, L, n), want["shares"][:, :, sl])
+        first += cc
     ctx.close()
 
 
@@ -440,6 +467,63 @@ def test_large_configs_on_sampled_ciphertext_indices(d2, index, sample):
         for a, i in enumerate(rec):
             lst = rows[offsets[i]:offsets[i + 1]]
             assert np.array_equal(got[a], values[lst].astype(np.int64).sum(axis=0))
+    ctx.close()
+
+
+@pytest.mark.parametrize("index", [3, 4])
+def test_whole_round_at_full_size_in_the_benchmark_configuration(d2, index):
+    """Configurations 3 and 4 at full K, N, L and all C ciphertext indices through one whole-round call,
+    cut as the benchmark cuts it (workspace sized from free memory, sub-chunks on three streams).
+    Every decrypted sum is checked against the plaintext neighbour sum; for the last ciphertext index
+    (the ragged tail), whose sub-chunk is still in the workspace when the call returns, the
+    ciphertexts, aggregates and the shares for three recipients are compared with the oracle."""
+    cfg = wl.round_config(index)
+    seed = 1
+    K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, cfg.num_cts
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, K, seed=seed)
+    dev = ctx.device
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    offsets, rows = wl.regular_graph(K, cfg.degree, seed)
+    # inputs: the workload's gradients on the sampled index, a seeded fill in the clip range elsewhere
+    last = C - 1
+    gen = torch.Generator(device="cpu").manual_seed(seed)
+    values = torch.randint(-cfg.clip, cfg.clip + 1, (K, C, n), dtype=torch.int32, generator=gen)
+    tail = wl.gradients(cfg, seed, ct_first=last, n_cts=1)
+    values[:, last] = torch.from_numpy(tail[:, 0])
+    dv = values.to(dev)
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    per_ct = ctx.round_workspace_bytes(1) - 256
+    cap = int(max(1, min(C, int(free_b * 0.35) // per_ct)))
+    sizes, lanes = d2.round_plan(C, cap)
+    assert lanes == 3 and sum(sizes) == C
+    ws = torch.empty(ctx.round_workspace_bytes(cap), dtype=torch.uint8, device=dev)
+    sums = torch.zeros((K, C, n), dtype=torch.int32, device=dev)
+    ctx.round_device(dv, 0, C, offsets, rows, sums, ws)
+    ctx.sync()
+    for i in range(K):
+        lst = torch.as_tensor(rows[offsets[i]:offsets[i + 1]].astype(np.int64), device=dev)
+        assert torch.equal(sums[i], dv[lst].sum(dim=0, dtype=torch.int32))
+    # where the last sub-chunk lives: stream (len - 1) mod lanes, whose part starts after the first
+    # sub-chunks of the streams before it
+    i_last = len(sizes) - 1
+    lane, cc = i_last % lanes, sizes[i_last]
+    base = sum(sizes[:lane]) * per_ct + 4 * K * cc * n
+    n_ct, n_sh = K * cc * 2 * L * n, K * K * cc * L * n
+    words = ws[base:base + 8 * (2 * n_ct + n_sh)].view(torch.int64)
+    ct = words[:n_ct].view(K, cc, 2, L, n)[:, cc - 1]
+    agg = words[n_ct:2 * n_ct].view(K, cc, 2, L, n)[:, cc - 1]
+    rec = [0, K // 2, K - 1]
+    shares = words[2 * n_ct:].view(K, K, cc, L, n)[rec][:, :, cc - 1]
+    o = make_oracle(cfg.log2_n, cfg.moduli, seed=seed)
+    want_pk = o.collective_pk(parties)
+    want_ct = o.encrypt(want_pk, parties, last, o.encode(tail))
+    assert np.array_equal(d2.to_u64_numpy(ct.contiguous()), want_ct[:, 0])
+    want_agg = o.aggregate(want_ct, offsets, rows)
+    assert np.array_equal(d2.to_u64_numpy(agg.contiguous()), want_agg[:, 0])
+    want_shares = o.partial_decrypt(want_agg[rec], rec, parties, last)
+    assert np.array_equal(d2.to_u64_numpy(shares.contiguous()), want_shares[:, :, 0])
     ctx.close()
 
 
