@@ -25,6 +25,7 @@ struct LimbTab {
   u64 mask;                     // 2^bitlen(q_l) - 1, for the rejection sampler
   u64 rmod, rmod_sh;            // 2^64 mod q_l: leaves Montgomery form; builds Shoup companions
   u32 red_shift, red_mul;       // bitlen(q_l) - 1 and floor(2^(bitlen + 15) / q_l): small-quotient reduction
+  u32 sf_d, sf_shift;           // q_l = 2^b - sf_d with b = 32 + sf_shift (set when b >= 32 and sf_d < 2^32)
   const ulonglong2* W;          // [N] forward twiddles psi^brv(i) as {w, floor(w 2^64 / q_l)}
   const ulonglong2* IW;         // [N] their inverses
   // The seven twiddles of octet i in the stride-1 round (last forward, first inverse), regrouped
@@ -229,15 +230,36 @@ __device__ __forceinline__ u64 shoup_approx(u64 y, u64 w, u64 ws, u64 np) {
   return join64(rl, rh);
 }
 
-// Lazy-reduction policy.  WIDE (every prime below 2^57): values may grow across stages, so
+// The same for a prime of the form p = 2^b - d, b >= 32, d < 2^32 (every "largest prime below 2^b"
+// is): -q p = q d - q 2^b, and q 2^b only reaches the high word as ql << (b - 32), so one of the low
+// multiplies becomes a shift.
+__device__ __forceinline__ u64 shoup_approx_sf(u64 y, u64 w, u64 ws, u32 d, u32 shift) {
+  u32 yl, yh, sl, sh, wl, wh;
+  split64(y, yl, yh);
+  split64(ws, sl, sh);
+  split64(w, wl, wh);
+  u64 q = madwide(yh, sh, join64(mulhi32(yh, sl), 0u));
+  q += (u64)mulhi32(yl, sh);
+  u32 ql, qh, rl, rh;
+  split64(q, ql, qh);
+  split64(madwide(ql, d, mulwide(yl, wl)), rl, rh);
+  rh = madlo(yl, wh, rh);
+  rh = madlo(yh, wl, rh);
+  rh = madlo(qh, d, rh);
+  rh -= ql << shift;
+  return join64(rl, rh);
+}
+
+// Lazy-reduction policy.  WIDE (every prime below 2^57 and of the form above): values may grow across stages, so
 // the forward transform needs no conditional subtraction at all and the inverse reduces only
 // the one element per octet that accumulates the sums.  Otherwise (primes up to 2^61) values
 // are kept below 8p with one conditional subtraction per butterfly.
 struct Mod {
   u64 p, np, twop, fourp;
-  u32 red_shift, red_mul;
+  u32 red_shift, red_mul, sf_d, sf_shift;
   __device__ __forceinline__ explicit Mod(const LimbTab& lt)
-      : p(lt.p), np(lt.np), twop(lt.twop), fourp(2 * lt.twop), red_shift(lt.red_shift), red_mul(lt.red_mul) {}
+      : p(lt.p), np(lt.np), twop(lt.twop), fourp(2 * lt.twop), red_shift(lt.red_shift), red_mul(lt.red_mul),
+        sf_d(lt.sf_d), sf_shift(lt.sf_shift) {}
 };
 
 // x - q p with q = floor(floor(x / 2^(b-1)) * floor(2^(b+15) / p) / 2^16), b = bitlen(p): q is
@@ -291,7 +313,7 @@ __device__ __forceinline__ void ct_bfly(u64& X, u64& Y, const ulonglong2 w, cons
   }
   constexpr bool WIDE = MODE == MODE_WIDE;
   const u64 x = WIDE ? X : csub(X, m.fourp);
-  const u64 t = shoup_approx(Y, w.x, w.y, m.np);  // [0,4p)
+  const u64 t = WIDE ? shoup_approx_sf(Y, w.x, w.y, m.sf_d, m.sf_shift) : shoup_approx(Y, w.x, w.y, m.np);  // [0,4p)
   X = x + t;
   Y = x - t + m.fourp;
 }
@@ -306,7 +328,7 @@ __device__ __forceinline__ void gs_bfly(u64& X, u64& Y, const ulonglong2 w, cons
   const u64 s = X + Y;
   const u64 d = X - Y + (WIDE ? c : m.fourp);
   X = WIDE ? s : csub(s, m.fourp);
-  Y = shoup_approx(d, w.x, w.y, m.np);
+  Y = WIDE ? shoup_approx_sf(d, w.x, w.y, m.sf_d, m.sf_shift) : shoup_approx(d, w.x, w.y, m.np);
 }
 
 // three (or fewer) forward stages on an octet; m = groups at the first stage, i = group index

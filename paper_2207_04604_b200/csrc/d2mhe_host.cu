@@ -215,6 +215,7 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   // floor(q/t) mod q_l: q = Delta t + (q mod t)  =>  Delta = -(q mod t) t^-1 (mod q_l)
   const u64 q_mod_t = q_mod(t);
 
+  bool all_special = true;  // every prime is 2^b - d with b >= 32, d < 2^32
   for (u32 l = 0; l < L; ++l) {
     const u64 p = c->moduli[l];
     LimbTab& T = limbs[l];
@@ -245,6 +246,11 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
     T.mask = bits >= 64 ? ~(u64)0 : (((u64)1 << bits) - 1);
     T.red_shift = bits - 1;
     T.red_mul = (u32)(((u128)1 << (bits + 15)) / p);
+    const u64 gap = bits >= 64 ? 0 : (((u64)1 << bits) - p);  // p = 2^bits - gap
+    const bool special = bits >= 32 && gap < ((u64)1 << 32);
+    T.sf_d = special ? (u32)gap : 0;
+    T.sf_shift = special ? bits - 32 : 0;
+    if (!special) all_special = false;
 
     const u64 psi = c->roots[l], psi_inv = h_inv(psi, p);
     std::vector<u64> pw(n), ipw(n);
@@ -384,7 +390,7 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   c->view.n = n;
   c->view.L = L;
   c->view.K = P.num_parties;
-  c->view.wide = 1;
+  c->view.wide = all_special ? 1 : 0;
   for (u32 l = 0; l < L; ++l)
     if (c->moduli[l] >= ((u64)1 << 57)) c->view.wide = 0;
 

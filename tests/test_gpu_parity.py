@@ -373,6 +373,33 @@ def test_degenerate_and_extreme_parameter_sets(d2, log2_n, bits, L, K, ct_first)
     ctx.close()
 
 
+def _check_whole_round_call(d2, ctx, cfg, offsets, rows, values, want):
+    """The same round in the launch configuration the benchmark times: one whole-round call with a
+    workspace for all C indices (configuration 2: sub-chunks of 5 + 4 + 4 indices on three streams).
+    Each part of the workspace is [plain | ciphertexts | aggregates | shares] of its sub-chunk; all
+    of it must be the oracle's messages (`want`, from the step-by-step comparison)."""
+    K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, cfg.num_cts
+    sizes, lanes = d2.round_plan(C, C)
+    assert len(sizes) == lanes and sum(sizes) == C  # one pass: every sub-chunk is still held afterwards
+    ws = torch.empty(ctx.round_workspace_bytes(C), dtype=torch.uint8, device=ctx.device)
+    sums = torch.zeros((K, C, n), dtype=torch.int32, device=ctx.device)
+    ctx.round_device(torch.from_numpy(values).to(ctx.device), 0, C, offsets, rows, sums, ws)
+    ctx.sync()
+    assert np.array_equal(sums.cpu().numpy(), want["sums"])
+    held = ws.cpu().numpy()
+    per_ct = ctx.round_workspace_bytes(1) - 256
+    first = 0
+    for cc in sizes:
+        part = held[first * per_ct:(first + cc) * per_ct]
+        words = part[4 * K * cc * n:].view(np.uint64)
+        n_ct, n_sh = K * cc * 2 * L * n, K * K * cc * L * n
+        sl = slice(first, first + cc)
+        assert np.array_equal(words[:n_ct].reshape(K, cc, 2, L, n), want["ct"][:, sl])
+        assert np.array_equal(words[n_ct:2 * n_ct].reshape(K, cc, 2, L, n), want["agg"][:, sl])
+        assert np.array_equal(words[2 * n_ct:2 * n_ct + n_sh].reshape(K, K, cc, L, n), want["shares"][:, :, sl])
+        first += cc
+
+
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_config1_every_message(d2, seed):
     cfg = wl.round_config(1)
@@ -382,29 +409,7 @@ def test_config1_every_message(d2, seed):
     values = wl.gradients(cfg, seed)
     want = {}
     _run_round(d2, ctx, o, cfg.num_parties, list(range(cfg.num_parties)), offsets, rows, values, 0, keep=want)
-    # The same round in the launch configuration the benchmark times: one whole-round call with a
-    # workspace for all 13 indices, i.e. sub-chunks of 5 + 4 + 4 indices on three streams.  Each part
-    # of the workspace is [plain | ciphertexts | aggregates | shares] of its sub-chunk; all of it must
-    # be the oracle's messages.
-    K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, cfg.num_cts
-    assert d2.round_plan(C, C) == ([5, 4, 4], 3)
-    ws = torch.empty(ctx.round_workspace_bytes(C), dtype=torch.uint8, device=ctx.device)
-    sums = torch.zeros((K, C, n), dtype=torch.int32, device=ctx.device)
-    ctx.round_device(torch.from_numpy(values).to(ctx.device), 0, C, offsets, rows, sums, ws)
-    ctx.sync()
-    assert np.array_equal(sums.cpu().numpy(), want["sums"])
-    held = ws.cpu().numpy()
-    per_ct = ctx.round_workspace_bytes(1) - 256
-    first = 0
-    for cc in (5, 4, 4):
-        part = held[first * per_ct:(first + cc) * per_ct]
-        words = part[4 * K * cc * n:].view(np.uint64)
-        n_ct, n_sh = K * cc * 2 * L * n, K * K * cc * L * n
-        sl = slice(first, first + cc)
-        assert np.array_equal(words[:n_ct].reshape(K, cc, 2, L, n), want["ct"][:, sl])
-        assert np.array_equal(words[n_ct:2 * n_ct].reshape(K, cc, 2, L, n), want["agg"][:, sl])
-        assert np.array_equal(words[2 * n_ct:2 * n_ct + n_sh].reshape(K, K, cc, L, n), want["shares"][:, :, sl])
-        first += cc
+    _check_whole_round_call(d2, ctx, cfg, offsets, rows, values, want)
     ctx.close()
 
 
@@ -415,7 +420,10 @@ def test_config2_every_message(d2):
     o = make_oracle(cfg.log2_n, cfg.moduli, seed=seed)
     offsets, rows = wl.regular_graph(cfg.num_parties, cfg.degree, seed)
     values = wl.gradients(cfg, seed)
-    _run_round(d2, ctx, o, cfg.num_parties, list(range(cfg.num_parties)), offsets, rows, values, 0)
+    want = {}
+    _run_round(d2, ctx, o, cfg.num_parties, list(range(cfg.num_parties)), offsets, rows, values, 0, keep=want)
+    assert d2.round_plan(cfg.num_cts, cfg.num_cts) == ([5, 4, 4], 3)
+    _check_whole_round_call(d2, ctx, cfg, offsets, rows, values, want)
     ctx.close()
 
 
