@@ -111,9 +111,11 @@ def algorithmic_bytes(cfg, n_cts):
 # multiply-add pipe: 64 lanes per SM per clock (a widening or high-half multiply occupies it
 # for two passes).  Peak = 148 SMs x 64 lanes x 1.965 GHz (the documented SM count and maximum
 # SM clock) = 18.6e12 multiply-add slots per second; a register-only probe of the butterfly
-# reaches 96 % of it.  Algorithmic slots: one lazy Shoup butterfly = 5 widening/high + 4 low
-# multiplies = 14 slots; a transform = (N/2) log2 N butterflies; a pointwise product = 14;
-# one Philox4x32-10 call = 20 widening multiplies = 40 slots (one call serves all L limbs).
+# reaches 96 % of it.  Algorithmic slots: one lazy Shoup butterfly = 5 widening/high + 3 low
+# multiplies = 13 slots (the primes of every configuration are 2^b - d with small d, which turns
+# a fourth low multiply into a shift); a transform = (N/2) log2 N butterflies; a pointwise
+# product = 14; one Philox4x32-10 call = 20 widening multiplies = 40 slots (one call serves all
+# L limbs).
 IMAD_LANES_PER_SM = 64
 NUM_SMS = 148
 SM_MAX_HZ = 1.965e9
@@ -122,7 +124,7 @@ IMAD_PEAK = NUM_SMS * IMAD_LANES_PER_SM * SM_MAX_HZ
 
 def algorithmic_mad_slots(cfg, n_cts):
     K, S, L, n = cfg.num_parties, cfg.num_parties, cfg.num_limbs, cfg.n
-    transform = 14 * (n // 2) * cfg.log2_n   # slots per limb-transform
+    transform = 13 * (n // 2) * cfg.log2_n   # slots per limb-transform
     units = K * n_cts
     return {
         # NTT(u) + 2 inverse transforms, 2 pointwise products, Lambda*m (10 slots) per limb; 3 samples per coefficient
@@ -134,7 +136,7 @@ def algorithmic_mad_slots(cfg, n_cts):
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures under profiles/
 # (null when the kernel has changed since the capture).
-NCU_TRAFFIC_BYTES = {("mnist-mlp-784-128-10-K10", "partial_decrypt"): 44320000 + 303841024}
+NCU_TRAFFIC_BYTES = {("mnist-mlp-784-128-10-K10", "partial_decrypt"): 43577600 + 304694784}
 
 
 # ----------------------------------------------------------------------------------
