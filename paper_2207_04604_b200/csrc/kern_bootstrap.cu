@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
             const u64 dm = shoup_u32(mask[j], lt.delta, lt.delta_sh, lt.np);  // Lambda M_k, below 2p
             // eta_0 = val - dm + e,  eta_1 = -val + dm + e; both sums below 8p
             const u64 s = (comp ? (2 * lt.twop - val) + dm : val + (lt.twop - dm)) + lt.p + (u64)(long long)e[j];
-            out[j] = csub(csub(csub(s, 2 * lt.twop), lt.twop), lt.p);
+            out[j] = canon8<WIDE>(s, lt);
           });
     }
   }

@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
               for (int k = 0; k < 8; ++k) x[k] += mont_lazy(a8[k], b8[k], lt.p, lt.pinv);  // below 4p
             }
           },
-          [&](u32 j, u64 val) { out[j] = add_small_canon(val, (int)e[j], lt); });
+          [&](u32 j, u64 val) { out[j] = add_small_canon<WIDE>(val, (int)e[j], lt); });
     }
   }
   cluster.sync();

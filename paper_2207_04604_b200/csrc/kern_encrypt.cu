@@ -68,9 +68,9 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
           if (comp == 0) {
             // below 4p + (p + 19) + 2p
             u64 t = val + lt.p + (u64)(long long)e[j] + shoup_u32(m[j], lt.delta, lt.delta_sh, lt.np);
-            out[j] = csub(csub(csub(t, 2 * lt.twop), lt.twop), lt.p);
+            out[j] = canon8<WIDE>(t, lt);  // t below 7p + 19
           } else {
-            out[j] = add_small_canon(val, (int)e[j], lt);
+            out[j] = add_small_canon<WIDE>(val, (int)e[j], lt);
           }
         });
   }

@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = mont_lazy(ch[k], x[k], lt.p, lt.pinv);
         },
-        [&](u32 j, u64 val) { out[j] = add_small_canon(val, (int)buf[j], lt); }, 0, 0,
+        [&](u32 j, u64 val) { out[j] = add_small_canon<WIDE>(val, (int)buf[j], lt); }, 0, 0,
         [&]() { cluster.barrier_wait(); });  // every CTA's part of e has landed in every CTA's buffer
   }
   cluster.sync();  // no CTA leaves while a peer may still write into its buffers
