@@ -218,8 +218,7 @@ __device__ __forceinline__ u64 shoup_approx(u64 y, u64 w, u64 ws, u64 np) {
   split64(ws, sl, sh);
   split64(w, wl, wh);
   split64(np, nl, nh);
-  u64 q = madwide(yh, sh, join64(mulhi32(yh, sl), 0u));
-  q += (u64)mulhi32(yl, sh);
+  const u64 q = madwide(yh, sh, (u64)mulhi32(yh, sl) + (u64)mulhi32(yl, sh));
   u32 ql, qh, rl, rh;
   split64(q, ql, qh);
   split64(madwide(ql, nl, mulwide(yl, wl)), rl, rh);
@@ -238,8 +237,9 @@ __device__ __forceinline__ u64 shoup_approx_sf(u64 y, u64 w, u64 ws, u32 d, u32 
   split64(y, yl, yh);
   split64(ws, sl, sh);
   split64(w, wl, wh);
-  u64 q = madwide(yh, sh, join64(mulhi32(yh, sl), 0u));
-  q += (u64)mulhi32(yl, sh);
+  // the two high halves are summed first: the 64-bit sum is a register pair that the widening
+  // multiply-add takes as it is (a zero-extended single word would need a move)
+  const u64 q = madwide(yh, sh, (u64)mulhi32(yh, sl) + (u64)mulhi32(yl, sh));
   u32 ql, qh, rl, rh;
   split64(q, ql, qh);
   split64(madwide(ql, d, mulwide(yl, wl)), rl, rh);
