@@ -58,8 +58,11 @@ __global__ void __launch_bounds__(256)
 //   x = ((q-1)/2 - w') q^-1 mod t  =  round(t v / q) mod t.
 // grid = (n_rec * n_cts, N / 256)
 // ---------------------------------------------------------------------------
+// Up to 8 limbs the kernel is held to 32 registers (a few spilled words) so that 8 CTAs = 2048 threads
+// are resident per SM: the share streams need the loads in flight more than the registers
+// (measured: -13 % at N = 16384, L = 8, 20 shares; -2 % at N = 8192, L = 4, 10 shares).
 template <int LMAX>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, LMAX <= 8 ? 8 : 3)
     k_combine(DevView v, const u64* __restrict__ agg, const u64* __restrict__ shares, u32 n_shares,
               u32 share_comps, u32 n_cts, u32* __restrict__ plain) {
   const u32 unit = blockIdx.x, irec = unit / n_cts, cl = unit % n_cts;
