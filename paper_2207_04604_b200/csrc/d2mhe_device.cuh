@@ -468,6 +468,33 @@ struct NttGeom {
   }
 };
 
+// Thread groups (N = 16384 only: one 1024-thread CTA per SM, where a CTA-wide barrier idles the
+// whole SM).  After its first two stages a forward transform is four independent quarter-size
+// transforms, and an inverse transform is so until its last two stages.  The threads of group h own
+// the octets of the h-th quarter in every round that stays inside the quarters (first stage
+// s >= GB), so those rounds are separated by a named barrier of the group only and the groups drift
+// apart: one group's shared-memory phase overlaps another's arithmetic.  Rounds that span the
+// quarters keep the CTA-wide barrier.  GB = 0 turns this off.
+__host__ __device__ constexpr int ntt_group_bits(int logn, int mode) {
+  return (logn == 14 && mode != MODE_PAIR) ? 2 : 0;
+}
+template <int GB>
+__device__ __forceinline__ u32 group_octet(u32 tid, int g, u32 T, u32 octets) {
+  if (GB == 0) return tid + (u32)g * T;
+  const u32 Tg = T >> GB;
+  return (tid / Tg) * (octets >> GB) + (tid % Tg) + (u32)g * Tg;
+}
+// inside: this round and the next one both stay inside the groups' parts
+template <int GB>
+__device__ __forceinline__ void group_barrier(u32 tid, u32 T, bool inside) {
+  if (GB == 0 || !inside) {
+    __syncthreads();
+  } else {
+    const u32 Tg = T >> GB;  // a multiple of the warp size
+    asm volatile("bar.sync %0, %1;" ::"r"(1u + tid / Tg), "r"(Tg) : "memory");
+  }
+}
+
 // Byte offsets into the swizzled shared-memory polynomial for the eight elements
 // base + (k << sh) of an octet.  The swizzle XORs the low four index bits with bits 4..6;
 // for the strides that occur (sh = 0, 3, 6 and >= 7) most of it is per-octet work, so an
@@ -515,6 +542,7 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
                                             Load load, Emit emit, u32 soff = 0, u32 blk = 0) {
   const NttGeom<LOGN, G> ge(logn_rt);
   const u32 T = ge.T, tid = threadIdx.x;
+  constexpr int GB = ntt_group_bits(LOGN, WIDE);
   const Mod md(lt);
   const ulonglong2* __restrict__ W = lt.W;
   u64 x[8];
@@ -525,7 +553,7 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
     const u32 sh = ge.logn - 3;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const u32 q = tid + g * T;
+      const u32 q = group_octet<GB>(tid, g, T, ge.octets);
       if (LOGN || q < ge.octets) {
         const OctAddr ad(q, sh);
 #pragma unroll
@@ -546,7 +574,7 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
     const bool last = (s + 3 == ge.logn);
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const u32 q = tid + g * T;
+      const u32 q = group_octet<GB>(tid, g, T, ge.octets);
       if (LOGN || q < ge.octets) {
         const u32 i = q >> sh, o = q & ((1u << sh) - 1);
         const u32 base = ((i << 3) << sh) + o;
@@ -571,7 +599,7 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
       }
     }
     from_load = false;
-    if (!last) __syncthreads();
+    if (!last) group_barrier<GB>(tid, T, (int)s >= GB);  // the next round starts at stage s + 3
   }
 }
 
@@ -588,6 +616,7 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
                                             Hook before_final = Hook()) {
   const NttGeom<LOGN, G> ge(logn_rt);
   const u32 T = ge.T, tid = threadIdx.x;
+  constexpr int GB = ntt_group_bits(LOGN, WIDE);
   const Mod md(lt);
   const ulonglong2* __restrict__ IW = lt.IW;
   u64 x[8];
@@ -601,7 +630,7 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
     if (final_round) before_final();
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const u32 q = tid + g * T;
+      const u32 q = group_octet<GB>(tid, g, T, ge.octets);
       if (LOGN || q < ge.octets) {
         const u32 i = q >> sh, o = q & ((1u << sh) - 1);
         const u32 base = ((i << 3) << sh) + o;
@@ -627,14 +656,15 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
       }
     }
     from_fetch = false;
-    if (!final_round) __syncthreads();
+    // the next round starts at stage s - 3, or is the short round that starts at stage 0
+    if (!final_round) group_barrier<GB>(tid, T, s - 3 >= (int)ge.r0 && s - 3 >= GB);
   }
   if (ge.r0) {
     const u32 sh = ge.logn - 3;
     before_final();
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const u32 q = tid + g * T;
+      const u32 q = group_octet<GB>(tid, g, T, ge.octets);
       if (LOGN || q < ge.octets) {
         const OctAddr ad(q, sh);
 #pragma unroll
