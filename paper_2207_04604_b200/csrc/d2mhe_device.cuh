@@ -475,8 +475,14 @@ struct NttGeom {
 // s >= GB), so those rounds are separated by a named barrier of the group only and the groups drift
 // apart: one group's shared-memory phase overlaps another's arithmetic.  Rounds that span the
 // quarters keep the CTA-wide barrier.  GB = 0 turns this off.
+#ifndef D2MHE_GB14
+#define D2MHE_GB14 2
+#endif
+#ifndef D2MHE_GB13
+#define D2MHE_GB13 0
+#endif
 __host__ __device__ constexpr int ntt_group_bits(int logn, int mode) {
-  return (logn == 14 && mode != MODE_PAIR) ? 2 : 0;
+  return mode == MODE_PAIR ? 0 : logn == 14 ? D2MHE_GB14 : logn == 13 ? D2MHE_GB13 : 0;
 }
 template <int GB>
 __device__ __forceinline__ u32 group_octet(u32 tid, int g, u32 T, u32 octets) {
