@@ -126,7 +126,7 @@ namespace d2mhe_launch {
 cudaError_t boot_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
                        const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties,
                        u32 ct_first, u32 n_cts, u64* shares) {
-  D2MHE_DISPATCH_EX(k_boot_share, v, n_rec * n_cts * v.L, s, 6 * (size_t)v.n, cluster_size_for(v.L), v, lp,
+  D2MHE_DISPATCH_EX(k_boot_share, v, n_rec * n_cts * v.L, s, 6 * (size_t)v.n, cluster_size_for(v.L, v.logn), v, lp,
                     agg, recipients_dev, parties_dev, n_parties, ct_first, n_cts, shares);
 }
 

@@ -82,7 +82,7 @@ namespace d2mhe_launch {
 
 cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
                     u32 ct_first, u32 n_cts, const u32* plain, u64* ct) {
-  D2MHE_DISPATCH_EX(k_encrypt, v, n_parties * n_cts * v.L, s, 3 * (size_t)v.n, cluster_size_for(v.L), v, lp,
+  D2MHE_DISPATCH_EX(k_encrypt, v, n_parties * n_cts * v.L, s, 3 * (size_t)v.n, cluster_size_for(v.L, v.logn), v, lp,
                     parties_dev, ct_first, n_cts, plain, ct);
 }
 

@@ -76,7 +76,7 @@ cudaError_t partial_decrypt(const DevView& v, const LimbParams& lp, cudaStream_t
                             const u32* recipients_dev, u32 n_rec, const u32* parties_dev,
                             u32 n_parties, u32 ct_first, u32 n_cts, u64* shares) {
   D2MHE_DISPATCH_EX(k_partial_decrypt, v, n_rec * n_cts * v.L, s, 2 * (size_t)v.n,
-                    cluster_size_for(v.L), v, lp, agg, recipients_dev, parties_dev, n_parties, ct_first,
+                    cluster_size_for(v.L, v.logn), v, lp, agg, recipients_dev, parties_dev, n_parties, ct_first,
                     n_cts, shares);
 }
 
