@@ -134,6 +134,10 @@ d2mhe_status d2mhe_aggregate(d2mhe_ctx* ctx, const uint64_t* ct_dev, uint32_t n_
  * e from chi on the stream (party k, recipient recipients[i], ciphertext index ct_first + c).
  * agg_dev: [n_rec, n_cts, 2, L, N];  shares_dev: out [n_rec, n_parties, n_cts, L, N].
  * recipients, parties: HOST arrays of indices < K.
+ * The noise of the shares is sampled by a kernel of its own into a 64 MiB scratch buffer that the
+ * context owns (one byte per share coefficient; as many (recipient, ciphertext) pairs per launch as
+ * fit), so the call is one or more pairs of launches on the context's stream.
+ * D2MHE_ERR_UNSUPPORTED if n_parties * N exceeds that buffer.
  */
 d2mhe_status d2mhe_partial_decrypt(d2mhe_ctx* ctx, const uint64_t* agg_dev,
                                    const uint32_t* recipients, uint32_t n_rec,
@@ -235,7 +239,8 @@ d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* ctx, const uint32_t* a_dev, const ui
  * of all K parties (Algorithm 2 from encryption to decryption, without the model update): encode,
  * encrypt, neighbour sums, shares from every share holder, combine, decode.  Ciphertext
  * indices are processed in sub-chunks so that all protocol messages of the sub-chunks in
- * flight (ciphertexts, aggregates, shares) live in the caller's workspace.  Up to three
+ * flight (ciphertexts, aggregates, shares, and one noise byte per share coefficient) live in
+ * the caller's workspace.  Up to three
  * sub-chunks are in flight at a time on internal streams, so that one sub-chunk's copies
  * and memory-bound kernels overlap another's arithmetic; the internal streams start after
  * the work already queued on the context's stream, and the context's stream continues

@@ -380,6 +380,9 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   if (err != cudaSuccess) return fail_cuda(c, err);
   c->view.upk_coef = dev_alloc<u64>(c, (size_t)P.num_parties * 2 * poly, &err);
   if (err != cudaSuccess) return fail_cuda(c, err);
+  c->noise_scratch_bytes = kNoiseScratchBytes;
+  c->noise_scratch = dev_alloc<unsigned char>(c, c->noise_scratch_bytes, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
   c->view.range_flag = dev_alloc<u32>(c, 4, &err);
   if (err != cudaSuccess) return fail_cuda(c, err);
   err = cudaMemset(c->view.range_flag, 0, 16);
@@ -612,10 +615,13 @@ d2mhe_status d2mhe_encrypt(d2mhe_ctx* c, const u32* parties, u32 n_parties, u32 
   const u32* arrays[1] = {parties};
   const size_t counts[1] = {n_parties};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
+  // u, e_0, e_1 are sampled ahead into the context's scratch, batch by batch
+  u32 launched = 0;
   cudaError_t e = d2mhe_launch::encrypt(c->view, c->limb_params, c->stream, sg.dev[0], n_parties, ct_first, n_cts,
-                                        plain_dev, reinterpret_cast<u64*>(ct_dev));
+                                        plain_dev, reinterpret_cast<u64*>(ct_dev), c->noise_scratch,
+                                        c->noise_scratch_bytes, &launched);
   if (e != cudaSuccess) return fail_cuda(c, e);
-  c->launches += 1;
+  c->launches += launched;
   return release_slot(c, sg);
 }
 
@@ -666,11 +672,14 @@ d2mhe_status d2mhe_partial_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev, const 
   const u32* arrays[2] = {recipients, parties};
   const size_t counts[2] = {n_rec, n_parties};
   if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::partial_decrypt(
+  // the noise of the shares is sampled ahead into the context's scratch, batch by batch
+  if ((size_t)n_parties * c->view.n > c->noise_scratch_bytes) return D2MHE_ERR_UNSUPPORTED;
+  u32 launched = 0;
+  cudaError_t e = d2mhe_launch::partial_decrypt_scratch(
       c->view, c->limb_params, c->stream, reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1], n_parties,
-      ct_first, n_cts, reinterpret_cast<u64*>(shares_dev));
+      ct_first, n_cts, reinterpret_cast<u64*>(shares_dev), c->noise_scratch, c->noise_scratch_bytes, &launched);
   if (e != cudaSuccess) return fail_cuda(c, e);
-  c->launches += 1;
+  c->launches += launched;
   return release_slot(c, sg);
 }
 
@@ -909,11 +918,16 @@ d2mhe_status d2mhe_bootstrap_combine(d2mhe_ctx* c, const uint64_t* agg_dev, cons
 // ---- whole round ---------------------------------------------------------------------
 
 // Per ciphertext index of a chunk: plain K*N u32, ct and agg K*2*L*N u64 each,
-// shares K*K*L*N u64 (S = K share holders).
+// shares K*K*L*N u64 (S = K share holders), and one byte per sample for what is sampled ahead of the
+// encryption and share kernels (3 K N for the ciphertexts, then K S N for the shares, in the same place).
+static size_t round_noise_bytes_per_ct(const d2mhe_ctx* c) {
+  const size_t K = c->params.num_parties, S = c->pk_parties.empty() ? K : c->pk_parties.size();
+  return (std::max(K * S, 3 * K) * c->view.n + 15) / 16 * 16;  // shares' noise, or [u | e_0 | e_1] per ciphertext
+}
 static size_t round_bytes_per_ct(const d2mhe_ctx* c) {
   const size_t K = c->params.num_parties, S = c->pk_parties.empty() ? K : c->pk_parties.size();
   const size_t n = c->view.n, poly = (size_t)c->view.L * n * sizeof(u64);
-  return K * n * sizeof(u32) + 2 * (K * 2 * poly) + K * S * poly;
+  return K * n * sizeof(u32) + 2 * (K * 2 * poly) + K * S * poly + round_noise_bytes_per_ct(c);
 }
 
 size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* c, u32 chunk_cts) {
@@ -1021,18 +1035,24 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
                           host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s);
     if (e != cudaSuccess) return fail_cuda(c, e);
     if ((e = d2mhe_launch::encode(c->view, s, vals_dev, K * cc, plain)) != cudaSuccess) return fail_cuda(c, e);
-    if ((e = d2mhe_launch::encrypt(c->view, c->limb_params, s, sg.dev[0], K, ct_first + done, cc, plain, ct)) !=
-        cudaSuccess)
+    unsigned char* noise = reinterpret_cast<unsigned char*>(shares + (size_t)K * S * cc * polyw);
+    const size_t noise_bytes = round_noise_bytes_per_ct(c) * cc;  // first u, e_0, e_1, later the shares' noise
+    u32 enc_launches = 0;
+    if ((e = d2mhe_launch::encrypt(c->view, c->limb_params, s, sg.dev[0], K, ct_first + done, cc, plain, ct, noise,
+                                   noise_bytes, &enc_launches)) != cudaSuccess)
       return fail_cuda(c, e);
     if ((e = d2mhe_launch::aggregate(c->view, s, ct, cc, sg.dev[2], sg.dev[3], K, agg)) != cudaSuccess)
       return fail_cuda(c, e);
-    if ((e = d2mhe_launch::partial_decrypt(c->view, c->limb_params, s, agg, sg.dev[0], K, sg.dev[1], S,
-                                           ct_first + done, cc, shares)) != cudaSuccess)
+    u32 pdec_launches = 0;
+    if ((e = d2mhe_launch::partial_decrypt_scratch(c->view, c->limb_params, s, agg, sg.dev[0], K, sg.dev[1], S,
+                                                   ct_first + done, cc, shares, noise, noise_bytes,
+                                                   &pdec_launches)) !=
+        cudaSuccess)
       return fail_cuda(c, e);
     if ((e = d2mhe_launch::combine(c->view, s, agg, shares, K, S, 1, cc, plain)) != cudaSuccess)
       return fail_cuda(c, e);
     if ((e = d2mhe_launch::decode(c->view, s, plain, K * cc, vals_dev)) != cudaSuccess) return fail_cuda(c, e);
-    c->launches += 6;
+    c->launches += 4 + enc_launches + pdec_launches;
     e = cudaMemcpy2DAsync(sums + (size_t)done * n, (size_t)n_cts * n * sizeof(int32_t), vals_dev,
                           (size_t)cc * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
                           host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, s);

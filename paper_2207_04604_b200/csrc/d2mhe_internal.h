@@ -59,6 +59,7 @@ struct DevView {
 
 static const size_t kIdxSlotWords = (size_t)1 << 21;  // u32 words per staging slot (8 MiB)
 static const int kIdxSlots = 4;
+static const size_t kNoiseScratchBytes = (size_t)64 << 20;  // per context, for the single calls
 #ifndef D2MHE_ROUND_LANES
 #define D2MHE_ROUND_LANES 3
 #endif
@@ -90,6 +91,8 @@ struct d2mhe_ctx {
   cudaStream_t lane_stream[kRoundLanes] = {};
   cudaEvent_t lane_event[kRoundLanes] = {};
   cudaEvent_t fork_event = nullptr;
+  unsigned char* noise_scratch = nullptr;  // device: noise bytes of the shares of one d2mhe_partial_decrypt batch
+  size_t noise_scratch_bytes = 0;
   cudaError_t last_cuda = cudaSuccess;
 };
 
@@ -99,13 +102,17 @@ cudaError_t collective_pk(const DevView& v, const LimbParams& lp, cudaStream_t s
                           u64* shares_out);
 cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain);
 cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values);
+// u, e_0, e_1 are sampled ahead into caller-lent scratch (at least 3 N bytes)
 cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
-                    u32 ct_first, u32 n_cts, const u32* plain, u64* ct);
+                    u32 ct_first, u32 n_cts, const u32* plain, u64* ct, void* scratch, size_t scratch_bytes,
+                    u32* launches);
 cudaError_t aggregate(const DevView& v, cudaStream_t s, const u64* ct, u32 n_cts,
                       const u32* offsets_dev, const u32* rows_dev, u32 n_out, u64* agg);
-cudaError_t partial_decrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
-                            const u32* recipients_dev, u32 n_rec, const u32* parties_dev,
-                            u32 n_parties, u32 ct_first, u32 n_cts, u64* shares);
+// decryption shares; their noise is sampled ahead into caller-lent scratch (at least n_parties * N bytes)
+cudaError_t partial_decrypt_scratch(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
+                                    const u32* recipients_dev, u32 n_rec, const u32* parties_dev,
+                                    u32 n_parties, u32 ct_first, u32 n_cts, u64* shares, void* scratch,
+                                    size_t scratch_bytes, u32* launches);
 // shares hold share_comps polynomials per (recipient, party, ciphertext); the first one is summed
 cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
                     u32 n_shares, u32 share_comps, u32 n_cts, u32* plain);

@@ -1,51 +1,56 @@
 // BFV.Encrypt under the collective key: ct = (Lambda m + u p_0 + e_0, u p_1 + e_1).
-#include "d2mhe_kernels_common.cuh"
+#include <algorithm>
 
-namespace cg = cooperative_groups;
+#include "d2mhe_kernels_common.cuh"
 
 namespace {
 
-// grid = n_units * L, launched in thread-block clusters of cs CTAs = cs limbs of the same
-// (party, ciphertext).  u, e_0 and e_1 do not depend on the limb: each CTA samples 1/cs of
-// their coefficients and pushes them (four to a word) into the shared memory of all cs CTAs.
+// u, e_0 and e_1 do not depend on the limb: a kernel of its own samples them once per (party,
+// ciphertext), one byte per coefficient, into scratch memory that the caller of the launcher lends
+// ([u | e_0 | e_1], N bytes each), and the encryption kernel stages them in shared memory.  No
+// thread-block clusters: every CTA is placed freely.
+// grid = ceil(n_units * 3 * N / 4 / 256); one thread = four samples = one packed word.
+__global__ void __launch_bounds__(256)
+    k_sample_encrypt_noise(DevView v, const u32* __restrict__ parties, u32 ct_first, u32 n_cts, u32 unit_first,
+                           u32 n_units, u32* __restrict__ small) {
+  __shared__ GaussTab gt;
+  load_gauss(&gt, v.gauss);
+  const u32 words = v.n >> 2;
+  const size_t total = (size_t)n_units * 3 * words;
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const u32 w = (u32)(e % words), which = (u32)((e / words) % 3), unit = unit_first + (u32)(e / (3 * (size_t)words));
+  const u32 party = parties[unit / n_cts], c = ct_first + unit % n_cts;
+  const Stream st(v.seed, which == 0 ? TAG_ENC_U : which == 1 ? TAG_ENC_E0 : TAG_ENC_E1, c, party, 0);
+  u32 pack = 0;
+  if (which == 0) {
+#pragma unroll
+    for (u32 b = 0; b < 4; ++b) pack |= ((u32)st.ternary(4 * w + b) & 0xffu) << (8 * b);
+  } else {
+#pragma unroll
+    for (u32 b = 0; b < 4; ++b) pack |= ((u32)gauss_from_r(gt, st.draw64(4 * w + b)) & 0xffu) << (8 * b);
+  }
+  small[e] = pack;
+}
+
+// grid = n_units * L; units unit_first .. unit_first + n_units - 1 of the (party, ciphertext) grid.
 // NTT(u) is parked in the output row of c_1 (re-read for both components, overwritten by
 // c_1 at the very end), so no registers are held across the two inverse transforms.
 template <int LOGN, int G, bool WIDE>
 __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
-    k_encrypt(DevView v, const __grid_constant__ LimbParams lp, const u32* __restrict__ parties, u32 ct_first, u32 n_cts,
+    k_encrypt(DevView v, const __grid_constant__ LimbParams lp, u32 unit_first, const u32* __restrict__ sampled,
               const u32* __restrict__ plain, u64* ct) {
-  cg::cluster_group cluster = cg::this_cluster();
-  const u32 cs = cluster.num_blocks(), rank = cluster.block_rank();
-  const u32 l = blockIdx.x % v.L, unit = blockIdx.x / v.L;
-  const u32 party = parties[unit / n_cts], c = ct_first + unit % n_cts;
+  const u32 l = blockIdx.x % v.L, ulocal = blockIdx.x / v.L, unit = unit_first + ulocal;
   const LimbTab& lt = lp.limbs[l];
-  GaussTab* gt = gauss_smem();
-  load_gauss(gt, v.gauss);
   signed char* small = bytes_smem();  // u, e_0, e_1: N bytes each
   u64* sm = poly_smem(3 * v.n);
   const size_t row = (size_t)l * v.n, poly = (size_t)v.L * v.n;
   const u32* m = plain + (size_t)unit * v.n;
   {
-    const Stream su(v.seed, TAG_ENC_U, c, party, 0);
-    const Stream s0(v.seed, TAG_ENC_E0, c, party, 0);
-    const Stream s1(v.seed, TAG_ENC_E1, c, party, 0);
-    for (u32 w = rank + cs * threadIdx.x; w < (v.n >> 2); w += cs * blockDim.x) {
-      u32 pu = 0, p0 = 0, p1 = 0;
-#pragma unroll
-      for (u32 b = 0; b < 4; ++b) {
-        pu |= ((u32)su.ternary(4 * w + b) & 0xffu) << (8 * b);
-        p0 |= ((u32)gauss_from_r(*gt, s0.draw64(4 * w + b)) & 0xffu) << (8 * b);
-        p1 |= ((u32)gauss_from_r(*gt, s1.draw64(4 * w + b)) & 0xffu) << (8 * b);
-      }
-      for (u32 r = 0; r < cs; ++r) {
-        u32* dst = cluster.map_shared_rank(reinterpret_cast<u32*>(small), r);
-        dst[w] = pu;
-        dst[(v.n >> 2) + w] = p0;
-        dst[(v.n >> 1) + w] = p1;
-      }
-    }
+    const u32* src = sampled + (size_t)ulocal * 3 * (v.n >> 2);
+    for (u32 w = threadIdx.x; w < 3 * (v.n >> 2); w += blockDim.x) reinterpret_cast<u32*>(small)[w] = __ldg(src + w);
   }
-  cluster.sync();  // all samples have landed everywhere; nothing is pushed after this point
+  // the barrier that opens the forward transform publishes the copy
   u64* park = ct + ((size_t)unit * 2 + 1) * poly + row;
   ntt_forward<LOGN, G, WIDE>(
       sm, lt, v.logn, [&](u32 j) { return lift_small((int)small[j], lt.p); },
@@ -80,10 +85,32 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 
 namespace d2mhe_launch {
 
+static cudaError_t encrypt_units(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 unit_first, u32 n_units,
+                                 const u32* sampled, const u32* plain, u64* ct) {
+  D2MHE_DISPATCH_EX(k_encrypt, v, n_units * v.L, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain, ct);
+}
+
+// scratch: at least 3 N bytes; (party, ciphertext) units are processed in batches of as many as it holds.
 cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
-                    u32 ct_first, u32 n_cts, const u32* plain, u64* ct) {
-  D2MHE_DISPATCH_EX(k_encrypt, v, n_parties * n_cts * v.L, s, 3 * (size_t)v.n, cluster_size_for(v.L, v.logn), v, lp,
-                    parties_dev, ct_first, n_cts, plain, ct);
+                    u32 ct_first, u32 n_cts, const u32* plain, u64* ct, void* scratch, size_t scratch_bytes,
+                    u32* launches) {
+  const size_t per_unit = 3 * (size_t)v.n;
+  const u32 n_units = n_parties * n_cts;
+  const u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
+  if (launches) *launches = 0;
+  if (per_batch == 0) return cudaErrorInvalidValue;
+  for (u32 first = 0; first < n_units; first += per_batch) {
+    const u32 nu = std::min(per_batch, n_units - first);
+    const size_t words = (size_t)nu * per_unit / 4;
+    k_sample_encrypt_noise<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(v, parties_dev, ct_first, n_cts, first, nu,
+                                                                          reinterpret_cast<u32*>(scratch));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    e = encrypt_units(v, lp, s, first, nu, reinterpret_cast<const u32*>(scratch), plain, ct);
+    if (e != cudaSuccess) return e;
+    if (launches) *launches += 2;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace d2mhe_launch

@@ -1,34 +1,49 @@
 // Decryption shares: h = s_k c_1 + e for every listed share holder.
-#include "d2mhe_kernels_common.cuh"
+#include <algorithm>
 
-namespace cg = cooperative_groups;
+#include "d2mhe_kernels_common.cuh"
 
 namespace {
 
-// grid = n_rec * n_cts * L, launched in thread-block clusters of cs CTAs = cs limbs of the same
-// (recipient, ciphertext).  The noise polynomial e of a share is the same for every limb, so
-// each CTA of the cluster samples 1/cs of its coefficients (Philox + table inversion) and
-// pushes them, four to a word, into the shared memory of all cs CTAs (distributed shared
-// memory); two noise buffers alternate so that one cluster barrier per share suffices, and
-// that barrier is split: arrive after the push, wait just before the last inverse round.
-// NTT(c_1) is computed once per CTA and parked in the output row of the LAST share
-// (L2-resident, re-read for every share, overwritten by that share at the very end), so no
-// registers are held across the party loop.  Each share costs one pointwise product, one
-// inverse transform and one store.
+// The noise polynomial e of a share does not depend on the limb.  It is sampled once per share by a
+// kernel of its own (Philox + table inversion, one byte per coefficient, into scratch memory that
+// the caller of the launcher lends), so the share kernel needs no thread-block clusters: every CTA
+// is placed freely and spends its time on the transforms.  (A variant that sampled inside the share
+// kernel and spread the samples over a cluster of the limbs' CTAs was 3 % slower at N = 8192 and
+// 8 % at N = 16384, where clusters of one-CTA-per-SM blocks also leave SMs idle.)
+//
+// grid = ceil(n_units * n_parties * N / 4 / 256); one thread = four samples = one packed word.
+// noise[(u * n_parties + a) * N + j], u = unit - unit_first, unit = irec * n_cts + cl.
+__global__ void __launch_bounds__(256)
+    k_sample_share_noise(DevView v, const u32* __restrict__ recipients, const u32* __restrict__ parties,
+                         u32 n_parties, u32 ct_first, u32 n_cts, u32 unit_first, u32 n_units,
+                         u32* __restrict__ noise) {
+  __shared__ GaussTab gt;
+  load_gauss(&gt, v.gauss);
+  const u32 words = v.n >> 2;
+  const size_t total = (size_t)n_units * n_parties * words;
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const u32 w = (u32)(e % words);
+  const size_t share = e / words;
+  const u32 a = (u32)(share % n_parties), unit = unit_first + (u32)(share / n_parties);
+  const Stream se(v.seed, TAG_DEC_ERR, ct_first + unit % n_cts, parties[a], recipients[unit / n_cts]);
+  u32 pack = 0;
+#pragma unroll
+  for (u32 b = 0; b < 4; ++b) pack |= ((u32)gauss_from_r(gt, se.draw64(4 * w + b)) & 0xffu) << (8 * b);
+  noise[e] = pack;
+}
+
+// grid = n_units * L; units unit_first .. unit_first + n_units - 1 of the (recipient, ciphertext) grid.
 template <int LOGN, int G, bool WIDE>
 __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
-    k_partial_decrypt(DevView v, const __grid_constant__ LimbParams lp, const u64* __restrict__ agg, const u32* __restrict__ recipients,
-                      const u32* __restrict__ parties, u32 n_parties, u32 ct_first, u32 n_cts,
-                      u64* shares) {
-  cg::cluster_group cluster = cg::this_cluster();
-  const u32 cs = cluster.num_blocks(), rank = cluster.block_rank();
-  const u32 l = blockIdx.x % v.L, unit = blockIdx.x / v.L;
-  const u32 irec = unit / n_cts, cl = unit % n_cts, c = ct_first + cl;
-  const u32 recipient = recipients[irec];
+    k_partial_decrypt_pre(DevView v, const __grid_constant__ LimbParams lp, const u64* __restrict__ agg,
+                          const u32* __restrict__ parties, u32 n_parties, u32 n_cts, u32 unit_first,
+                          const signed char* __restrict__ noise, u64* shares) {
+  const u32 l = blockIdx.x % v.L, ulocal = blockIdx.x / v.L, unit = unit_first + ulocal;
+  const u32 irec = unit / n_cts, cl = unit % n_cts;
   const LimbTab& lt = lp.limbs[l];
-  GaussTab* gt = gauss_smem();
-  load_gauss(gt, v.gauss);
-  signed char* noise = bytes_smem();  // two buffers of N bytes
+  signed char* staged = bytes_smem();  // two buffers of N bytes: the noise of this share and of the next
   u64* sm = poly_smem(2 * v.n);
   const size_t row = (size_t)l * v.n, poly = (size_t)v.L * v.n;
   const u64* c1 = agg + ((size_t)unit * 2 + 1) * poly + row;
@@ -38,20 +53,15 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
       [&](int, u32 q, u64(&x)[8]) { store_octet(park + 8 * (size_t)q, x); });
 #pragma unroll 1
   for (u32 a = 0; a < n_parties; ++a) {
-    const u32 party = parties[a];
-    signed char* buf = noise + (a & 1u) * v.n;
+    const u64* sk = v.s_mont + ((size_t)parties[a] * v.L + l) * v.n;
+    // Buffer a & 1 was last read in the final round of share a - 2, which every thread left before
+    // it passed the barrier that opens the transform of share a - 1; the barrier that opens this
+    // share's transform publishes the copy.
+    signed char* e = staged + (a & 1u) * v.n;
     {
-      const Stream se(v.seed, TAG_DEC_ERR, c, party, recipient);
-      for (u32 w = rank + cs * threadIdx.x; w < (v.n >> 2); w += cs * blockDim.x) {
-        u32 pack = 0;
-#pragma unroll
-        for (u32 b = 0; b < 4; ++b)
-          pack |= ((u32)gauss_from_r(*gt, se.draw64(4 * w + b)) & 0xffu) << (8 * b);
-        for (u32 r = 0; r < cs; ++r) cluster.map_shared_rank(reinterpret_cast<u32*>(buf), r)[w] = pack;
-      }
+      const u32* src = reinterpret_cast<const u32*>(noise + ((size_t)ulocal * n_parties + a) * v.n);
+      for (u32 w = threadIdx.x; w < (v.n >> 2); w += blockDim.x) reinterpret_cast<u32*>(e)[w] = __ldg(src + w);
     }
-    cluster.barrier_arrive();  // waited for just before the last round, the only reader of the noise
-    const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
     u64* out = shares + (((size_t)irec * n_parties + a) * n_cts + cl) * poly + row;
     ntt_inverse<LOGN, G, WIDE>(
         sm, lt, v.logn,
@@ -62,22 +72,46 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = mont_lazy(ch[k], x[k], lt.p, lt.pinv);
         },
-        [&](u32 j, u64 val) { out[j] = add_small_canon<WIDE>(val, (int)buf[j], lt); }, 0, 0,
-        [&]() { cluster.barrier_wait(); });  // every CTA's part of e has landed in every CTA's buffer
+        [&](u32 j, u64 val) { out[j] = add_small_canon<WIDE>(val, (int)e[j], lt); });
   }
-  cluster.sync();  // no CTA leaves while a peer may still write into its buffers
 }
 
 }  // namespace
 
 namespace d2mhe_launch {
 
-cudaError_t partial_decrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
-                            const u32* recipients_dev, u32 n_rec, const u32* parties_dev,
-                            u32 n_parties, u32 ct_first, u32 n_cts, u64* shares) {
-  D2MHE_DISPATCH_EX(k_partial_decrypt, v, n_rec * n_cts * v.L, s, 2 * (size_t)v.n,
-                    cluster_size_for(v.L, v.logn), v, lp, agg, recipients_dev, parties_dev, n_parties, ct_first,
-                    n_cts, shares);
+static cudaError_t pdec_pre_units(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
+                                  const u32* parties_dev, u32 n_parties, u32 n_cts, u32 unit_first,
+                                  u32 n_units, const signed char* noise, u64* shares) {
+  D2MHE_DISPATCH_EX(k_partial_decrypt_pre, v, n_units * v.L, s, 2 * (size_t)v.n, 1, v, lp, agg, parties_dev, n_parties,
+                    n_cts, unit_first, noise, shares);
+}
+
+// Shares with the noise sampled ahead into `scratch` (scratch_bytes >= n_parties * N), in batches of
+// as many (recipient, ciphertext) units as the scratch holds.  *launches receives the number of
+// kernel launches.
+cudaError_t partial_decrypt_scratch(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
+                                    const u32* recipients_dev, u32 n_rec, const u32* parties_dev,
+                                    u32 n_parties, u32 ct_first, u32 n_cts, u64* shares, void* scratch,
+                                    size_t scratch_bytes, u32* launches) {
+  const size_t per_unit = (size_t)n_parties * v.n;
+  const u32 n_units = n_rec * n_cts;
+  const u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
+  if (launches) *launches = 0;
+  if (per_batch == 0) return cudaErrorInvalidValue;
+  for (u32 first = 0; first < n_units; first += per_batch) {
+    const u32 nu = std::min(per_batch, n_units - first);
+    const size_t words = (size_t)nu * per_unit / 4;
+    k_sample_share_noise<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(
+        v, recipients_dev, parties_dev, n_parties, ct_first, n_cts, first, nu, reinterpret_cast<u32*>(scratch));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    e = pdec_pre_units(v, lp, s, agg, parties_dev, n_parties, n_cts, first, nu,
+                       reinterpret_cast<const signed char*>(scratch), shares);
+    if (e != cudaSuccess) return e;
+    if (launches) *launches += 2;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace d2mhe_launch

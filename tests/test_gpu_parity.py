@@ -738,7 +738,7 @@ def test_round_driver_matches_stepwise_and_plain_sums(d2):
         assert np.array_equal(sums.cpu().numpy(), want)
     # The messages themselves, not only the sums: a workspace for three indices makes thirteen
     # one-index sub-chunks that rotate over three parts of it, so that at the end the parts hold
-    # indices 12, 10 and 11, each as [plain | ciphertexts | aggregates | shares].  They must be
+    # indices 12, 10 and 11, each as [plain | ciphertexts | aggregates | shares | noise bytes].  They must be
     # the messages the step-by-step calls produce for those indices.
     L = cfg.num_limbs
     ws = torch.empty(ctx.round_workspace_bytes(3), dtype=torch.uint8, device=ctx.device)
@@ -748,7 +748,7 @@ def test_round_driver_matches_stepwise_and_plain_sums(d2):
     assert np.array_equal(sums.cpu().numpy(), want)
     per_ct = ctx.round_workspace_bytes(1) - 256
     ct_words, share_words = K * 2 * L * n, K * K * L * n
-    assert per_ct == 4 * K * n + 8 * (2 * ct_words + share_words)
+    assert per_ct == 4 * K * n + 8 * (2 * ct_words + share_words) + max(K * K, 3 * K) * n  # the last term: one byte per sample drawn ahead of a kernel
     held = ws.cpu().numpy()
     for part, index in enumerate((12, 10, 11)):
         plain = ctx.empty_u32(K, 1, n)
@@ -763,7 +763,7 @@ def test_round_driver_matches_stepwise_and_plain_sums(d2):
         words = held[part * per_ct + 4 * K * n:(part + 1) * per_ct].view(np.uint64)
         assert np.array_equal(words[:ct_words], d2.to_u64_numpy(ct).ravel())
         assert np.array_equal(words[ct_words:2 * ct_words], d2.to_u64_numpy(agg).ravel())
-        assert np.array_equal(words[2 * ct_words:], d2.to_u64_numpy(shares).ravel())
+        assert np.array_equal(words[2 * ct_words:2 * ct_words + share_words], d2.to_u64_numpy(shares).ravel())
     # host variant, pinned buffers
     hv = torch.from_numpy(values).pin_memory()
     hs = torch.zeros((K, C, n), dtype=torch.int32).pin_memory()
