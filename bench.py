@@ -136,7 +136,7 @@ def algorithmic_mad_slots(cfg, n_cts):
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures under profiles/
 # (null when the kernel has changed since the capture).
-NCU_TRAFFIC_BYTES = {("mnist-mlp-784-128-10-K10", "partial_decrypt"): 43931136 + 303016448}
+NCU_TRAFFIC_BYTES = {("mnist-mlp-784-128-10-K10", "partial_decrypt"): 56150272 + 304640000}
 
 
 # ----------------------------------------------------------------------------------
@@ -444,6 +444,8 @@ def run_cuda(args, cfg):
                         "unit": "T int32 multiply-add slots/s", "frac": got / IMAD_PEAK,
                         "peak_source": "148 SMs x 64 lanes x 1.965 GHz (unit counts and clocks)",
                         "traffic": traffic, "avg_launch_ms": dur_ms,
+                        "launches_note": "one call = the sampling kernel (about 5 % of the time) followed by the "
+                                         "transform kernel; traffic is the transform kernel's",
                         "hbm": {"achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                                 "peak_source": "of " + peak_kind}}
         else:
