@@ -124,11 +124,13 @@ inline u32 ntt_threads(u32 n, int g) {
   return t < 32 ? 32 : t;
 }
 
-// Largest divisor of L that is a portable thread-block-cluster size, at most `cap`.  At N = 16384 a
-// CTA fills an SM, a cluster must sit inside one GPC, and clusters of 8 leave the SMs of every GPC
-// beyond a multiple of 8 idle (120 of 148 SMs busy in the share kernel).  Measured there (L = 8):
-// clusters of 2 beat 4, 8 and 1 although each CTA then samples half of the noise itself; at
-// N = 8192 (two CTAs per SM, L = 4) clusters of 4 beat 2 and 1.
+// Largest divisor of L that is a portable thread-block-cluster size, at most `cap` (the conversion
+// and bootstrap share kernels sample their noise inside the kernel, each CTA of a cluster a part of
+// it).  At N = 16384 a CTA fills an SM, a cluster must sit inside one GPC, and clusters of 8 leave the
+// SMs of every GPC beyond a multiple of 8 idle (120 of 148 SMs were busy when the decryption-share
+// kernel still ran that way).  Measured there (L = 8): clusters of 2 beat 4, 8 and 1 although each
+// CTA then samples half of the noise itself; at N = 8192 (two CTAs per SM, L = 4) clusters of 4 beat
+// 2 and 1.
 #ifndef D2MHE_CS_CAP14
 #define D2MHE_CS_CAP14 2
 #endif
