@@ -462,7 +462,7 @@ def run_cuda(args, cfg):
             "vs_baseline": None, "dtype": "u64", "data": "synthetic",
             "config": {"workload": cfg.name, "K": K, "N": n, "L": L, "cts_per_user": C, "params_per_user": cfg.params,
                        "graph_degree": cfg.degree, "share_holders": K, "chunk_cts": chunk,
-                       "entry_point": "d2mhe_round_device (sub-chunks overlapped on three internal streams)",
+                       "entry_point": "d2mhe_round_device (sub-chunks overlapped on two internal streams)",
                        "l2": "384 MB buffer written between timed steps (L2 flush)",
                        "parallelism": "ciphertext-index shards, no exchange" if world > 1 else "single GPU"},
             "clocks": clocks,

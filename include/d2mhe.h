@@ -240,8 +240,8 @@ d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* ctx, const uint32_t* a_dev, const ui
  * encrypt, neighbour sums, shares from every share holder, combine, decode.  Ciphertext
  * indices are processed in sub-chunks so that all protocol messages of the sub-chunks in
  * flight (ciphertexts, aggregates, shares, and one noise byte per share coefficient) live in
- * the caller's workspace.  Up to three
- * sub-chunks are in flight at a time on internal streams, so that one sub-chunk's copies
+ * the caller's workspace.  Up to two sub-chunks (three for d2mhe_round_host) are in flight
+ * at a time on internal streams, so that one sub-chunk's copies
  * and memory-bound kernels overlap another's arithmetic; the internal streams start after
  * the work already queued on the context's stream, and the context's stream continues
  * after they have finished (so the call behaves like one operation on that stream).
@@ -258,12 +258,13 @@ d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* ctx, const uint32_t* a_dev, const ui
  */
 size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* ctx, uint32_t chunk_cts);
 /*
- * Host-only (touches no device): how a whole-round call cuts n_cts ciphertext indices when its
+ * Host-only (touches no device): how d2mhe_round_device cuts n_cts ciphertext indices when its
  * workspace holds cap_cts of them.  Writes the sizes of the first max_out sub-chunks to sizes
  * (may be NULL) and the number of internal streams used to *lanes_out (may be NULL); returns the
  * number of sub-chunks, 0 for n_cts == 0 or cap_cts == 0.  Sub-chunk i runs on stream i mod
  * lanes; sizes differ by at most one, larger ones first; the sizes of the first `lanes`
- * sub-chunks add up to at most cap_cts.
+ * sub-chunks add up to at most cap_cts.  (d2mhe_round_host cuts by the same rule over three
+ * streams.)
  */
 uint32_t d2mhe_round_plan(uint32_t n_cts, uint64_t cap_cts, uint32_t* sizes, uint32_t max_out,
                           uint32_t* lanes_out);

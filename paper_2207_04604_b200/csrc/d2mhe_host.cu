@@ -941,9 +941,9 @@ size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* c, u32 chunk_cts) {
 struct RoundPlan {
   u32 lanes, n_sub, sub_small, n_large;  // the first n_large sub-chunks hold sub_small + 1 indices
 };
-static RoundPlan plan_round(u32 n_cts, size_t cap, size_t max_sub) {
+static RoundPlan plan_round(u32 n_cts, size_t cap, size_t max_sub, int max_lanes) {
   RoundPlan pl;
-  pl.lanes = (u32)std::min<size_t>(std::min<size_t>(kRoundLanes, cap), n_cts);
+  pl.lanes = (u32)std::min<size_t>(std::min<size_t>(max_lanes, cap), n_cts);
   u32 n_sub = pl.lanes;
   for (;; n_sub += pl.lanes) {
     if (n_sub >= n_cts) {
@@ -963,7 +963,7 @@ static RoundPlan plan_round(u32 n_cts, size_t cap, size_t max_sub) {
 
 uint32_t d2mhe_round_plan(u32 n_cts, uint64_t cap_cts, u32* sizes, u32 max_out, u32* lanes_out) {
   if (n_cts == 0 || cap_cts == 0) return 0;
-  const RoundPlan pl = plan_round(n_cts, (size_t)cap_cts, 0x7fffffffu);
+  const RoundPlan pl = plan_round(n_cts, (size_t)cap_cts, 0x7fffffffu, kRoundLanesDevice);
   if (lanes_out) *lanes_out = pl.lanes;
   for (u32 i = 0; sizes && i < pl.n_sub && i < max_out; ++i) sizes[i] = pl.sub_small + (i < pl.n_large ? 1u : 0u);
   return pl.n_sub;
@@ -997,7 +997,7 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
   if (ws_bytes < per_ct + 256) return D2MHE_ERR_WORKSPACE;
   const size_t cap = (ws_bytes - 256) / per_ct;  // ciphertext indices the workspace holds
   const size_t grid_cap = 0x7fffffffull / ((u64)K * std::max(L, 2u));  // launch-grid limit of the kernels
-  const RoundPlan plan = plan_round(n_cts, cap, grid_cap);
+  const RoundPlan plan = plan_round(n_cts, cap, grid_cap, host_io ? kRoundLanesHost : kRoundLanesDevice);
   const u32 lanes = plan.lanes, n_sub = plan.n_sub, sub_small = plan.sub_small, n_large = plan.n_large;
   size_t lane_first[kRoundLanes + 1] = {};                       // lane l starts this many indices into the workspace
   for (u32 l = 0; l < lanes; ++l) lane_first[l + 1] = lane_first[l] + sub_small + (l < n_large ? 1u : 0u);

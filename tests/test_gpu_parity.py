@@ -375,7 +375,7 @@ def test_degenerate_and_extreme_parameter_sets(d2, log2_n, bits, L, K, ct_first)
 
 def _check_whole_round_call(d2, ctx, cfg, offsets, rows, values, want):
     """The same round in the launch configuration the benchmark times: one whole-round call with a
-    workspace for all C indices (configuration 2: sub-chunks of 5 + 4 + 4 indices on three streams).
+    workspace for all C indices (configuration 2: sub-chunks of 7 + 6 indices on two streams).
     Each part of the workspace is [plain | ciphertexts | aggregates | shares] of its sub-chunk; all
     of it must be the oracle's messages (`want`, from the step-by-step comparison)."""
     K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, cfg.num_cts
@@ -422,7 +422,7 @@ def test_config2_every_message(d2):
     values = wl.gradients(cfg, seed)
     want = {}
     _run_round(d2, ctx, o, cfg.num_parties, list(range(cfg.num_parties)), offsets, rows, values, 0, keep=want)
-    assert d2.round_plan(cfg.num_cts, cfg.num_cts) == ([5, 4, 4], 3)
+    assert d2.round_plan(cfg.num_cts, cfg.num_cts) == ([7, 6], 2)
     _check_whole_round_call(d2, ctx, cfg, offsets, rows, values, want)
     ctx.close()
 
@@ -481,7 +481,7 @@ def test_large_configs_on_sampled_ciphertext_indices(d2, index, sample):
 @pytest.mark.parametrize("index", [3, 4])
 def test_whole_round_at_full_size_in_the_benchmark_configuration(d2, index):
     """Configurations 3 and 4 at full K, N, L and all C ciphertext indices through one whole-round call,
-    cut as the benchmark cuts it (workspace sized from free memory, sub-chunks on three streams).
+    cut as the benchmark cuts it (workspace sized from free memory, sub-chunks on two streams).
     Every decrypted sum is checked against the plaintext neighbour sum; for the last ciphertext index
     (the ragged tail), whose sub-chunk is still in the workspace when the call returns, the
     ciphertexts, aggregates and the shares for three recipients are compared with the oracle."""
@@ -505,7 +505,7 @@ def test_whole_round_at_full_size_in_the_benchmark_configuration(d2, index):
     per_ct = ctx.round_workspace_bytes(1) - 256
     cap = int(max(1, min(C, int(free_b * 0.35) // per_ct)))
     sizes, lanes = d2.round_plan(C, cap)
-    assert lanes == 3 and sum(sizes) == C
+    assert lanes == 2 and sum(sizes) == C
     ws = torch.empty(ctx.round_workspace_bytes(cap), dtype=torch.uint8, device=dev)
     sums = torch.zeros((K, C, n), dtype=torch.int32, device=dev)
     ctx.round_device(dv, 0, C, offsets, rows, sums, ws)
@@ -736,10 +736,11 @@ def test_round_driver_matches_stepwise_and_plain_sums(d2):
         ctx.round_device(dv, 0, C, offsets, rows, sums, ws)
         ctx.sync()
         assert np.array_equal(sums.cpu().numpy(), want)
-    # The messages themselves, not only the sums: a workspace for three indices makes thirteen
-    # one-index sub-chunks that rotate over three parts of it, so that at the end the parts hold
-    # indices 12, 10 and 11, each as [plain | ciphertexts | aggregates | shares | noise bytes].  They must be
-    # the messages the step-by-step calls produce for those indices.
+    # The messages themselves, not only the sums: a workspace for three indices makes twelve
+    # sub-chunks (2, 1, 1, ... indices) that alternate over two parts of it, the first two indices
+    # wide, so that at the end the parts hold indices 11 (at offset 0) and 12 (at offset two), each as
+    # [plain | ciphertexts | aggregates | shares | noise bytes].  They must be the messages the
+    # step-by-step calls produce for those indices.
     L = cfg.num_limbs
     ws = torch.empty(ctx.round_workspace_bytes(3), dtype=torch.uint8, device=ctx.device)
     sums = torch.zeros((K, C, n), dtype=torch.int32, device=ctx.device)
@@ -750,7 +751,8 @@ def test_round_driver_matches_stepwise_and_plain_sums(d2):
     ct_words, share_words = K * 2 * L * n, K * K * L * n
     assert per_ct == 4 * K * n + 8 * (2 * ct_words + share_words) + max(K * K, 3 * K) * n  # the last term: one byte per sample drawn ahead of a kernel
     held = ws.cpu().numpy()
-    for part, index in enumerate((12, 10, 11)):
+    assert d2.round_plan(C, 3) == ([2] + [1] * 11, 2)
+    for part, index in ((0, 11), (2, 12)):
         plain = ctx.empty_u32(K, 1, n)
         ct = ctx.empty_u64(K, 1, 2, L, n)
         agg = ctx.empty_u64(K, 1, 2, L, n)

@@ -72,7 +72,7 @@ def test_round_plan_invariants():
     for n_cts in list(range(1, 40)) + [66, 683, 1000]:
         for cap in list(range(1, 12)) + [13, 23, 66, 100, 5000]:
             sizes, lanes = d2mhe.round_plan(n_cts, cap)
-            assert lanes == min(3, cap, n_cts)
+            assert lanes == min(2, cap, n_cts)
             assert sum(sizes) == n_cts and min(sizes) >= 1
             assert max(sizes) - min(sizes) <= 1
             assert sizes == sorted(sizes, reverse=True)
@@ -84,8 +84,8 @@ def test_round_plan_invariants():
                 small, big = divmod(n_cts, fewer)
                 first = sum(small + (1 if l < big else 0) for l in range(lanes))
                 assert first > cap
-    # the benchmark configurations: 13 indices in a workspace for 13 -> 5 + 4 + 4 on three streams
-    assert d2mhe.round_plan(13, 13) == ([5, 4, 4], 3)
-    assert d2mhe.round_plan(13, 3) == ([1] * 13, 3)
+    # the benchmark configurations: 13 indices in a workspace for 13 -> 7 + 6 on two streams
+    assert d2mhe.round_plan(13, 13) == ([7, 6], 2)
+    assert d2mhe.round_plan(13, 3) == ([2] + [1] * 11, 2)
     assert d2mhe.round_plan(13, 1) == ([1] * 13, 1)
     assert d2mhe.round_plan(2, 100) == ([1, 1], 2)
