@@ -63,7 +63,9 @@ typedef struct {
   int32_t device;         /* CUDA device ordinal                                         */
 } d2mhe_params;
 
-/* Validates params, builds all tables on `device`.  *out is NULL on failure. */
+/* Validates params, builds all tables on `device` and allocates the context's device memory (tables,
+ * key storage, index staging, and 64 MiB of scratch for the samples that d2mhe_encrypt and
+ * d2mhe_partial_decrypt draw ahead of their kernels).  *out is NULL on failure. */
 d2mhe_status d2mhe_create(const d2mhe_params* params, d2mhe_ctx** out);
 void d2mhe_destroy(d2mhe_ctx* ctx);
 /* Stream (a cudaStream_t passed as void*) on which later calls are enqueued; NULL = default. */
