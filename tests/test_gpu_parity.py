@@ -803,6 +803,37 @@ def test_ciphertext_index_shards_reproduce_the_whole(d2):
     ctx.close()
 
 
+def test_sample_batches_of_one_call_reproduce_separate_calls(d2):
+    """d2mhe_encrypt and d2mhe_partial_decrypt draw their samples into the context's 64 MiB scratch,
+    as many (party, ciphertext) or (recipient, ciphertext) units per pair of launches as fit.  A call
+    large enough to need several batches must produce, unit for unit, what one small call per slice
+    of the index range produces (every sample is addressed by its counters, not by its batch)."""
+    cfg = wl.round_config(1)
+    K, n = cfg.num_parties, cfg.n
+    moduli = cfg.moduli[:1]
+    ctx = d2.Context(cfg.log2_n, moduli, K, seed=9)
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    C = 1536  # encrypt: 4 * 1536 units of 3 N bytes = 72 MiB; shares: 4 * 1536 units of 4 N bytes = 96 MiB
+    assert K * C * 3 * n > 64 << 20
+    gen = torch.Generator().manual_seed(3)
+    plain = torch.randint(0, T, (K, C, n), dtype=torch.int32, generator=gen).to(ctx.device)
+    whole = ctx.empty_u64(K, C, 2, 1, n)
+    ctx.encrypt(parties, 7, C, plain, whole)
+    shares = ctx.empty_u64(K, K, C, 1, n)
+    ctx.partial_decrypt(whole, parties, parties, 7, C, shares)
+    # batches end after 5461 encryption units (party 3, index 853) and after 4096 share units (recipient 2, index 1024)
+    for first, cnt in ((0, 3), (851, 5), (1022, 5), (C - 3, 3)):
+        part = ctx.empty_u64(K, cnt, 2, 1, n)
+        ctx.encrypt(parties, 7 + first, cnt, plain[:, first:first + cnt].contiguous(), part)
+        assert torch.equal(part, whole[:, first:first + cnt])
+        sh = ctx.empty_u64(K, K, cnt, 1, n)
+        ctx.partial_decrypt(part, parties, parties, 7 + first, cnt, sh)
+        assert torch.equal(sh, shares[:, :, first:first + cnt])
+    ctx.close()
+
+
 def test_error_statuses(d2):
     cfg = wl.round_config(1)
     K, L, n = cfg.num_parties, cfg.num_limbs, cfg.n
