@@ -94,3 +94,39 @@ def test_muladd_definition():
         for l, q in enumerate(moduli):
             for j in range(32):
                 assert int(d[r, l, j]) == (int(a[r, l, j]) * int(b[r, l, j]) + int(c[r, l, j])) % q
+
+
+@pytest.mark.parametrize("log2_n,bits,L,batch", [(4, 30, 2, 2), (6, 54, 3, 3), (12, 36, 3, 2), (13, 54, 4, 2)])
+def test_batched_transform_row_to_limb_mapping(log2_n, bits, L, batch):
+    """Row (b, l) of a batch goes with limb l's prime and root (the ring isomorphism behind every
+    product of Sec. 3.2): values by Horner evaluation in Python integers at psi_l^(2j+1), inverse by
+    round trip and by the single-polynomial interpolation.  The limbs have different primes and
+    different roots, and every row holds different data, so that a wrong limb-of-row mapping, a
+    swapped root or a flipped direction switch fails."""
+    n = 1 << log2_n
+    moduli = wl.ntt_primes(bits, 2 * n, L)
+    assert len(set(moduli)) == L
+    o = orc.Oracle(log2_n, moduli, 65537, seed=1)
+    psi = [orc.find_psi(p, log2_n) for p in moduli]
+    # a second, different set of roots for the same primes: the wrapper must use the ones it is given
+    psi_alt = [pow(r, 3, p) for r, p in zip(psi, moduli)]
+    polys = wl.random_polys(moduli, log2_n, batch, seed=7)
+    assert polys.shape == (batch, L, n)
+    for roots in (psi, psi_alt):
+        fwd = o.ntt(polys, np.array(roots, dtype=np.uint64))
+        sample = range(n) if n <= 64 else (0, 1, 2, n // 2 - 1, n // 2, n - 2, n - 1)
+        for b in range(batch):
+            for l, p in enumerate(moduli):
+                coeffs = [int(x) for x in polys[b, l]]
+                for j in sample:
+                    assert int(fwd[b, l, j]) == defs.horner(coeffs, pow(roots[l], 2 * j + 1, p), p)
+        back = o.ntt(fwd, np.array(roots, dtype=np.uint64), inverse=True)
+        assert np.array_equal(back, polys)
+        # the inverse switch on its own: interpolation of one row through the single-polynomial routine
+        b, l = batch - 1, L - 1
+        assert np.array_equal(back[b, l], orc.negacyclic_interp(fwd[b, l], roots[l], moduli[l]))
+        assert not np.array_equal(fwd[b, l], polys[b, l])
+    # rows of different limbs really differ in modulus: the same coefficients under two limbs give different values
+    same = np.broadcast_to(polys[0, 0] % np.uint64(min(moduli)), (1, L, n)).copy()
+    f = o.ntt(same, np.array(psi, dtype=np.uint64))
+    assert not np.array_equal(f[0, 0], f[0, 1])
