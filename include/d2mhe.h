@@ -13,8 +13,11 @@
  *    holding the residues mod q_l in [0, q_l), in the COEFFICIENT domain.
  *  - Unless a parameter says "host", every data pointer is a DEVICE pointer,
  *    16-byte aligned, sized exactly as annotated, owned by the caller.
- *  - Hot calls are asynchronous on the context's stream, allocate nothing and
- *    do not synchronise.  The library allocates only in d2mhe_create.
+ *  - Hot calls are asynchronous on the context's stream and allocate nothing.  Calls that take
+ *    HOST index lists (parties, recipients, neighbour lists) copy them through a ring of four
+ *    pinned staging slots; a call waits on the host only when all four slots belong to calls whose
+ *    work on the GPU has not finished yet, i.e. from the fifth such call in flight.  The library
+ *    allocates only in d2mhe_create (and in the test hooks).
  *  - Every function returns a d2mhe_status (0 = success, < 0 = error) and
  *    never aborts.  Arguments visible on the host are validated before any
  *    launch; a failed validation launches nothing.  Asynchronous CUDA errors
@@ -44,7 +47,8 @@ enum {
   D2MHE_ERR_WORKSPACE = -4,   /* caller-provided workspace too small                     */
   D2MHE_ERR_CUDA = -5,        /* a CUDA runtime call failed                              */
   D2MHE_ERR_RANGE = -6,       /* index out of range, or a value outside (-t/2, t/2)      */
-  D2MHE_ERR_UNSUPPORTED = -7  /* operation not available for these parameters            */
+  D2MHE_ERR_UNSUPPORTED = -7, /* operation not available for these parameters            */
+  D2MHE_ERR_DEVICE_CHECK = -8 /* a check that runs on the device failed (see `flags`)    */
 };
 
 typedef struct {
@@ -256,7 +260,9 @@ d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* ctx, const uint32_t* a_dev, const ui
  *   more, smaller sub-chunks.  The contents left in the workspace are unspecified.
  * d2mhe_round_device takes device values/sums.  d2mhe_round_host takes HOST values/sums
  * (pinned memory recommended), copies each sub-chunk in and out on the stream that
- * computes it and returns after all of it has finished.
+ * computes it and returns after all of it has finished; it returns D2MHE_ERR_RANGE (sums then
+ * unspecified) if a value was outside [-(t-1)/2, (t-1)/2].  If a launch or copy fails part-way,
+ * the internal streams are still joined back into the context's stream before the call returns.
  */
 size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* ctx, uint32_t chunk_cts);
 /*
@@ -285,14 +291,19 @@ d2mhe_status d2mhe_round_host(d2mhe_ctx* ctx, const int32_t* values_host, uint32
  * Think of a service that gave all device memory to a fixed pool at start-up, a plug-in
  * that receives only its input and output buffers, or a latency-critical loop in which
  * cudaMalloc is banned because it synchronises the device.  The chunk's protocol messages
- * live in a 64 MiB array that is part of the library image (every GPU that loads the
- * library holds those 64 MiB until the process exits); the caller passes only values and sums.
+ * live in a 64 MiB array that is part of the library image (a GPU reserves those 64 MiB when the
+ * first call of this function on it loads that part of the image, and holds them until the process
+ * exits); the caller passes only values and sums.
  *  - Calls no cudaMalloc / cudaFree and no allocating library routine.
  *  - Returns D2MHE_ERR_WORKSPACE when one ciphertext index of this parameter set needs more
  *    than 64 MiB, i.e. when d2mhe_round_workspace_bytes(ctx, 1) > 67108864 (configuration 2,
  *    K = 10, N = 8192, L = 4, needs 36.3 MB and fits; K = 20, N = 16384, L = 8 does not).
- *  - The first call on a device looks up the array's device address (a synchronous runtime
- *    query); make that first call before starting any stream capture.
+ *  - The first call on a device loads the array's image and looks up its device address (a
+ *    synchronous runtime query that makes the device set the 64 MiB aside): make that first call
+ *    at start-up, before the rest of the device memory is handed to a pool and before starting any
+ *    stream capture.  If the device has no room left, that call returns D2MHE_ERR_CUDA and a later
+ *    call tries again.  Later calls only read the cached address; first calls from several host
+ *    threads are serialised by a lock.
  *  - All contexts and all calls on one GPU share the array, which keeps the last call's
  *    contents.  Nothing has to be cleared (every buffer is written before it is read), but
  *    two calls whose work overlaps on the GPU (different streams, threads or contexts) race.
@@ -303,9 +314,12 @@ d2mhe_status d2mhe_round_device_static(d2mhe_ctx* ctx, const int32_t* values_dev
                                        const uint32_t* nbr_rows, int32_t* sums_dev);
 
 /* Test hooks. */
-/* s_k as int8 [N] on the HOST (needs a key share for `party`). */
+/* s_k as int8 [N] on the HOST (needs a key share for `party`): the key that the device stores (in
+ * the transform domain) is inverse-transformed on the GPU, limb by limb, and copied back;
+ * D2MHE_ERR_DEVICE_CHECK if the limbs disagree or a coefficient is not in {-1, 0, 1}.  Allocates a
+ * temporary device buffer and synchronises the stream. */
 d2mhe_status d2mhe_debug_export_secret(d2mhe_ctx* ctx, uint32_t party, int8_t* s_host);
-/* sk_i of a user's own key pair as int8 [N] on the HOST (needs d2mhe_user_keygen for `user`). */
+/* The same for sk_i of a user's own key pair (needs d2mhe_user_keygen for `user`). */
 d2mhe_status d2mhe_debug_export_user_secret(d2mhe_ctx* ctx, uint32_t user, int8_t* s_host);
 /* The primitive 2N-th root of unity used for limb `limb`. */
 d2mhe_status d2mhe_get_root(const d2mhe_ctx* ctx, uint32_t limb, uint64_t* psi);

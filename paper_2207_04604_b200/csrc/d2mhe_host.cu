@@ -11,6 +11,9 @@
 
 typedef unsigned __int128 u128;
 
+// launcher of the context's kernel build
+#define L_(fn) d2mhe_launch::fn
+
 namespace {
 
 const u64 kGaussCdt[D2MHE_CDT_LEN] = {
@@ -179,6 +182,12 @@ d2mhe_status release_slot(d2mhe_ctx* c, const Staged& s) {
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->idx_event_valid[s.slot] = true;
   return D2MHE_OK;
+}
+// Exit of a call that staged indices and then failed with CUDA error `e`: the slot still gets its
+// event (whatever was queued before the failure reads it), and the failure is what is reported.
+d2mhe_status fail_staged(d2mhe_ctx* c, const Staged& s, cudaError_t e) {
+  (void)release_slot(c, s);
+  return fail_cuda(c, e);
 }
 
 d2mhe_status check_party_list(const d2mhe_ctx* c, const u32* parties, u32 n, bool need_share,
@@ -435,6 +444,7 @@ const char* d2mhe_strerror(d2mhe_status s) {
     case D2MHE_ERR_CUDA: return "CUDA error";
     case D2MHE_ERR_RANGE: return "index or value out of range";
     case D2MHE_ERR_UNSUPPORTED: return "unsupported for these parameters";
+    case D2MHE_ERR_DEVICE_CHECK: return "a device-side check failed";
     default: return "unknown status";
   }
 }
@@ -471,6 +481,8 @@ d2mhe_status d2mhe_create(const d2mhe_params* P, d2mhe_ctx** out) {
   c->narrow = true;
   for (u32 l = 0; l < P->num_limbs; ++l)
     if (P->moduli[l] >= ((u64)1 << 30)) c->narrow = false;
+  c->all_parties.resize(P->num_parties);
+  for (u32 i = 0; i < P->num_parties; ++i) c->all_parties[i] = i;
   c->has_share.assign(P->num_parties, false);
   c->has_user_key.assign(P->num_parties, false);
   std::memset(&c->view, 0, sizeof(c->view));
@@ -546,7 +558,7 @@ d2mhe_status d2mhe_keygen_share(d2mhe_ctx* c, const u32* parties, u32 n_parties)
   const size_t counts[1] = {n_parties};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
   cudaError_t e = d2mhe_launch::keygen(c->view, c->limb_params, c->stream, sg.dev[0], n_parties);
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
   for (u32 i = 0; i < n_parties; ++i) c->has_share[parties[i]] = true;
   return release_slot(c, sg);
@@ -566,12 +578,12 @@ d2mhe_status d2mhe_collective_pk(d2mhe_ctx* c, const u32* parties, u32 n_parties
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
   cudaError_t e = d2mhe_launch::collective_pk(c->view, c->limb_params, c->stream, sg.dev[0], n_parties,
                                               reinterpret_cast<u64*>(pk_shares_dev));
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
   if (pk_dev) {
     e = cudaMemcpyAsync(pk_dev, c->view.pk_coef, 2 * (size_t)c->view.L * c->view.n * sizeof(u64),
                         cudaMemcpyDeviceToDevice, c->stream);
-    if (e != cudaSuccess) return fail_cuda(c, e);
+    if (e != cudaSuccess) return fail_staged(c, sg, e);
   }
   c->pk_parties.assign(parties, parties + n_parties);
   c->has_pk = true;
@@ -620,7 +632,7 @@ d2mhe_status d2mhe_encrypt(d2mhe_ctx* c, const u32* parties, u32 n_parties, u32 
   cudaError_t e = d2mhe_launch::encrypt(c->view, c->limb_params, c->stream, sg.dev[0], n_parties, ct_first, n_cts,
                                         plain_dev, reinterpret_cast<u64*>(ct_dev), c->noise_scratch,
                                         c->noise_scratch_bytes, &launched);
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += launched;
   return release_slot(c, sg);
 }
@@ -650,7 +662,7 @@ d2mhe_status d2mhe_aggregate(d2mhe_ctx* c, const uint64_t* ct_dev, u32 n_rows, u
   if (st != D2MHE_OK) return st;
   cudaError_t e = d2mhe_launch::aggregate(c->view, c->stream, reinterpret_cast<const u64*>(ct_dev), n_cts,
                                           sg.dev[0], sg.dev[1], n_out, reinterpret_cast<u64*>(agg_dev));
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
   return release_slot(c, sg);
 }
@@ -671,14 +683,14 @@ d2mhe_status d2mhe_partial_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev, const 
   Staged sg;
   const u32* arrays[2] = {recipients, parties};
   const size_t counts[2] = {n_rec, n_parties};
-  if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
   // the noise of the shares is sampled ahead into the context's scratch, batch by batch
   if ((size_t)n_parties * c->view.n > c->noise_scratch_bytes) return D2MHE_ERR_UNSUPPORTED;
+  if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
   u32 launched = 0;
   cudaError_t e = d2mhe_launch::partial_decrypt_scratch(
       c->view, c->limb_params, c->stream, reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1], n_parties,
       ct_first, n_cts, reinterpret_cast<u64*>(shares_dev), c->noise_scratch, c->noise_scratch_bytes, &launched);
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += launched;
   return release_slot(c, sg);
 }
@@ -776,14 +788,14 @@ d2mhe_status d2mhe_user_keygen(d2mhe_ctx* c, const u32* users, u32 n_users, uint
   const size_t counts[1] = {n_users};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
   cudaError_t e = d2mhe_launch::user_keygen(c->view, c->limb_params, c->stream, sg.dev[0], n_users);
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
   const size_t pk_words = 2 * (size_t)c->view.L * c->view.n;
   if (pk_out_dev) {
     for (u32 i = 0; i < n_users; ++i) {
       e = cudaMemcpyAsync(pk_out_dev + (size_t)i * pk_words, c->view.upk_coef + (size_t)users[i] * pk_words,
                           pk_words * sizeof(u64), cudaMemcpyDeviceToDevice, c->stream);
-      if (e != cudaSuccess) return fail_cuda(c, e);
+      if (e != cudaSuccess) return fail_staged(c, sg, e);
     }
   }
   for (u32 i = 0; i < n_users; ++i) c->has_user_key[users[i]] = true;
@@ -812,7 +824,7 @@ d2mhe_status d2mhe_convert_share(d2mhe_ctx* c, const uint64_t* agg_dev, const u3
   cudaError_t e = d2mhe_launch::convert_share(c->view, c->limb_params, c->stream,
                                               reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1],
                                               n_parties, ct_first, n_cts, reinterpret_cast<u64*>(shares_dev));
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
   return release_slot(c, sg);
 }
@@ -851,11 +863,11 @@ d2mhe_status d2mhe_decrypt(d2mhe_ctx* c, const u32* users, u32 n_users, const ui
   cudaError_t e = d2mhe_launch::secret_product(c->view, c->limb_params, c->stream,
                                                reinterpret_cast<const u64*>(ct_dev), sg.dev[0], n_users, n_cts,
                                                reinterpret_cast<u64*>(scratch_dev));
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   // [c_0 + c_1 sk_i]_q then the exact scale-and-round: the product plays the role of one share
   e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(ct_dev),
                             reinterpret_cast<const u64*>(scratch_dev), n_users, 1, 1, n_cts, plain_dev);
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 2;
   return release_slot(c, sg);
 }
@@ -882,7 +894,7 @@ d2mhe_status d2mhe_bootstrap_share(d2mhe_ctx* c, const uint64_t* agg_dev, const 
   cudaError_t e = d2mhe_launch::boot_share(c->view, c->limb_params, c->stream,
                                            reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1],
                                            n_parties, ct_first, n_cts, reinterpret_cast<u64*>(shares_dev));
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
   return release_slot(c, sg);
 }
@@ -907,10 +919,10 @@ d2mhe_status d2mhe_bootstrap_combine(d2mhe_ctx* c, const uint64_t* agg_dev, cons
   cudaError_t e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
                                         reinterpret_cast<const u64*>(shares_dev), n_rec, n_shares, 2, n_cts,
                                         plain_scratch_dev);
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   e = d2mhe_launch::boot_finish(c->view, c->stream, plain_scratch_dev, reinterpret_cast<const u64*>(shares_dev),
                                 sg.dev[0], n_rec, n_shares, ct_first, n_cts, reinterpret_cast<u64*>(ct_out_dev));
-  if (e != cudaSuccess) return fail_cuda(c, e);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 2;
   return release_slot(c, sg);
 }
@@ -1003,72 +1015,83 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
   for (u32 l = 0; l < lanes; ++l) lane_first[l + 1] = lane_first[l] + sub_small + (l < n_large ? 1u : 0u);
 
   DeviceGuard guard(c->device);
-  std::vector<u32> all(K);
-  for (u32 i = 0; i < K; ++i) all[i] = i;
   const u32 dummy = 0;
   Staged sg;  // the four index lists of every sub-chunk, staged once
-  const u32* arrays[4] = {all.data(), c->pk_parties.data(), nbr_offsets, nnz ? nbr_rows : &dummy};
+  const u32* arrays[4] = {c->all_parties.data(), c->pk_parties.data(), nbr_offsets, nnz ? nbr_rows : &dummy};
   const size_t counts[4] = {K, S, (size_t)K + 1, nnz ? (size_t)nnz : 1};
   d2mhe_status st = stage_indices(c, arrays, counts, 4, &sg);
   if (st != D2MHE_OK) return st;
-  cudaError_t e;
-  if (lanes > 1) {
-    if ((e = cudaEventRecord(c->fork_event, c->stream)) != cudaSuccess) return fail_cuda(c, e);
-    for (u32 l = 0; l < lanes; ++l)
-      if ((e = cudaStreamWaitEvent(c->lane_stream[l], c->fork_event, 0)) != cudaSuccess) return fail_cuda(c, e);
-  }
   unsigned char* base = reinterpret_cast<unsigned char*>(ws);
-  u32 done = 0;
-  for (u32 i = 0; i < n_sub; ++i) {
-    const u32 cc = sub_small + (i < n_large ? 1u : 0u), lane = i % lanes;
-    cudaStream_t s = lanes > 1 ? c->lane_stream[lane] : c->stream;
-    // layout of the lane's part (all 16-byte aligned: every block is a multiple of 16 bytes)
-    unsigned char* lane_base = base + lane_first[lane] * per_ct;
-    u32* plain = reinterpret_cast<u32*>(lane_base);
-    u64* ct = reinterpret_cast<u64*>(lane_base + (size_t)K * cc * n * sizeof(u32));
-    u64* agg = ct + (size_t)K * cc * 2 * polyw;
-    u64* shares = agg + (size_t)K * cc * 2 * polyw;
-    int32_t* vals_dev = reinterpret_cast<int32_t*>(plain);  // encode and decode run in place
-    // values are [K, n_cts, N]: one strided copy, K rows of cc*N values, rows n_cts*N apart
-    e = cudaMemcpy2DAsync(vals_dev, (size_t)cc * n * sizeof(int32_t), values + (size_t)done * n,
-                          (size_t)n_cts * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
-                          host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s);
-    if (e != cudaSuccess) return fail_cuda(c, e);
-    if ((e = d2mhe_launch::encode(c->view, s, vals_dev, K * cc, plain)) != cudaSuccess) return fail_cuda(c, e);
-    unsigned char* noise = reinterpret_cast<unsigned char*>(shares + (size_t)K * S * cc * polyw);
-    const size_t noise_bytes = round_noise_bytes_per_ct(c) * cc;  // first u, e_0, e_1, later the shares' noise
-    u32 enc_launches = 0;
-    if ((e = d2mhe_launch::encrypt(c->view, c->limb_params, s, sg.dev[0], K, ct_first + done, cc, plain, ct, noise,
-                                   noise_bytes, &enc_launches)) != cudaSuccess)
-      return fail_cuda(c, e);
-    if ((e = d2mhe_launch::aggregate(c->view, s, ct, cc, sg.dev[2], sg.dev[3], K, agg)) != cudaSuccess)
-      return fail_cuda(c, e);
-    u32 pdec_launches = 0;
-    if ((e = d2mhe_launch::partial_decrypt_scratch(c->view, c->limb_params, s, agg, sg.dev[0], K, sg.dev[1], S,
-                                                   ct_first + done, cc, shares, noise, noise_bytes,
-                                                   &pdec_launches)) !=
-        cudaSuccess)
-      return fail_cuda(c, e);
-    if ((e = d2mhe_launch::combine(c->view, s, agg, shares, K, S, 1, cc, plain)) != cudaSuccess)
-      return fail_cuda(c, e);
-    if ((e = d2mhe_launch::decode(c->view, s, plain, K * cc, vals_dev)) != cudaSuccess) return fail_cuda(c, e);
-    c->launches += 4 + enc_launches + pdec_launches;
-    e = cudaMemcpy2DAsync(sums + (size_t)done * n, (size_t)n_cts * n * sizeof(int32_t), vals_dev,
-                          (size_t)cc * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
-                          host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, s);
-    if (e != cudaSuccess) return fail_cuda(c, e);
-    done += cc;
-  }
+  // Everything between the fork and the join; a failure stops issuing, and the join below still runs,
+  // so that the context's stream stays ordered after whatever the lanes were given.
+  auto issue = [&]() -> cudaError_t {
+    cudaError_t e;
+    if (lanes > 1) {
+      if ((e = cudaEventRecord(c->fork_event, c->stream)) != cudaSuccess) return e;
+      for (u32 l = 0; l < lanes; ++l)
+        if ((e = cudaStreamWaitEvent(c->lane_stream[l], c->fork_event, 0)) != cudaSuccess) return e;
+    }
+    u32 done = 0;
+    for (u32 i = 0; i < n_sub; ++i) {
+      const u32 cc = sub_small + (i < n_large ? 1u : 0u), lane = i % lanes;
+      cudaStream_t s = lanes > 1 ? c->lane_stream[lane] : c->stream;
+      // layout of the lane's part (all 16-byte aligned: every block is a multiple of 16 bytes)
+      unsigned char* lane_base = base + lane_first[lane] * per_ct;
+      u32* plain = reinterpret_cast<u32*>(lane_base);
+      u64* ct = reinterpret_cast<u64*>(lane_base + (size_t)K * cc * n * sizeof(u32));
+      u64* agg = ct + (size_t)K * cc * 2 * polyw;
+      u64* shares = agg + (size_t)K * cc * 2 * polyw;
+      int32_t* vals_dev = reinterpret_cast<int32_t*>(plain);  // encode and decode run in place
+      // values are [K, n_cts, N]: one strided copy, K rows of cc*N values, rows n_cts*N apart
+      e = cudaMemcpy2DAsync(vals_dev, (size_t)cc * n * sizeof(int32_t), values + (size_t)done * n,
+                            (size_t)n_cts * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
+                            host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s);
+      if (e != cudaSuccess) return e;
+      if ((e = L_(encode)(c->view, s, vals_dev, K * cc, plain)) != cudaSuccess) return e;
+      unsigned char* noise = reinterpret_cast<unsigned char*>(shares + (size_t)K * S * cc * polyw);
+      const size_t noise_bytes = round_noise_bytes_per_ct(c) * cc;  // first u, e_0, e_1, later the shares' noise
+      u32 enc_launches = 0;
+      if ((e = L_(encrypt)(c->view, c->limb_params, s, sg.dev[0], K, ct_first + done, cc, plain, ct, noise,
+                           noise_bytes, &enc_launches)) != cudaSuccess)
+        return e;
+      if ((e = L_(aggregate)(c->view, s, ct, cc, sg.dev[2], sg.dev[3], K, agg)) != cudaSuccess) return e;
+      u32 pdec_launches = 0;
+      if ((e = L_(partial_decrypt_scratch)(c->view, c->limb_params, s, agg, sg.dev[0], K, sg.dev[1], S,
+                                           ct_first + done, cc, shares, noise, noise_bytes, &pdec_launches)) !=
+          cudaSuccess)
+        return e;
+      if ((e = L_(combine)(c->view, s, agg, shares, K, S, 1, cc, plain)) != cudaSuccess) return e;
+      if ((e = L_(decode)(c->view, s, plain, K * cc, vals_dev)) != cudaSuccess) return e;
+      c->launches += 4 + enc_launches + pdec_launches;
+      e = cudaMemcpy2DAsync(sums + (size_t)done * n, (size_t)n_cts * n * sizeof(int32_t), vals_dev,
+                            (size_t)cc * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
+                            host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, s);
+      if (e != cudaSuccess) return e;
+      done += cc;
+    }
+    return cudaSuccess;
+  };
+  cudaError_t e = issue();
   if (lanes > 1) {
     for (u32 l = 0; l < lanes; ++l) {
-      if ((e = cudaEventRecord(c->lane_event[l], c->lane_stream[l])) != cudaSuccess) return fail_cuda(c, e);
-      if ((e = cudaStreamWaitEvent(c->stream, c->lane_event[l], 0)) != cudaSuccess) return fail_cuda(c, e);
+      cudaError_t j = cudaEventRecord(c->lane_event[l], c->lane_stream[l]);
+      if (j == cudaSuccess) j = cudaStreamWaitEvent(c->stream, c->lane_event[l], 0);
+      if (e == cudaSuccess) e = j;
     }
   }
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
   if ((st = release_slot(c, sg)) != D2MHE_OK) return st;
   if (host_io) {
-    e = cudaStreamSynchronize(c->stream);
-    if (e != cudaSuccess) return fail_cuda(c, e);
+    // the call returns when the sums are in host memory, so it can also report values that
+    // d2mhe_encode found out of range (the flag is cleared, as d2mhe_sync does)
+    if ((e = cudaStreamSynchronize(c->stream)) != cudaSuccess) return fail_cuda(c, e);
+    u32 flag = 0;
+    if ((e = cudaMemcpy(&flag, c->view.range_flag, sizeof(u32), cudaMemcpyDeviceToHost)) != cudaSuccess)
+      return fail_cuda(c, e);
+    if (flag) {
+      if ((e = cudaMemset(c->view.range_flag, 0, sizeof(u32))) != cudaSuccess) return fail_cuda(c, e);
+      return D2MHE_ERR_RANGE;
+    }
   }
   return D2MHE_OK;
 }
@@ -1088,22 +1111,48 @@ d2mhe_status d2mhe_round_host(d2mhe_ctx* c, const int32_t* values_host, u32 ct_f
 
 // ---- test hooks ----------------------------------------------------------------------
 
+// What the device holds for a key, read back: the stored rows go through an inverse transform on the
+// GPU (one CTA per limb) and every limb must give the same polynomial with coefficients in {-1, 0, 1}.
+// Allocates a temporary device buffer and synchronises: a test hook, not a hot call.
+static d2mhe_status export_key(d2mhe_ctx* c, const u64* key_dev, int8_t* s_host) {
+  DeviceGuard guard(c->device);
+  const size_t n = c->view.n, L = c->view.L;
+  signed char* tmp = nullptr;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&tmp), L * n);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  std::vector<signed char> host(L * n);
+  e = d2mhe_launch::export_secret(c->view, c->limb_params, c->stream, key_dev, tmp);
+  if (e == cudaSuccess) {
+    c->launches += 1;
+    e = cudaMemcpyAsync(host.data(), tmp, L * n, cudaMemcpyDeviceToHost, c->stream);
+  }
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  cudaFree(tmp);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  for (size_t j = 0; j < n; ++j) {
+    const signed char v0 = host[j];
+    if (v0 == 127) return D2MHE_ERR_DEVICE_CHECK;
+    for (size_t l = 1; l < L; ++l)
+      if (host[l * n + j] != v0) return D2MHE_ERR_DEVICE_CHECK;
+    s_host[j] = (int8_t)v0;
+  }
+  return D2MHE_OK;
+}
+
 d2mhe_status d2mhe_debug_export_secret(d2mhe_ctx* c, u32 party, int8_t* s_host) {
   if (!c || !s_host) return D2MHE_ERR_INVALID_ARG;
   if (party >= c->params.num_parties) return D2MHE_ERR_RANGE;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
   if (!c->has_share[party]) return D2MHE_ERR_STATE;
-  const Stream st(c->params.seed, TAG_SECRET, 0, party, 0);
-  for (u32 j = 0; j < c->view.n; ++j) s_host[j] = (int8_t)st.ternary(j);
-  return D2MHE_OK;
+  return export_key(c, c->view.s_mont + (size_t)party * c->view.L * c->view.n, s_host);
 }
 
 d2mhe_status d2mhe_debug_export_user_secret(d2mhe_ctx* c, u32 user, int8_t* s_host) {
   if (!c || !s_host) return D2MHE_ERR_INVALID_ARG;
   if (user >= c->params.num_parties) return D2MHE_ERR_RANGE;
+  if (!protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
   if (!c->has_user_key[user]) return D2MHE_ERR_STATE;
-  const Stream st(c->params.seed, TAG_USER_SECRET, 0, user, 0);
-  for (u32 j = 0; j < c->view.n; ++j) s_host[j] = (int8_t)st.ternary(j);
-  return D2MHE_OK;
+  return export_key(c, c->view.usk_mont + (size_t)user * c->view.L * c->view.n, s_host);
 }
 
 d2mhe_status d2mhe_get_root(const d2mhe_ctx* c, u32 limb, uint64_t* psi) {

@@ -88,6 +88,7 @@ struct d2mhe_ctx {
   std::vector<bool> has_share;
   std::vector<bool> has_user_key;
   std::vector<u32> pk_parties;      // party set of the last collective_pk
+  std::vector<u32> all_parties;     // 0 .. K-1 (the users of a whole-round call)
   bool has_pk = false;
   u64 launches = 0;
   // index staging: pinned host ring + device ring, one event per slot
@@ -108,6 +109,8 @@ namespace d2mhe_launch {
 cudaError_t keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties);
 cudaError_t collective_pk(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
                           u64* shares_out);
+// test hook: key rows [L][N] (transform domain, Montgomery form) -> int8 coefficients [L][N] (127 = not ternary)
+cudaError_t export_secret(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* key, signed char* out);
 cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain);
 cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values);
 // u, e_0, e_1 are sampled ahead into caller-lent scratch (at least 3 N bytes)

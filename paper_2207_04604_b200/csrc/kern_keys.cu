@@ -84,9 +84,36 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
       });
 }
 
+// Test hook: a stored key (rows of NTT(s) * N^-1 in Montgomery form, one per limb) brought back to
+// the coefficient domain; out[l][j] = the coefficient as -1, 0 or 1, or 127 if the residue of limb l
+// is none of these.   grid = L
+template <int LOGN, int G, bool WIDE>
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+    k_export_secret(DevView v, const __grid_constant__ LimbParams lp, const u64* key, signed char* __restrict__ out) {
+  const u32 l = blockIdx.x;
+  const LimbTab& lt = lp.limbs[l];
+  const u64* row = key + (size_t)l * v.n;
+  signed char* o = out + (size_t)l * v.n;
+  ntt_inverse<LOGN, G, WIDE>(
+      poly_smem(), lt, v.logn,
+      [&](int, u32 q, u64(&x)[8]) {
+        load_octet_rw(row + 8 * (size_t)q, x);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x[k] = mont_lazy(x[k], 1, lt.p, lt.pinv);  // leaves Montgomery form; below 2p
+      },
+      [&](u32 j, u64 val) {
+        const u64 c = canon4(val, lt);
+        o[j] = c == 0 ? 0 : c == 1 ? 1 : c == lt.p - 1 ? -1 : 127;
+      });
+}
+
 }  // namespace
 
 namespace d2mhe_launch {
+
+cudaError_t export_secret(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* key, signed char* out) {
+  D2MHE_DISPATCH(k_export_secret, v, v.L, s, v, lp, key, out);
+}
 
 cudaError_t keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties) {
   D2MHE_DISPATCH(k_keygen, v, n_parties * v.L, s, v, lp, parties_dev);

@@ -142,8 +142,10 @@ __device__ __forceinline__ void ct32(u32& X, u32& Y, uint2 w, u32 t, u32 twot) {
 }
 
 // encode: values -> slots at bit-reversed positions -> inverse transform, two stages per barrier
+// values and plain may be the same storage (every CTA reads its whole row into shared memory before
+// it writes the row back), so neither pointer is declared __restrict__
 __global__ void __launch_bounds__(1024)
-    k_encode(DevView v, const int32_t* __restrict__ values, u32* __restrict__ plain) {
+    k_encode(DevView v, const int32_t* values, u32* plain) {
   u32* sm = reinterpret_cast<u32*>(smem_raw);
   const PlainTab pt = v.plain;
   const u32 n = v.n, logn = v.logn, t = pt.t, twot = pt.twot;
@@ -194,8 +196,9 @@ __global__ void __launch_bounds__(1024)
 }
 
 // decode: forward transform (two stages per barrier), slots read back from bit-reversed positions
+// plain and values may be the same storage (see k_encode)
 __global__ void __launch_bounds__(1024)
-    k_decode(DevView v, const u32* __restrict__ plain, int32_t* __restrict__ values) {
+    k_decode(DevView v, const u32* plain, int32_t* values) {
   u32* sm = reinterpret_cast<u32*>(smem_raw);
   const PlainTab pt = v.plain;
   const u32 n = v.n, logn = v.logn, t = pt.t, twot = pt.twot;

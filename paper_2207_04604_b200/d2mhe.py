@@ -22,6 +22,7 @@ ERR_WORKSPACE = -4
 ERR_CUDA = -5
 ERR_RANGE = -6
 ERR_UNSUPPORTED = -7
+ERR_DEVICE_CHECK = -8
 
 EXPORTS = [
     "d2mhe_create", "d2mhe_destroy", "d2mhe_set_stream", "d2mhe_sync", "d2mhe_strerror",

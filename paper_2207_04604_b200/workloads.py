@@ -13,6 +13,8 @@ the cryptographic path.
 from dataclasses import dataclass, field
 from typing import List
 
+import os
+
 import numpy as np
 
 PLAIN_MODULUS = 65537
@@ -185,27 +187,41 @@ def quantise(grad_f32: np.ndarray, clip: int) -> np.ndarray:
     return np.clip(scaled, -clip, clip).astype(np.int32)
 
 
-def gradients(cfg: RoundConfig, seed: int, ct_first: int = 0, n_cts: int = None) -> np.ndarray:
+def gradients(cfg: RoundConfig, seed: int, ct_first: int = 0, n_cts: int = None, threads: int = 0) -> np.ndarray:
     """int32 [K, n_cts, N] slot values for ciphertext indices ct_first .. ct_first+n_cts-1.
 
     Each (party, ciphertext index) block has its own generator, so any slice of
-    the gradient can be produced without materialising the whole of it.
+    the gradient can be produced without materialising the whole of it, and the
+    blocks can be filled by `threads` host threads (0: one per core, at most 16)
+    with the same result.
     """
     n_cts = cfg.num_cts if n_cts is None else n_cts
     out = np.zeros((cfg.num_parties, n_cts, cfg.n), dtype=np.int32)
-    for k in range(cfg.num_parties):
-        for c in range(n_cts):
-            idx = ct_first + c
+
+    def fill(c):
+        idx = ct_first + c
+        first = idx * cfg.n
+        valid = max(0, min(cfg.n, cfg.params - first))
+        for k in range(cfg.num_parties):
             rng = np.random.default_rng([1000 + seed, k, idx])
             if cfg.int_range:
                 block = rng.integers(-cfg.int_range, cfg.int_range + 1, size=cfg.n).astype(np.int32)
             else:
                 g = rng.normal(0.0, cfg.grad_sigma, size=cfg.n).astype(np.float32)
                 block = quantise(g, cfg.clip)
-            first = idx * cfg.n
-            valid = max(0, min(cfg.n, cfg.params - first))
             block[valid:] = 0
             out[k, c] = block
+
+    if threads <= 0:
+        threads = min(16, os.cpu_count() or 1)
+    if threads == 1 or n_cts * cfg.num_parties < 64:
+        for c in range(n_cts):
+            fill(c)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(fill, range(n_cts)))
     return out
 
 

@@ -478,10 +478,68 @@ def test_large_configs_on_sampled_ciphertext_indices(d2, index, sample):
     ctx.close()
 
 
+def test_config3_every_message_of_every_index(d2):
+    """Configuration 3 (K = 20, N = 16384, L = 8) on all 66 ciphertext indices, three at a time:
+    plaintexts, ciphertexts, neighbour sums, all K x K decryption shares, decrypted plaintexts and
+    decoded sums against the oracle.  The slow test of the suite (the oracle needs about a minute
+    and a half for this workload on 16 cores)."""
+    cfg = wl.round_config(3)
+    seed = 1
+    K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, cfg.num_cts
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, K, seed=seed)
+    o = make_oracle(cfg.log2_n, cfg.moduli, seed=seed)
+    offsets, rows = wl.regular_graph(K, cfg.degree, seed)
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    pk = ctx.empty_u64(2, L, n)
+    ctx.collective_pk(parties, None, pk)
+    want_pk = o.collective_pk(parties)
+    assert np.array_equal(d2.to_u64_numpy(pk), want_pk)
+    step = 3
+    for first in range(0, C, step):
+        cc = min(step, C - first)
+        values = wl.gradients(cfg, seed, ct_first=first, n_cts=cc)
+        dv = torch.from_numpy(values).to(ctx.device)
+        plain = ctx.empty_u32(K, cc, n)
+        ctx.encode(dv, K * cc, plain)
+        ct = ctx.empty_u64(K, cc, 2, L, n)
+        ctx.encrypt(parties, first, cc, plain, ct)
+        agg = ctx.empty_u64(K, cc, 2, L, n)
+        ctx.aggregate(ct, K, cc, offsets, rows, agg)
+        shares = ctx.empty_u64(K, K, cc, L, n)
+        ctx.partial_decrypt(agg, parties, parties, first, cc, shares)
+        out_plain = ctx.empty_u32(K, cc, n)
+        ctx.combine_decrypt(agg, shares, K, K, cc, out_plain)
+        sums = torch.empty((K, cc, n), dtype=torch.int32, device=ctx.device)
+        ctx.decode(out_plain, K * cc, sums)
+        ctx.sync()
+        want_plain = o.encode(values)
+        assert np.array_equal(d2.to_u32_numpy(plain), want_plain)
+        want_ct = o.encrypt(want_pk, parties, first, want_plain)
+        assert np.array_equal(d2.to_u64_numpy(ct), want_ct)
+        del ct
+        want_agg = o.aggregate(want_ct, offsets, rows)
+        del want_ct
+        assert np.array_equal(d2.to_u64_numpy(agg), want_agg)
+        want_shares = o.partial_decrypt(want_agg, parties, parties, first)
+        assert np.array_equal(d2.to_u64_numpy(shares), want_shares)
+        del shares
+        want_out = o.combine(want_agg, want_shares)
+        del want_shares, want_agg
+        assert np.array_equal(d2.to_u32_numpy(out_plain), want_out)
+        got = sums.cpu().numpy()
+        assert np.array_equal(got, o.decode(want_out))
+        for i in range(K):
+            lst = rows[offsets[i]:offsets[i + 1]]
+            assert np.array_equal(got[i], values[lst].astype(np.int64).sum(axis=0))
+    ctx.close()
+
+
 @pytest.mark.parametrize("index", [3, 4])
 def test_whole_round_at_full_size_in_the_benchmark_configuration(d2, index):
     """Configurations 3 and 4 at full K, N, L and all C ciphertext indices through one whole-round call,
     cut as the benchmark cuts it (workspace sized from free memory, sub-chunks on two streams).
+    Every index carries the workload's gradients.
     Every decrypted sum is checked against the plaintext neighbour sum; for the last ciphertext index
     (the ragged tail), whose sub-chunk is still in the workspace when the call returns, the
     ciphertexts, aggregates and the shares for three recipients are compared with the oracle."""
@@ -494,12 +552,10 @@ def test_whole_round_at_full_size_in_the_benchmark_configuration(d2, index):
     ctx.keygen_share(parties)
     ctx.collective_pk(parties)
     offsets, rows = wl.regular_graph(K, cfg.degree, seed)
-    # inputs: the workload's gradients on the sampled index, a seeded fill in the clip range elsewhere
+    # inputs: the workload's gradients on every index (clipped Gaussian, zero-padded ragged tail)
     last = C - 1
-    gen = torch.Generator(device="cpu").manual_seed(seed)
-    values = torch.randint(-cfg.clip, cfg.clip + 1, (K, C, n), dtype=torch.int32, generator=gen)
-    tail = wl.gradients(cfg, seed, ct_first=last, n_cts=1)
-    values[:, last] = torch.from_numpy(tail[:, 0])
+    values = torch.from_numpy(wl.gradients(cfg, seed))
+    tail = values[:, last:last + 1].numpy()
     dv = values.to(dev)
     free_b, _ = torch.cuda.mem_get_info(dev)
     per_ct = ctx.round_workspace_bytes(1) - 256
@@ -862,6 +918,24 @@ def test_error_statuses(d2):
     assert status(ctx.combine_decrypt, agg, shares, 1, 2, 1, out) == d2.ERR_INVALID_ARG  # a share is missing
     misaligned = ctx.empty_u64(2 * L * n + 1)[1:]
     assert status(ctx.ntt_forward, misaligned, 1) == d2.ERR_INVALID_ARG
+    ctx.sync()
+    # the host-buffer round reports an out-of-range value itself (it returns after its own sync)
+    offsets, rows = wl.regular_graph(K, cfg.degree, 1)
+    ctx.keygen_share([3])
+    ctx.collective_pk([0, 1, 2, 3])
+    hv = torch.zeros((K, 1, n), dtype=torch.int32).pin_memory()
+    hs = torch.zeros((K, 1, n), dtype=torch.int32).pin_memory()
+    ws = torch.empty(ctx.round_workspace_bytes(1), dtype=torch.uint8, device=ctx.device)
+    ctx.round_host(hv, 0, 1, offsets, rows, hs, ws)
+    hv[1, 0, 5] = -(T - 1) // 2 - 1
+    assert status(ctx.round_host, hv, 0, 1, offsets, rows, hs, ws) == d2.ERR_RANGE
+    ctx.sync()  # the flag was cleared by the call that reported it
+    hv[1, 0, 5] = 0
+    ctx.round_host(hv, 0, 1, offsets, rows, hs, ws)
+    assert not hs.any()
+    # a run of more staged calls than the staging ring has slots keeps working (the fifth waits for the first)
+    for _ in range(9):
+        ctx.keygen_share([0])
     ctx.sync()
     big = d2.Context(15, wl.ntt_primes(54, 1 << 16, 1), 2, seed=1)
     assert status(big.keygen_share, [0]) == d2.ERR_UNSUPPORTED
