@@ -6,7 +6,7 @@ encode -> encrypt -> neighbour sums -> decryption shares -> combine (scale-and-r
 with every protocol message (ciphertexts, aggregates, shares) written to and read from HBM.
 Metric: gradient coefficients per second per full round = K * params / t_round.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 4] [--impl reference]
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same configuration on its
 own range of ciphertext indices; nothing is exchanged inside a round (weak scaling).
@@ -108,23 +108,25 @@ def algorithmic_bytes(cfg, n_cts):
 
 
 # Integer roofline of the transform-bearing kernels.  The scarce unit is the 32-bit integer
-# multiply-add pipe: 64 lanes per SM per clock (a widening or high-half multiply occupies it
-# for two passes).  Peak = 148 SMs x 64 lanes x 1.965 GHz (the documented SM count and maximum
-# SM clock) = 18.6e12 multiply-add slots per second; a register-only probe of the butterfly
-# reaches 96 % of it.  Algorithmic slots: one lazy Shoup butterfly = 5 widening/high + 3 low
-# multiplies = 13 slots (the primes of every configuration are 2^b - d with small d, which turns
-# a fourth low multiply into a shift); a transform = (N/2) log2 N butterflies; a pointwise
-# product = 14; one Philox4x32-10 call = 20 widening multiplies = 40 slots (one call serves all
-# L limbs).
+# multiply-add pipe.  Its rate is MEASURED in every run by the library's register-only loops
+# (d2mhe_debug_int_throughput: mad.lo.u32, mad.wide.u32, mad.hi.u32, and the engine's butterfly)
+# and the roofline's peak is the measured mad.lo rate in lane operations ("slots") per second;
+# 148 SMs x 64 lanes x 1.965 GHz (unit counts and maximum clock) is printed beside it.  A widening
+# or high-half multiply occupies the pipe for two slots (the measured rates say so).  Algorithmic
+# slots: one lazy Shoup butterfly = 5 widening/high + 3 low multiplies = 13 slots (the primes of
+# every configuration are 2^b - d with small d, which turns a fourth low multiply into a shift);
+# a transform = (N/2) log2 N butterflies; a pointwise product = 14; one Philox4x32-10 call = 20
+# widening multiplies = 40 slots (one call serves all L limbs).
 IMAD_LANES_PER_SM = 64
 NUM_SMS = 148
 SM_MAX_HZ = 1.965e9
-IMAD_PEAK = NUM_SMS * IMAD_LANES_PER_SM * SM_MAX_HZ
+IMAD_PEAK_UNIT_COUNTS = NUM_SMS * IMAD_LANES_PER_SM * SM_MAX_HZ
+SLOTS_PER_BUTTERFLY = 13
 
 
 def algorithmic_mad_slots(cfg, n_cts):
     K, S, L, n = cfg.num_parties, cfg.num_parties, cfg.num_limbs, cfg.n
-    transform = 13 * (n // 2) * cfg.log2_n   # slots per limb-transform
+    transform = SLOTS_PER_BUTTERFLY * (n // 2) * cfg.log2_n   # slots per limb-transform
     units = K * n_cts
     return {
         # NTT(u) + 2 inverse transforms, 2 pointwise products, Lambda*m (10 slots) per limb; 3 samples per coefficient
@@ -134,9 +136,34 @@ def algorithmic_mad_slots(cfg, n_cts):
     }
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures under profiles/
-# (null when the kernel has changed since the capture).
-NCU_TRAFFIC_BYTES = {("mnist-mlp-784-128-10-K10", "partial_decrypt"): 56150272 + 304640000}
+# dram__bytes_read.sum + dram__bytes_write.sum of the share kernel per (recipient, ciphertext) unit,
+# from the ncu captures under profiles/ (taken on a few ciphertext indices of the configuration and
+# scaled by the units of a launch: the traffic is the shares written plus c_1 and the noise bytes
+# read, all proportional to the units).  None when the kernel has changed since the capture.
+NCU_TRAFFIC_BYTES_PER_UNIT = {}
+
+
+def measure_int_peak(ctx):
+    """The integer rates of this GPU, measured now (lane operations per second)."""
+    lo = max(ctx.debug_int_throughput(0, 4096) for _ in range(3))
+    wide = max(ctx.debug_int_throughput(1, 4096) for _ in range(3))
+    hi = max(ctx.debug_int_throughput(2, 4096) for _ in range(3))
+    mul_wide = max(ctx.debug_int_throughput(4, 4096) for _ in range(3))
+    mul_hi = max(ctx.debug_int_throughput(5, 4096) for _ in range(3))
+    out = {"mad_lo_per_s": lo, "mad_wide_per_s": wide, "mad_hi_per_s": hi, "mul_wide_per_s": mul_wide,
+           "mul_hi_per_s": mul_hi,
+           "slots_per_mad_wide": lo / wide if wide else None, "slots_per_mad_hi": lo / hi if hi else None,
+           "slots_per_mul_wide": lo / mul_wide if mul_wide else None, "slots_per_mul_hi": lo / mul_hi if mul_hi else None,
+           "unit_count_peak_per_s": IMAD_PEAK_UNIT_COUNTS,
+           "mad_lo_warp_instr_per_clk_per_sm_at_max_clock": lo / 32 / NUM_SMS / SM_MAX_HZ}
+    try:
+        bf = max(ctx.debug_int_throughput(3, 2048) for _ in range(3))
+        out["butterflies_per_s_registers_only"] = bf
+        out["butterfly_loop_frac_of_peak"] = bf * SLOTS_PER_BUTTERFLY / lo
+        out["cycles_per_warp_butterfly_per_scheduler_at_max_clock"] = NUM_SMS * 4 * SM_MAX_HZ / (bf / 32)
+    except Exception:  # primes outside the form the probe's butterfly is written for
+        pass
+    return out
 
 
 # ----------------------------------------------------------------------------------
@@ -165,17 +192,30 @@ def oracle_round(cfg, seed, ct_first, n_cts, o=None, pk=None):
     return dt, sums, values, offsets, rows, o, pk
 
 
-def cpu_baseline(cfg, seed, budget_s=12.0):
+def coeffs_of(cfg, ct_first, n_cts):
+    """Gradient coefficients (of all K users) carried by ciphertext indices ct_first .. ct_first+n_cts-1."""
+    lo, hi = ct_first * cfg.n, min(cfg.params, (ct_first + n_cts) * cfg.n)
+    return cfg.num_parties * max(0, hi - lo)
+
+
+def cpu_baseline(cfg, seed, budget_s=15.0):
     """Times the oracle on as many ciphertext indices of the workload as fit the budget."""
     from oracle import d2mhe_oracle as orc
 
-    dt1, _, _, _, _, o, pk = oracle_round(cfg, seed, 0, 1)
-    n_cts = int(max(1, min(cfg.num_cts, budget_s / max(dt1, 1e-6))))
-    dt, sums, values, offsets, rows, _, _ = oracle_round(cfg, seed, 0, n_cts, o, pk)
-    coeffs = cfg.num_parties * min(cfg.params, n_cts * cfg.n)
-    return {"value": coeffs / dt, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
+    dt, _, _, _, _, o, pk = oracle_round(cfg, seed, 0, 1)
+    n_cts = 1
+    if dt < budget_s / 3:
+        n_cts = int(max(1, min(cfg.num_cts, budget_s / max(dt, 1e-6))))
+        dt, *_ = oracle_round(cfg, seed, 0, n_cts, o, pk)
+    return {"value": coeffs_of(cfg, 0, n_cts) / dt, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
             "sample": "ciphertext indices 0..%d of %d, all %d users and share holders, %.2f s"
                       % (n_cts - 1, cfg.num_cts, cfg.num_parties, dt)}
+
+
+def config_dict(cfg):
+    """The workload's description: the same keys and values in both arms."""
+    return {"workload": cfg.name, "K": cfg.num_parties, "N": cfg.n, "L": cfg.num_limbs,
+            "cts_per_user": cfg.num_cts, "params_per_user": cfg.params}
 
 
 def run_reference(args, cfg):
@@ -193,16 +233,14 @@ def run_reference(args, cfg):
     for _ in range(args.steps):
         dt, *_ = oracle_round(cfg, args.seed, 0, n_cts, o, pk)
         total += dt
-    coeffs = cfg.num_parties * min(cfg.params, n_cts * cfg.n)
-    value = coeffs * args.steps / total
+    value = coeffs_of(cfg, 0, n_cts) * args.steps / total
     sample = "each step: ciphertext indices 0..%d of %d, all %d users and share holders" % (
         n_cts - 1, cfg.num_cts, cfg.num_parties)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-        "config": {"workload": cfg.name, "K": cfg.num_parties, "N": cfg.n, "L": cfg.num_limbs,
-                   "cts_per_user": cfg.num_cts, "params_per_user": cfg.params},
+        "config": config_dict(cfg),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -215,21 +253,17 @@ def run_reference(args, cfg):
 # ----------------------------------------------------------------------------------
 
 
-def run_cuda(args, cfg):
+def measure_round(cfg, args, steps, warmup, rank, local_rank, world, detailed, sampler=None, n_cts=None):
+    """Times one configuration.  detailed: also the call-by-call pass (per-kernel durations), the
+    host-buffer pass (e2e) and the transform micro-benchmark.  n_cts: only the first n_cts
+    ciphertext indices of the workload (a labelled slice, for profiling)."""
     import torch
 
-    from paper_2207_04604_b200 import build, d2mhe, parallel
+    from paper_2207_04604_b200 import d2mhe, parallel
 
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
-    rank, local_rank, world = parallel.init()
-    torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if rank == 0:
-        build.build()
-    parallel.barrier(dev)
-
-    K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, cfg.num_cts
+    K, L, n = cfg.num_parties, cfg.num_limbs, cfg.n
+    C = cfg.num_cts if not n_cts else min(n_cts, cfg.num_cts)
     parties = list(range(K))
     offsets, rows = wl.regular_graph(K, cfg.degree, args.seed)
     ct_first, _ = wl.shard_ct_range(rank, world, C)  # each rank: its own C ciphertext indices
@@ -244,20 +278,24 @@ def run_cuda(args, cfg):
     ev1.record(stream)
     ctx.sync()
     init_ms = ev0.elapsed_time(ev1)
+    int_peak = measure_int_peak(ctx) if detailed and rank == 0 else None
 
-    # chunking: keep all protocol messages of a chunk in HBM at once (the workspace of the whole-round
-    # call and the buffers of the call-by-call pass exist side by side)
-    free_b, _ = torch.cuda.mem_get_info(dev)
-    per_ct = ctx.round_workspace_bytes(1) - 256
-    chunk = int(max(1, min(C, (int(free_b * 0.35)) // per_ct)))
-    if args.chunk:
-        chunk = min(chunk, args.chunk)
     values_np = wl.gradients(cfg, args.seed, ct_first, C)
     values = torch.from_numpy(values_np).to(dev)
     sums = torch.empty((K, C, n), dtype=torch.int32, device=dev)
+    # chunking: keep all protocol messages of the sub-chunks in flight in HBM at once
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    per_ct = ctx.round_workspace_bytes(1) - 256
+    chunk = int(max(1, min(C, (int(free_b * 0.6)) // per_ct)))
+    if args.chunk:
+        chunk = min(chunk, args.chunk)
     ws = torch.empty(ctx.round_workspace_bytes(chunk), dtype=torch.uint8, device=dev)
     flush = torch.empty(384 * 1024 * 1024, dtype=torch.uint8, device=dev)  # > 126 MB L2
-    want = np.stack([values_np[rows[offsets[i]:offsets[i + 1]]].astype(np.int64).sum(axis=0) for i in range(K)])
+    idx = [torch.as_tensor(rows[offsets[i]:offsets[i + 1]].astype(np.int64), device=dev) for i in range(K)]
+
+    def sums_are_right(t):
+        """Every decrypted sum equals the plaintext neighbour sum (checked on the device)."""
+        return all(bool(torch.equal(t[i], values[idx[i]].sum(dim=0, dtype=torch.int32))) for i in range(K))
 
     def barrier():
         parallel.barrier(dev)
@@ -266,22 +304,20 @@ def run_cuda(args, cfg):
     def step():
         ctx.round_device(values, ct_first, C, offsets, rows, sums, ws)
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         flush.zero_()
         step()
     barrier()
-    # correctness of what is being timed: every decrypted sum equals the plaintext neighbour sum
-    if not np.array_equal(sums.cpu().numpy(), want):
+    if not sums_are_right(sums):
         raise RuntimeError("decrypted neighbour sums differ from the plaintext sums")
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
+    if sampler is not None:
         sampler.start()
     launches0 = ctx.launch_count()
     step_events = []
     barrier()
     wall0 = time.perf_counter()
-    for _ in range(args.steps):
+    for _ in range(steps):
         flush.zero_()  # evict the previous step's messages from L2 (outside the timed events)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
@@ -291,21 +327,33 @@ def run_cuda(args, cfg):
     barrier()
     wall = time.perf_counter() - wall0
     launches = ctx.launch_count() - launches0
-    step_ms = sum(a.elapsed_time(b) for a, b in step_events) / args.steps
+    step_ms = sum(a.elapsed_time(b) for a, b in step_events) / steps
     step_ms_max = parallel.max_over_ranks(step_ms, dev)
-    coeffs_per_step = world * K * cfg.params
-    value = coeffs_per_step / (step_ms_max * 1e-3)
+    coeffs_per_step = world * coeffs_of(cfg, 0, C)
+    res = {"cfg": cfg, "C": C, "chunk": chunk, "ms_per_step": step_ms_max, "value": coeffs_per_step / (step_ms_max * 1e-3),
+           "launches": int(launches), "init_ms": init_ms, "wall_ms_per_step_incl_flush": wall * 1e3 / steps,
+           "int_peak": int_peak, "sub_chunks": d2mhe.round_plan(C, chunk)[0]}
+    if not detailed:
+        if sampler is not None:
+            res["clocks"] = sampler.stop()
+        ctx.close()
+        return res
 
     # ---- the same round call by call on one stream, with an event between the calls: each kernel's
     # launch duration (nothing overlaps here), its share of the step and the roofline entry ----
+    # The three large message buffers of this pass are views of the round call's workspace (the two
+    # passes never run at the same time); the ragged last chunk uses the same storage.
     def alloc(cc):
+        n_ct, n_sh = K * cc * 2 * L * n, K * K * cc * L * n
+        words = ws[:8 * (2 * n_ct + n_sh)].view(torch.int64)
         return (torch.empty((K, cc, n), dtype=torch.int32, device=dev), ctx.empty_u32(K, cc, n),
-                ctx.empty_u64(K, cc, 2, L, n), ctx.empty_u64(K, cc, 2, L, n), ctx.empty_u64(K, K, cc, L, n),
+                words[:n_ct].view(K, cc, 2, L, n), words[n_ct:2 * n_ct].view(K, cc, 2, L, n),
+                words[2 * n_ct:].view(K, K, cc, L, n),
                 ctx.empty_u32(K, cc, n), torch.empty((K, cc, n), dtype=torch.int32, device=dev))
 
     bufs = {chunk: alloc(chunk)}
     if C % chunk:
-        bufs[C % chunk] = alloc(C % chunk)  # the ragged last chunk has buffers of its own size
+        bufs[C % chunk] = alloc(C % chunk)
 
     def serial_step(events=None):
         for first in range(0, C, chunk):
@@ -337,12 +385,13 @@ def run_cuda(args, cfg):
             if events is not None:
                 events.append(marks)
 
-    serial_steps = max(3, min(args.steps, 50))
+    long_step = step_ms_max > 500.0  # seconds-long rounds: a few steps per extra pass are enough
+    serial_steps = 2 if long_step else max(3, min(steps, 50))
     sums.zero_()
-    for _ in range(min(args.warmup, 3)):
+    for _ in range(1 if long_step else min(warmup, 3)):
         flush.zero_()
         serial_step()
-    if not np.array_equal(sums.cpu().numpy(), want):
+    if not sums_are_right(sums):
         raise RuntimeError("call-by-call round differs from the plaintext sums")
     chunk_events, serial_events = [], []
     for _ in range(serial_steps):
@@ -353,24 +402,26 @@ def run_cuda(args, cfg):
         e1.record(stream)
         serial_events.append((e0, e1))
     torch.cuda.synchronize(dev)
-    clocks = sampler.stop() if rank == 0 else None
-    serial_ms = sum(a.elapsed_time(b) for a, b in serial_events) / serial_steps
+    if sampler is not None:
+        res["clocks"] = sampler.stop()
+    res["serial_ms"] = sum(a.elapsed_time(b) for a, b in serial_events) / serial_steps
     per_call = {name: 0.0 for name in STEP_CALLS}
     for marks in chunk_events:
         for i, name in enumerate(STEP_CALLS):
             per_call[name] += marks[i].elapsed_time(marks[i + 1])
-    n_chunks_total = len(chunk_events)
+    res.update(per_call=per_call, serial_steps=serial_steps, n_chunks_total=len(chunk_events))
     bufs.clear()
     torch.cuda.empty_cache()
 
     # end to end through the host-buffer entry point: H2D of the gradients, the round, D2H of the sums
     hv = torch.from_numpy(values_np).pin_memory()
     hs = torch.zeros((K, C, n), dtype=torch.int32).pin_memory()
-    for _ in range(2):
+    for _ in range(1 if long_step else 2):
         ctx.round_host(hv, ct_first, C, offsets, rows, hs, ws)
-    if not np.array_equal(hs.numpy(), want):
+    sums.copy_(hs)
+    if not sums_are_right(sums):
         raise RuntimeError("host-buffer round differs from the plaintext sums")
-    e2e_steps = max(3, min(args.steps, 50))
+    e2e_steps = 3 if long_step else max(3, min(steps, 50))
     barrier()
     e2e_total, e2e_each = 0.0, []
     for _ in range(e2e_steps):
@@ -381,107 +432,173 @@ def run_cuda(args, cfg):
         e2e_each.append(time.perf_counter() - t0)
         e2e_total += e2e_each[-1]
     barrier()
-    e2e_ms = e2e_total * 1e3 / e2e_steps
-    e2e_ms_max = parallel.max_over_ranks(e2e_ms, dev)
-    e2e_value = coeffs_per_step / (e2e_ms_max * 1e-3)
+    e2e_ms_max = parallel.max_over_ranks(e2e_total * 1e3 / e2e_steps, dev)
+    res["e2e"] = {"value": coeffs_per_step / (e2e_ms_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": K * C * n * 4,
+                  "d2h_bytes_per_step": K * C * n * 4, "ms_per_step": e2e_ms_max,
+                  "ms_per_step_median": float(np.median(e2e_each)) * 1e3, "steps": e2e_steps}
+    del hv, hs
 
     # transform / multiply-add micro-benchmark on this configuration's ring (batch > L2)
-    ntt = None
     if rank == 0:
         del ws
         torch.cuda.empty_cache()
-        batch = max(1, (384 << 20) // (8 * n * L))
-        polys = torch.randint(0, min(cfg.moduli), (batch, L, n), dtype=torch.int64, device=dev)
-        other = polys.clone()
-        third = polys.clone()
-        res = torch.empty_like(polys)
+        res["ntt"] = ntt_microbench(ctx, cfg, dev, stream, flush)
+    ctx.close()
+    return res
 
-        def timed(fn, reps=5):
+
+def ntt_microbench(ctx, cfg, dev, stream, flush):
+    import torch
+
+    L, n = cfg.num_limbs, cfg.n
+    batch = max(1, (384 << 20) // (8 * n * L))
+    polys = torch.randint(0, min(cfg.moduli), (batch, L, n), dtype=torch.int64, device=dev)
+    other, third, out = polys.clone(), polys.clone(), torch.empty_like(polys)
+
+    def timed(fn, reps=5):
+        fn()
+        best = None
+        for _ in range(reps):
+            flush.zero_()
+            a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a_.record(stream)
             fn()
-            best = None
-            for _ in range(reps):
-                flush.zero_()
-                a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a_.record(stream)
-                fn()
-                b_.record(stream)
-                torch.cuda.synchronize(dev)
-                ms = a_.elapsed_time(b_)
-                best = ms if best is None else min(best, ms)
-            return best
+            b_.record(stream)
+            torch.cuda.synchronize(dev)
+            ms = a_.elapsed_time(b_)
+            best = ms if best is None else min(best, ms)
+        return best
 
-        nbytes = 16.0 * n * L * batch
-        f_ms = timed(lambda: ctx.ntt_forward(polys, batch))
-        i_ms = timed(lambda: ctx.ntt_inverse(polys, batch))
-        m_ms = timed(lambda: ctx.poly_muladd(polys, other, third, res, batch))
-        ntt = {"shape": [batch, L, n], "forward_GBps": nbytes / 1e9 / (f_ms * 1e-3),
-               "inverse_GBps": nbytes / 1e9 / (i_ms * 1e-3), "muladd_GBps": 2 * nbytes / 1e9 / (m_ms * 1e-3),
-               "bytes_per_coeff": {"ntt": 16, "muladd": 32}}
-        del polys, other, third, res
+    nbytes = 16.0 * n * L * batch
+    f_ms = timed(lambda: ctx.ntt_forward(polys, batch))
+    i_ms = timed(lambda: ctx.ntt_inverse(polys, batch))
+    m_ms = timed(lambda: ctx.poly_muladd(polys, other, third, out, batch))
+    bfly = batch * L * (n // 2) * cfg.log2_n
+    return {"shape": [batch, L, n], "forward_GBps": nbytes / 1e9 / (f_ms * 1e-3),
+            "inverse_GBps": nbytes / 1e9 / (i_ms * 1e-3), "muladd_GBps": 2 * nbytes / 1e9 / (m_ms * 1e-3),
+            "forward_butterflies_per_s": bfly / (f_ms * 1e-3), "inverse_butterflies_per_s": bfly / (i_ms * 1e-3),
+            "bytes_per_coeff": {"ntt": 16, "muladd": 32}}
+
+
+def run_cuda(args, cfg):
+    import torch
+
+    from paper_2207_04604_b200 import build, parallel
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    rank, local_rank, world = parallel.init()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if rank == 0:
+        build.build()
+    parallel.barrier(dev)
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    res = measure_round(cfg, args, args.steps, args.warmup, rank, local_rank, world, True, sampler, args.cts)
+    others = {}
+    if rank == 0 and world == 1 and not args.no_other_configs and not args.cts:
+        # the smaller round configurations, one short pass each (device-resident value only)
+        for i in (1, 2, 3):
+            c2 = wl.round_config(i)
+            if c2.name == cfg.name:
+                continue
+            torch.cuda.empty_cache()
+            r2 = measure_round(c2, args, 10, 3, 0, local_rank, 1, False)
+            others[c2.name] = {"config": config_dict(c2), "ms_per_step": r2["ms_per_step"], "value": r2["value"],
+                               "unit": UNIT, "steps": 10, "warmup": 3, "sub_chunks": r2["sub_chunks"],
+                               "round_hbm_frac": sum(algorithmic_bytes(c2, c2.num_cts).values()) / 1e9
+                               / (r2["ms_per_step"] * 1e-3) / measured_peaks()[0]}
 
     if rank == 0:
+        K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, res["C"]
         peak, peak_kind = measured_peaks()
+        clocks = res.get("clocks") or {}
+        mhz = clocks.get("sm_mhz")
+        ip = res["int_peak"]
+        imad_peak = ip["mad_lo_per_s"]
+
+        def mcycles(ms):  # duration x median sampled SM clock: comparable across clock states
+            return ms * mhz * 1e-3 if (mhz and ms is not None) else None
+
         ab = algorithmic_bytes(cfg, C)
-        for k_ in ("forward_GBps", "inverse_GBps", "muladd_GBps"):
-            ntt[k_.replace("GBps", "frac_of_hbm")] = ntt[k_] / peak
+        per_call, serial_steps, n_chunks_total = res["per_call"], res["serial_steps"], res["n_chunks_total"]
         total_ms = sum(per_call.values())
+        slots = algorithmic_mad_slots(cfg, C)
+        ntt = res["ntt"]
+        for k_ in ("forward", "inverse", "muladd"):
+            ntt[k_ + "_frac_of_hbm"] = ntt[k_ + "_GBps"] / peak
+        for k_ in ("forward", "inverse"):
+            ntt[k_ + "_alu_frac"] = ntt[k_ + "_butterflies_per_s"] * SLOTS_PER_BUTTERFLY / imad_peak
         kernels = {}
         for name in STEP_CALLS:
             ms = per_call[name] / serial_steps  # per step, summed over chunks
-            kernels[name] = {"ms_per_step": ms, "share": per_call[name] / total_ms if total_ms else None,
-                             "algorithmic_GB": ab[name] / 1e9, "GBps": ab[name] / 1e9 / (ms * 1e-3) if ms else None}
+            kernels[name] = {"ms_per_step": ms, "mcycles_per_step": mcycles(ms),
+                             "share": per_call[name] / total_ms if total_ms else None,
+                             "algorithmic_GB": ab[name] / 1e9, "GBps": ab[name] / 1e9 / (ms * 1e-3) if ms else None,
+                             "hbm_frac": ab[name] / 1e9 / (ms * 1e-3) / peak if ms else None}
+            if name in slots:
+                kernels[name]["alu_frac"] = slots[name] / (ms * 1e-3) / imad_peak if ms else None
+        kernels["aggregate"]["note"] = ("algorithmic bytes count every list's read of a ciphertext; the ciphertexts were "
+                                        "just written and most of those reads hit L2, so this is not a DRAM roofline fraction")
         dominant = max(STEP_CALLS, key=lambda k_: per_call[k_])
-        launches_dom = n_chunks_total
-        dur_ms = per_call[dominant] / launches_dom
-        bytes_per_launch = ab[dominant] / (n_chunks_total / serial_steps)
-        achieved = bytes_per_launch / 1e9 / (dur_ms * 1e-3)
-        traffic = NCU_TRAFFIC_BYTES.get((cfg.name, dominant))
-        slots = algorithmic_mad_slots(cfg, C)
+        chunks_per_step = n_chunks_total / serial_steps
+        dur_ms = per_call[dominant] / n_chunks_total
+        units_per_launch = K * C / chunks_per_step
+        achieved = ab[dominant] / chunks_per_step / 1e9 / (dur_ms * 1e-3)
+        per_unit = NCU_TRAFFIC_BYTES_PER_UNIT.get((cfg.name, dominant))
+        traffic = per_unit * units_per_launch if per_unit else None
         if dominant in slots:  # transform-bearing kernel: bound by the integer multiply-add pipe
-            slots_per_launch = slots[dominant] / (n_chunks_total / serial_steps)
-            got = slots_per_launch / (dur_ms * 1e-3)
-            roofline = {"bound": "alu", "kernel": dominant, "achieved": got / 1e12, "peak": IMAD_PEAK / 1e12,
-                        "unit": "T int32 multiply-add slots/s", "frac": got / IMAD_PEAK,
-                        "peak_source": "148 SMs x 64 lanes x 1.965 GHz (unit counts and clocks)",
-                        "traffic": traffic, "avg_launch_ms": dur_ms,
+            got = slots[dominant] / chunks_per_step / (dur_ms * 1e-3)
+            roofline = {"bound": "alu", "kernel": dominant, "achieved": got / 1e12, "peak": imad_peak / 1e12,
+                        "unit": "T int32 multiply-add slots/s", "frac": got / imad_peak,
+                        "peak_source": "measured in this run: mad.lo.u32 lane operations/s of a register-only loop on "
+                                       "all SMs (d2mhe_debug_int_throughput); unit counts x maximum clock give %.2f"
+                                       % (IMAD_PEAK_UNIT_COUNTS / 1e12),
+                        "frac_of_unit_count_peak": got / IMAD_PEAK_UNIT_COUNTS,
+                        "traffic": traffic, "avg_launch_ms": dur_ms, "avg_launch_mcycles": mcycles(dur_ms),
+                        "units_per_launch": units_per_launch,
                         "launches_note": "one call = the sampling kernel (about 5 % of the time) followed by the "
-                                         "transform kernel; traffic is the transform kernel's",
+                                         "transform kernel; traffic is the transform kernel's, scaled from a capture "
+                                         "of a few ciphertext indices by the (recipient, ciphertext) units of a launch",
                         "hbm": {"achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                                 "peak_source": "of " + peak_kind}}
         else:
             roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                         "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": traffic,
                         "avg_launch_ms": dur_ms}
-        for name in slots:
-            ms = kernels[name]["ms_per_step"]
-            kernels[name]["alu_frac"] = slots[name] / (ms * 1e-3) / IMAD_PEAK if ms else None
         round_bytes = sum(ab.values())
+        config = config_dict(cfg)
+        if args.cts:
+            config["slice"] = "first %d ciphertext indices only (profiling run, not the benchmark)" % C
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": step_ms_max, "higher_is_better": True, "scaling": "weak",
+            "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "mcycles_per_step": mcycles(res["ms_per_step"]),
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-            "config": {"workload": cfg.name, "K": K, "N": n, "L": L, "cts_per_user": C, "params_per_user": cfg.params,
-                       "graph_degree": cfg.degree, "share_holders": K, "chunk_cts": chunk,
+            "config": config,
+            "launch": {"graph_degree": cfg.degree, "share_holders": K, "chunk_cts": res["chunk"],
+                       "sub_chunks": res["sub_chunks"],
                        "entry_point": "d2mhe_round_device (sub-chunks overlapped on two internal streams)",
                        "l2": "384 MB buffer written between timed steps (L2 flush)",
                        "parallelism": "ciphertext-index shards, no exchange" if world > 1 else "single GPU"},
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": K * C * n * 4,
-                    "d2h_bytes_per_step": K * C * n * 4, "ms_per_step": e2e_ms_max,
-                    "ms_per_step_median": float(np.median(e2e_each)) * 1e3, "steps": e2e_steps},
-            "gpu_launches": int(launches),
+            "e2e": res["e2e"],
+            "gpu_launches": res["launches"],
             "roofline": roofline,
-            "round_hbm_frac": round_bytes / 1e9 / (step_ms_max * 1e-3) / peak,
-            "ms_per_step_call_by_call": serial_ms,
-            "kernels_note": "per-call durations from a separate pass of the same round, call by call on one stream",
+            "integer_peak": ip,
+            "round_hbm_frac": round_bytes / 1e9 / (res["ms_per_step"] * 1e-3) / peak,
+            "ms_per_step_call_by_call": res["serial_ms"],
+            "kernels_note": "per-call durations from a separate pass of the same round, call by call on one stream; "
+                            "mcycles = duration x median sampled SM clock",
             "kernels": kernels,
             "ntt": ntt,
-            "init_ms": init_ms,
-            "wall_ms_per_step_incl_flush": wall * 1e3 / args.steps,
+            "other_configs": others,
+            "init_ms": res["init_ms"],
+            "wall_ms_per_step_incl_flush": res["wall_ms_per_step_incl_flush"],
             "cpu_baseline": cpu_baseline(cfg, args.seed) if world == 1 and not args.no_cpu_baseline else None,
         }
         print(json.dumps(line))
-    ctx.close()
     parallel.finish()
 
 
@@ -569,13 +686,18 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--config", type=int, default=2, help="round configuration 1..4 (default 2: MNIST-shaped); 5 = kernel sweep")
+    ap.add_argument("--config", type=int, default=4,
+                    help="round configuration 1..4 (default 4: ResNet-18-shaped, the largest one); 5 = kernel sweep")
     ap.add_argument("--seed", type=int, default=1)
     ap.add_argument("--chunk", type=int, default=0, help="ciphertext indices per chunk (0: as many as fit)")
+    ap.add_argument("--cts", type=int, default=0,
+                    help="run only the first CTS ciphertext indices of the workload (a labelled slice, for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the short passes over the other round configurations")
     ap.add_argument("--sweep-bits", type=int, default=60, choices=[30, 50, 60])
     ap.add_argument("--sweep-point", default="", help="N,L,batch: run this one point of the sweep (any batch)")
     args = ap.parse_args()

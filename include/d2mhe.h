@@ -321,6 +321,18 @@ d2mhe_status d2mhe_round_device_static(d2mhe_ctx* ctx, const int32_t* values_dev
 d2mhe_status d2mhe_debug_export_secret(d2mhe_ctx* ctx, uint32_t party, int8_t* s_host);
 /* The same for sk_i of a user's own key pair (needs d2mhe_user_keygen for `user`). */
 d2mhe_status d2mhe_debug_export_user_secret(d2mhe_ctx* ctx, uint32_t user, int8_t* s_host);
+/* Measurement hook for the integer roofline of the transform kernels (Sec. 3.2 / 4.2: the ring
+ * products are where the time goes): runs a loop on registers only that fills every SM (2048
+ * resident threads, eight independent chains per thread, no memory traffic) for `iters`
+ * iterations and reports lane operations per second, timed with CUDA events on the context's
+ * stream (the call synchronises).  kind 0: mad.lo.u32, 1: mad.wide.u32 with a 64-bit addend,
+ * 2: mad.hi.u32 (32 lane operations per warp instruction), 3: the engine's forward butterfly on
+ * eight coefficients per thread (operations = butterflies; needs a parameter set whose primes
+ * are all below 2^57 and of the form 2^b - d, else D2MHE_ERR_UNSUPPORTED), 4: mul.wide.u32,
+ * 5: mul.hi.u32 (both without an addend), 6: mad.wide.u32 with a loop-invariant addend.
+ * 1 <= iters <= 2^24. */
+d2mhe_status d2mhe_debug_int_throughput(d2mhe_ctx* ctx, uint32_t kind, uint32_t iters,
+                                        double* ops_per_second);
 /* The primitive 2N-th root of unity used for limb `limb`. */
 d2mhe_status d2mhe_get_root(const d2mhe_ctx* ctx, uint32_t limb, uint64_t* psi);
 /* psi_t, the slot root (D2MHE_ERR_UNSUPPORTED if t != 1 mod 2N). */

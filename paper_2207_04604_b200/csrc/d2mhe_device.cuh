@@ -204,6 +204,11 @@ __device__ __forceinline__ u32 mulhi32(u32 a, u32 b) {
   asm("mul.hi.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
   return r;
 }
+__device__ __forceinline__ u32 madhi32(u32 a, u32 b, u32 c) {  // hi32(a b) + c, wrapping
+  u32 r;
+  asm("mad.hi.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
 __device__ __forceinline__ void split64(u64 x, u32& lo, u32& hi) {
   asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(x));
 }
@@ -238,7 +243,10 @@ __device__ __forceinline__ u64 shoup_approx_sf(u64 y, u64 w, u64 ws, u32 d, u32 
   split64(ws, sl, sh);
   split64(w, wl, wh);
   // the two high halves are summed first: the 64-bit sum is a register pair that the widening
-  // multiply-add takes as it is (a zero-extended single word would need a move)
+  // multiply-add takes as it is (a zero-extended single word would need a move).  Measured on this
+  // GPU, in units of one mad.lo.u32: mul.hi 2.0, mul.wide 2.2, mad.hi 2.2, mad.wide with its 64-bit
+  // addend 2.8.  Splitting either widening multiply-add into mul.wide plus a 64-bit addition on the
+  // other integer pipe, or taking the high halves from mul.wide, made the butterfly 2-10 % slower.
   const u64 q = madwide(yh, sh, (u64)mulhi32(yh, sl) + (u64)mulhi32(yl, sh));
   u32 ql, qh, rl, rh;
   split64(q, ql, qh);

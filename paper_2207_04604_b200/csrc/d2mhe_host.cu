@@ -1155,6 +1155,22 @@ d2mhe_status d2mhe_debug_export_user_secret(d2mhe_ctx* c, u32 user, int8_t* s_ho
   return export_key(c, c->view.usk_mont + (size_t)user * c->view.L * c->view.n, s_host);
 }
 
+d2mhe_status d2mhe_debug_int_throughput(d2mhe_ctx* c, u32 kind, u32 iters, double* ops_per_second) {
+  if (!c || !ops_per_second || kind > 6 || iters == 0 || iters > (1u << 24)) return D2MHE_ERR_INVALID_ARG;
+  if (kind == 3 && !c->view.wide) return D2MHE_ERR_UNSUPPORTED;
+  DeviceGuard guard(c->device);
+  float ms = 0.f;
+  double ops = 0.0;
+  // the loops never store (their store is guarded by a condition that does not occur); the sink is
+  // the context's scratch all the same
+  cudaError_t e = L_(int_probe)(c->view, c->limb_params, c->stream, kind, iters,
+                                reinterpret_cast<u32*>(c->noise_scratch), &ms, &ops);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 2;
+  *ops_per_second = ms > 0.f ? ops / (ms * 1e-3) : 0.0;
+  return D2MHE_OK;
+}
+
 d2mhe_status d2mhe_get_root(const d2mhe_ctx* c, u32 limb, uint64_t* psi) {
   if (!c || !psi) return D2MHE_ERR_INVALID_ARG;
   if (limb >= c->params.num_limbs) return D2MHE_ERR_RANGE;

@@ -109,6 +109,9 @@ namespace d2mhe_launch {
 cudaError_t keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties);
 cudaError_t collective_pk(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
                           u64* shares_out);
+// measurement hook: register-only integer loops (kern_probe.cu); synchronises the stream
+cudaError_t int_probe(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 kind, u32 iters, u32* sink,
+                      float* ms, double* lane_ops);
 // test hook: key rows [L][N] (transform domain, Montgomery form) -> int8 coefficients [L][N] (127 = not ternary)
 cudaError_t export_secret(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* key, signed char* out);
 cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain);

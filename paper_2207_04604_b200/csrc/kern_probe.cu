@@ -1,0 +1,116 @@
+// Measurement hook: what the integer pipes of this GPU deliver, in the units the integer roofline
+// of the transform kernels is counted in.  Four loops on registers only (no memory traffic), every
+// SM filled with 2048 resident threads, eight independent chains per thread:
+//   kind 0  mad.lo.u32        one multiply-add slot per lane and instruction
+//   kind 1  mad.wide.u32      (64-bit addend)
+//   kind 2  mad.hi.u32
+//   kind 3  the forward butterfly of the engine (lazy Shoup product with the approximate
+//           quotient, primes 2^b - d) on eight coefficients per thread: four butterflies per pass
+//   kind 4  mul.wide.u32      (no addend)
+//   kind 5  mul.hi.u32        (no addend)
+//   kind 6  mad.wide.u32      with a loop-invariant 64-bit addend (the chain runs through a factor)
+#include "d2mhe_kernels_common.cuh"
+
+namespace {
+
+template <int KIND>
+__global__ void __launch_bounds__(256, 8) k_int_probe(u32 iters, u32 a0, u32 b0, u32* __restrict__ sink) {
+  u32 x[8];
+  u64 y[8];
+  const u32 t = blockIdx.x * blockDim.x + threadIdx.x;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    x[k] = t * 2654435761u + (u32)k * 40503u + a0;
+    y[k] = ((u64)x[k] << 32) | (t + (u32)k);
+  }
+  const u32 a = a0 | 1u, b = b0 | 3u;
+  const u64 c64 = ((u64)b0 << 32) | a0;
+#pragma unroll 1
+  for (u32 i = 0; i < iters; ++i) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (KIND == 0) x[k] = madlo(x[k], a, b);
+        if (KIND == 1) y[k] = madwide((u32)y[k], a, y[k]);
+        if (KIND == 2) x[k] = madhi32(x[k], a, b);
+        if (KIND == 4) y[k] = mulwide((u32)(y[k] >> 32) | 1u, a);
+        if (KIND == 5) x[k] = mulhi32(x[k] | 0x80000000u, a | 0x80000000u);
+        if (KIND == 6) y[k] = madwide((u32)(y[k] >> 32), a, c64);
+      }
+    }
+  }
+  u32 acc = 0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) acc ^= x[k] ^ (u32)y[k] ^ (u32)(y[k] >> 32);
+  if (acc == 0x9e3779b9u && iters == 0xffffffffu) sink[t] = acc;  // keeps the chains alive; never taken in practice
+}
+
+__global__ void __launch_bounds__(256, 4)
+    k_bfly_probe(const __grid_constant__ LimbParams lp, u32 iters, u32* __restrict__ sink) {
+  const LimbTab& lt = lp.limbs[0];
+  const Mod md(lt);
+  const u32 t = blockIdx.x * blockDim.x + threadIdx.x;
+  u64 x[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) x[k] = ((u64)(t * 2654435761u + (u32)k) << 20) % lt.p;
+  const ulonglong2 w = make_ulonglong2(lt.delta, lt.delta_sh);  // any residue with its Shoup companion
+  // The values grow past the lazy range after a few passes and wrap mod 2^64: the butterfly has no
+  // data-dependent branch, so its timing does not depend on them (the results mean nothing).
+#pragma unroll 1
+  for (u32 i = 0; i < iters; ++i) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) ct_bfly<MODE_WIDE>(x[k], x[k + 4], w, md);
+  }
+  u64 acc = 0;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) acc ^= x[k];
+  if (acc == 0x9e3779b97f4a7c15ull && iters == 0xffffffffu) sink[t] = (u32)acc;
+}
+
+}  // namespace
+
+namespace d2mhe_launch {
+
+// Runs the loop `kind` for `iters` iterations between two events on stream s and returns the
+// elapsed milliseconds and the number of lane operations (kind 0-2: multiply instructions x 32
+// lanes; kind 3: butterflies) that the launch executed.  Synchronises the stream.
+cudaError_t int_probe(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 kind, u32 iters, u32* sink,
+                      float* ms, double* lane_ops) {
+  (void)v;
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  cudaEvent_t e0, e1;
+  if ((e = cudaEventCreate(&e0)) != cudaSuccess) return e;
+  if ((e = cudaEventCreate(&e1)) != cudaSuccess) {
+    cudaEventDestroy(e0);
+    return e;
+  }
+  const u32 grid = (u32)sms * (kind == 3 ? 4u : 8u);
+  for (int pass = 0; pass < 2 && e == cudaSuccess; ++pass) {  // the first pass warms up
+    e = cudaEventRecord(e0, s);
+    if (e != cudaSuccess) break;
+    switch (kind) {
+      case 0: k_int_probe<0><<<grid, 256, 0, s>>>(iters, 12345u, 777u, sink); break;
+      case 1: k_int_probe<1><<<grid, 256, 0, s>>>(iters, 12345u, 777u, sink); break;
+      case 2: k_int_probe<2><<<grid, 256, 0, s>>>(iters, 12345u, 777u, sink); break;
+      case 4: k_int_probe<4><<<grid, 256, 0, s>>>(iters, 12345u, 777u, sink); break;
+      case 5: k_int_probe<5><<<grid, 256, 0, s>>>(iters, 12345u, 777u, sink); break;
+      case 6: k_int_probe<6><<<grid, 256, 0, s>>>(iters, 12345u, 777u, sink); break;
+      default: k_bfly_probe<<<grid, 256, 0, s>>>(lp, iters, sink); break;
+    }
+    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaEventRecord(e1, s);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+  }
+  if (e == cudaSuccess) e = cudaEventElapsedTime(ms, e0, e1);
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  const double threads = (double)grid * 256.0;
+  *lane_ops = kind == 3 ? threads * 4.0 * iters : threads * 32.0 * iters;
+  return e;
+}
+
+}  // namespace d2mhe_launch

@@ -31,7 +31,7 @@ EXPORTS = [
     "d2mhe_ntt_inverse", "d2mhe_poly_muladd", "d2mhe_ntt32_forward", "d2mhe_ntt32_inverse",
     "d2mhe_poly_muladd32", "d2mhe_round_workspace_bytes", "d2mhe_round_plan", "d2mhe_round_device",
     "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_user_keygen", "d2mhe_convert_share",
-    "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_bootstrap_share", "d2mhe_bootstrap_combine", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_get_root", "d2mhe_get_plain_root",
+    "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_bootstrap_share", "d2mhe_bootstrap_combine", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_debug_int_throughput", "d2mhe_get_root", "d2mhe_get_plain_root",
     "d2mhe_launch_count",
 ]
 
@@ -106,6 +106,7 @@ def load():
         lib.d2mhe_decrypt.argtypes = [vp, vp, u32, vp, u32, vp, vp]
         lib.d2mhe_bootstrap_share.argtypes = [vp, vp, vp, u32, vp, u32, u32, u32, vp]
         lib.d2mhe_bootstrap_combine.argtypes = [vp, vp, vp, vp, u32, u32, u32, u32, vp, vp]
+        lib.d2mhe_debug_int_throughput.argtypes = [vp, u32, u32, ctypes.POINTER(ctypes.c_double)]
         lib.d2mhe_get_root.argtypes = [vp, u32, ctypes.POINTER(u64)]
         lib.d2mhe_get_plain_root.argtypes = [vp, ctypes.POINTER(u64)]
         lib.d2mhe_launch_count.argtypes = [vp]
@@ -339,6 +340,13 @@ class Context:
         self._check(load().d2mhe_debug_export_secret(self._h, party, out.ctypes.data_as(ctypes.c_void_p)),
                     "d2mhe_debug_export_secret")
         return out
+
+    def debug_int_throughput(self, kind, iters):
+        """Lane operations per second of a register-only integer loop: d2mhe_debug_int_throughput."""
+        v = ctypes.c_double()
+        self._check(load().d2mhe_debug_int_throughput(self._h, kind, iters, ctypes.byref(v)),
+                    "d2mhe_debug_int_throughput")
+        return float(v.value)
 
     def get_root(self, limb):
         v = ctypes.c_uint64()
