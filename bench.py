@@ -438,11 +438,14 @@ def measure_round(cfg, args, steps, warmup, rank, local_rank, world, detailed, s
                   "ms_per_step_median": float(np.median(e2e_each)) * 1e3, "steps": e2e_steps}
     del hv, hs
 
-    # transform / multiply-add micro-benchmark on this configuration's ring (batch > L2)
+    # transform / multiply-add micro-benchmark on this configuration's ring (batch > L2), and the
+    # conversion / refresh calls (the paper's own decryption path and its bootstrap) on a few indices
     if rank == 0:
         del ws
         torch.cuda.empty_cache()
         res["ntt"] = ntt_microbench(ctx, cfg, dev, stream, flush)
+        torch.cuda.empty_cache()
+        res["convert_bootstrap"] = convert_bootstrap_bench(ctx, cfg, dev, stream, flush, offsets, rows, args.seed)
     ctx.close()
     return res
 
@@ -478,6 +481,77 @@ def ntt_microbench(ctx, cfg, dev, stream, flush):
             "inverse_GBps": nbytes / 1e9 / (i_ms * 1e-3), "muladd_GBps": 2 * nbytes / 1e9 / (m_ms * 1e-3),
             "forward_butterflies_per_s": bfly / (f_ms * 1e-3), "inverse_butterflies_per_s": bfly / (i_ms * 1e-3),
             "bytes_per_coeff": {"ntt": 16, "muladd": 32}}
+
+
+def convert_bootstrap_bench(ctx, cfg, dev, stream, flush, offsets, rows, seed):
+    """MBFV.Convert to the recipients' own keys (+ BFV.Decrypt) and MBFV.Bootstrap on the first few
+    ciphertext indices of the workload, all K recipients and share holders: CUDA-event time per call
+    and the share calls' fraction of the integer roofline (slots counted as for the decryption shares:
+    Convert = NTT(c_1) once, then per share NTT(mu_k), two inverse transforms, three pointwise
+    products per limb and three samples per coefficient; Bootstrap = NTT(c_1), NTT(alpha) and L
+    samples per coefficient once, then per share two inverse transforms, two products and Lambda M_k
+    per limb and three samples per coefficient)."""
+    import torch
+
+    K, L, n = cfg.num_parties, cfg.num_limbs, cfg.n
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    per_ct = K * K * 2 * L * n * 8 + 4 * K * 2 * L * n * 8
+    cc = int(max(1, min(cfg.num_cts, 4, int(free_b * 0.5) // per_ct)))
+    parties = list(range(K))
+    values = torch.from_numpy(wl.gradients(cfg, seed, 0, cc)).to(dev)
+    plain = ctx.empty_u32(K, cc, n)
+    ct, agg = ctx.empty_u64(K, cc, 2, L, n), ctx.empty_u64(K, cc, 2, L, n)
+    shares = ctx.empty_u64(K, K, cc, 2, L, n)
+    conv, scratch = ctx.empty_u64(K, cc, 2, L, n), ctx.empty_u64(K, cc, L, n)
+    out_plain = ctx.empty_u32(K, cc, n)
+    sums = torch.empty((K, cc, n), dtype=torch.int32, device=dev)
+    ctx.encode(values, K * cc, plain)
+    ctx.encrypt(parties, 0, cc, plain, ct)
+    ctx.aggregate(ct, K, cc, offsets, rows, agg)
+    ctx.user_keygen(parties)
+
+    def timed(fn, reps=3):
+        fn()
+        best = None
+        for _ in range(reps):
+            flush.zero_()
+            a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a_.record(stream)
+            fn()
+            b_.record(stream)
+            torch.cuda.synchronize(dev)
+            ms = a_.elapsed_time(b_)
+            best = ms if best is None else min(best, ms)
+        return best
+
+    idx = [torch.as_tensor(rows[offsets[i]:offsets[i + 1]].astype(np.int64), device=dev) for i in range(K)]
+
+    def check(what):
+        ctx.decode(out_plain, K * cc, sums)
+        ok = all(bool(torch.equal(sums[i], values[idx[i]].sum(dim=0, dtype=torch.int32))) for i in range(K))
+        if not ok:
+            raise RuntimeError(what + ": decrypted sums differ from the plaintext sums")
+
+    t_cs = timed(lambda: ctx.convert_share(agg, parties, parties, 0, cc, shares))
+    t_cc = timed(lambda: ctx.convert_combine(agg, shares, K, K, cc, conv))
+    t_cd = timed(lambda: ctx.decrypt(parties, conv, cc, scratch, out_plain))
+    check("Convert")
+    t_bs = timed(lambda: ctx.bootstrap_share(agg, parties, parties, 0, cc, shares))
+    t_bc = timed(lambda: ctx.bootstrap_combine(agg, shares, parties, K, 0, cc, out_plain, conv))
+    # the refreshed ciphertext decrypts to the same sums through the ordinary collective decryption
+    sh1 = shares.view(-1)[:K * K * cc * L * n].view(K, K, cc, L, n)
+    ctx.partial_decrypt(conv, parties, parties, 0, cc, sh1)
+    ctx.combine_decrypt(conv, sh1, K, K, cc, out_plain)
+    check("Bootstrap")
+    T = SLOTS_PER_BUTTERFLY * (n // 2) * cfg.log2_n
+    units, S = K * cc, K
+    slots_conv = units * (L * (T + S * (3 * T + 3 * 14 * n)) + S * 3 * 40 * n)
+    slots_boot = units * (L * (2 * T + 40 * n + S * (2 * T + 2 * 14 * n + 10 * n)) + S * 3 * 40 * n)
+    return {"cts": cc, "units": units,
+            "convert_share_ms": t_cs, "convert_combine_ms": t_cc, "decrypt_ms": t_cd,
+            "bootstrap_share_ms": t_bs, "bootstrap_combine_ms": t_bc,
+            "convert_share_slots": slots_conv, "bootstrap_share_slots": slots_boot,
+            "share_bytes": units * S * 2 * 8 * n * L}
 
 
 def run_cuda(args, cfg):
@@ -530,6 +604,10 @@ def run_cuda(args, cfg):
             ntt[k_ + "_frac_of_hbm"] = ntt[k_ + "_GBps"] / peak
         for k_ in ("forward", "inverse"):
             ntt[k_ + "_alu_frac"] = ntt[k_ + "_butterflies_per_s"] * SLOTS_PER_BUTTERFLY / imad_peak
+        cb = res["convert_bootstrap"]
+        for k_ in ("convert", "bootstrap"):
+            cb[k_ + "_share_alu_frac"] = cb[k_ + "_share_slots"] / (cb[k_ + "_share_ms"] * 1e-3) / imad_peak
+            cb[k_ + "_share_GBps"] = cb["share_bytes"] / 1e9 / (cb[k_ + "_share_ms"] * 1e-3)
         kernels = {}
         for name in STEP_CALLS:
             ms = per_call[name] / serial_steps  # per step, summed over chunks
@@ -593,6 +671,7 @@ def run_cuda(args, cfg):
                             "mcycles = duration x median sampled SM clock",
             "kernels": kernels,
             "ntt": ntt,
+            "convert_bootstrap": cb,
             "other_configs": others,
             "init_ms": res["init_ms"],
             "wall_ms_per_step_incl_flush": res["wall_ms_per_step_incl_flush"],

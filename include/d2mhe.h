@@ -51,6 +51,14 @@ enum {
   D2MHE_ERR_DEVICE_CHECK = -8 /* a check that runs on the device failed (see `flags`)    */
 };
 
+/* d2mhe_params.flags: run this context on the checked build of every kernel.  Each kernel then
+ * tests the indices it is about to use (coefficient and octet numbers, shared-memory offsets,
+ * twiddle indices, party numbers read from the index lists) against their limits; the first
+ * violation is recorded in a device word and the access is skipped (no trap: the context stays
+ * usable).  d2mhe_sync returns D2MHE_ERR_DEVICE_CHECK once for it.  Results are the same as
+ * without the flag; the kernels are a few per cent slower. */
+#define D2MHE_FLAG_DEVICE_CHECKS 1u
+
 typedef struct {
   uint32_t struct_size;   /* = sizeof(d2mhe_params)                                      */
   uint32_t log2_n;        /* ring degree N = 2^log2_n, 3 <= log2_n <= 16.  The protocol
@@ -63,7 +71,7 @@ typedef struct {
                              (encode/decode) additionally needs t = 1 mod 2N.            */
   uint64_t seed;          /* Philox key                                                  */
   uint32_t gauss_bound;   /* B of the error distribution; must be 19 (sigma = 3.2)       */
-  uint32_t flags;         /* reserved, must be 0                                         */
+  uint32_t flags;         /* 0, or D2MHE_FLAG_DEVICE_CHECKS; other bits must be 0        */
   int32_t device;         /* CUDA device ordinal                                         */
 } d2mhe_params;
 
@@ -74,8 +82,10 @@ d2mhe_status d2mhe_create(const d2mhe_params* params, d2mhe_ctx** out);
 void d2mhe_destroy(d2mhe_ctx* ctx);
 /* Stream (a cudaStream_t passed as void*) on which later calls are enqueued; NULL = default. */
 d2mhe_status d2mhe_set_stream(d2mhe_ctx* ctx, void* cuda_stream);
-/* Waits for the stream; returns the first asynchronous error or D2MHE_ERR_RANGE if
- * d2mhe_encode saw a value outside [-(t-1)/2, (t-1)/2] since the last sync (flag is cleared). */
+/* Waits for the stream; returns the first asynchronous error, D2MHE_ERR_DEVICE_CHECK if a kernel of
+ * a context created with D2MHE_FLAG_DEVICE_CHECKS recorded an index violation since the last sync,
+ * or D2MHE_ERR_RANGE if d2mhe_encode saw a value outside [-(t-1)/2, (t-1)/2] since the last sync
+ * (either record is cleared by the call that reports it). */
 d2mhe_status d2mhe_sync(d2mhe_ctx* ctx);
 const char* d2mhe_strerror(d2mhe_status status);
 
@@ -143,7 +153,8 @@ d2mhe_status d2mhe_aggregate(d2mhe_ctx* ctx, const uint64_t* ct_dev, uint32_t n_
  * The noise of the shares is sampled by a kernel of its own into a 64 MiB scratch buffer that the
  * context owns (one byte per share coefficient; as many (recipient, ciphertext) pairs per launch as
  * fit), so the call is one or more pairs of launches on the context's stream.
- * D2MHE_ERR_UNSUPPORTED if n_parties * N exceeds that buffer.
+ * D2MHE_ERR_UNSUPPORTED if n_parties * N exceeds that buffer (d2mhe_convert_share and
+ * d2mhe_bootstrap_share work the same way with 3 and 6 bytes per share coefficient).
  */
 d2mhe_status d2mhe_partial_decrypt(d2mhe_ctx* ctx, const uint64_t* agg_dev,
                                    const uint32_t* recipients, uint32_t n_rec,
@@ -314,6 +325,14 @@ d2mhe_status d2mhe_round_device_static(d2mhe_ctx* ctx, const int32_t* values_dev
                                        const uint32_t* nbr_rows, int32_t* sums_dev);
 
 /* Test hooks. */
+/* The violation that d2mhe_sync last reported as D2MHE_ERR_DEVICE_CHECK:
+ * info = {site (1 load, 2 store, 3 octet, 4 shared-memory offset, 5 twiddle index, 6 party number,
+ * 7 limb, 8 streaming element, 9 staged bytes, 15 self-test), index, limit, thread block}. */
+d2mhe_status d2mhe_debug_last_device_check(const d2mhe_ctx* ctx, uint32_t info[4]);
+/* Launches one thread that runs the checked build's index test on the index 1 with limit 1 (it
+ * touches no memory): with D2MHE_FLAG_DEVICE_CHECKS the next d2mhe_sync returns
+ * D2MHE_ERR_DEVICE_CHECK with site 15, without the flag nothing happens. */
+d2mhe_status d2mhe_debug_check_selftest(d2mhe_ctx* ctx);
 /* s_k as int8 [N] on the HOST (needs a key share for `party`): the key that the device stores (in
  * the transform domain) is inverse-transformed on the GPU, limb by limb, and copied back;
  * D2MHE_ERR_DEVICE_CHECK if the limbs disagree or a coefficient is not in {-1, 0, 1}.  Allocates a

@@ -41,9 +41,11 @@ def build(force=False, verbose=False, defines=()):
     nvcc = _nvcc()
     extra = (["-Xptxas", "-v"] if verbose else []) + ["-D" + d for d in defines]
 
-    def compile_one(src):
-        obj = os.path.join(obj_dir, src.replace(".cu", ".o"))
-        cmd = [nvcc] + NVCC_FLAGS + extra + ["-c", os.path.join(CSRC, src), "-o", obj]
+    def compile_one(job):
+        src, checked = job
+        obj = os.path.join(obj_dir, src.replace(".cu", "_chk.o" if checked else ".o"))
+        cmd = [nvcc] + NVCC_FLAGS + extra + (["-DD2MHE_CHECKED"] if checked else []) + [
+            "-c", os.path.join(CSRC, src), "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             raise RuntimeError("nvcc failed for %s:\n%s" % (src, r.stderr))
@@ -51,8 +53,11 @@ def build(force=False, verbose=False, defines=()):
             sys.stderr.write(r.stderr)
         return obj
 
-    with ThreadPoolExecutor(max_workers=len(SOURCES)) as ex:
-        objs = list(ex.map(compile_one, SOURCES))
+    # every kernel file is compiled twice: as it is, and with index checks in every kernel (the build
+    # that contexts created with D2MHE_FLAG_DEVICE_CHECKS launch)
+    jobs = [(s, False) for s in SOURCES] + [(s, True) for s in SOURCES if s.startswith("kern_")]
+    with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 4)) as ex:
+        objs = list(ex.map(compile_one, jobs))
     tmp = LIB + ".%d.tmp" % os.getpid()
     r = subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"], capture_output=True, text=True)
     if r.returncode != 0:

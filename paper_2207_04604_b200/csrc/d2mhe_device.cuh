@@ -33,7 +33,43 @@ struct LimbTab {
   // [0][i] = W[N/8 + i], [1 + b][i] = W[N/4 + 2i + b], [3 + r][i] = W[N/2 + 4i + r].
   const ulonglong2* WL;         // [7][N/8]
   const ulonglong2* IWL;        // [7][N/8]
+  u32* chk;                     // device check words (read by the checked kernel build only)
 };
+
+// ---------------------------------------------------------------------------
+// Checked build.  Compiled with D2MHE_CHECKED every kernel tests the indices it is about to use
+// (coefficient and octet numbers, shared-memory byte offsets, twiddle indices, party numbers read
+// from index lists) against their limits.  A violation is recorded once in four device words
+// {site, index, limit, block} and the access is skipped: no trap, no assert, the context stays
+// usable, and the host reads the words at the next synchronisation.  Without the macro the checks
+// compile to nothing.
+// ---------------------------------------------------------------------------
+enum : u32 {
+  SITE_LOAD = 1,       // coefficient index handed to a load functor
+  SITE_STORE = 2,      // coefficient index handed to a store functor
+  SITE_OCTET = 3,      // octet index handed to a fetch / emit functor
+  SITE_SMEM = 4,       // byte offset into the shared-memory polynomial
+  SITE_TWIDDLE = 5,    // twiddle-table index
+  SITE_PARTY = 6,      // party / user / recipient number read from an index list
+  SITE_LIMB = 7,       // limb number
+  SITE_ELEMENT = 8,    // element index of a streaming kernel
+  SITE_STAGED = 9,     // offset into staged bytes in shared memory
+  SITE_SELFTEST = 15   // raised on purpose by the self-test hook
+};
+#ifdef D2MHE_CHECKED
+__device__ __forceinline__ bool d2mhe_chk(u32* w, unsigned long long idx, unsigned long long limit, u32 site) {
+  if (idx < limit) return true;
+  if (w && atomicCAS(w, 0u, site) == 0u) {
+    w[1] = (u32)idx;
+    w[2] = (u32)limit;
+    w[3] = blockIdx.x;
+  }
+  return false;
+}
+#define D2MHE_CHK(w, idx, limit, site) d2mhe_chk((w), (unsigned long long)(idx), (unsigned long long)(limit), (site))
+#else
+#define D2MHE_CHK(w, idx, limit, site) true
+#endif
 
 // ---------------------------------------------------------------------------
 // Modular arithmetic on [0, 2^64)
@@ -265,10 +301,17 @@ __device__ __forceinline__ u64 shoup_approx_sf(u64 y, u64 w, u64 ws, u32 d, u32 
 struct Mod {
   u64 p, np, twop, fourp;
   u32 red_shift, red_mul, sf_d, sf_shift;
+  u32* chk;       // check words and limits of the checked build (unused otherwise)
+  u32 tw_limit;   // entries of the twiddle tables W / IW
+  u32 twl_limit;  // entries of the regrouped tables WL / IWL
   __device__ __forceinline__ explicit Mod(const LimbTab& lt)
       : p(lt.p), np(lt.np), twop(lt.twop), fourp(2 * lt.twop), red_shift(lt.red_shift), red_mul(lt.red_mul),
-        sf_d(lt.sf_d), sf_shift(lt.sf_shift) {}
+        sf_d(lt.sf_d), sf_shift(lt.sf_shift), chk(lt.chk), tw_limit(0xffffffffu), twl_limit(0xffffffffu) {}
 };
+__device__ __forceinline__ ulonglong2 tw_ld(const ulonglong2* __restrict__ T, u32 idx, u32 limit, const Mod& m) {
+  if (!D2MHE_CHK(m.chk, idx, limit, SITE_TWIDDLE)) return make_ulonglong2(0, 0);
+  return __ldg(T + idx);
+}
 
 // x - q p with q = floor(floor(x / 2^(b-1)) * floor(2^(b+15) / p) / 2^16), b = bitlen(p): q is
 // floor(x/p) or up to 2 below it, so the result is below 3p.  Needs x < 2^(b+8) (true for every
@@ -344,12 +387,12 @@ template <int WIDE>
 __device__ __forceinline__ void fwd_octet(u64 (&x)[8], const ulonglong2* __restrict__ W, u32 m,
                                           u32 i, int nst, const Mod& md) {
   {
-    const ulonglong2 w = __ldg(W + m + i);
+    const ulonglong2 w = tw_ld(W, m + i, md.tw_limit, md);
 #pragma unroll
     for (int k = 0; k < 4; ++k) ct_bfly<WIDE>(x[k], x[k + 4], w, md);
   }
   if (nst >= 2) {
-    const ulonglong2 w0 = __ldg(W + 2 * m + 2 * i), w1 = __ldg(W + 2 * m + 2 * i + 1);
+    const ulonglong2 w0 = tw_ld(W, 2 * m + 2 * i, md.tw_limit, md), w1 = tw_ld(W, 2 * m + 2 * i + 1, md.tw_limit, md);
     ct_bfly<WIDE>(x[0], x[2], w0, md);
     ct_bfly<WIDE>(x[1], x[3], w0, md);
     ct_bfly<WIDE>(x[4], x[6], w1, md);
@@ -358,7 +401,7 @@ __device__ __forceinline__ void fwd_octet(u64 (&x)[8], const ulonglong2* __restr
   if (nst >= 3) {
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-      const ulonglong2 w = __ldg(W + 4 * m + 4 * i + r);
+      const ulonglong2 w = tw_ld(W, 4 * m + 4 * i + r, md.tw_limit, md);
       ct_bfly<WIDE>(x[2 * r], x[2 * r + 1], w, md);
     }
   }
@@ -368,12 +411,12 @@ template <int MODE>
 __device__ __forceinline__ void fwd_octet_last(u64 (&x)[8], const ulonglong2* __restrict__ WL, u32 oc,
                                                u32 i, const Mod& md) {
   {
-    const ulonglong2 w = __ldg(WL + i);
+    const ulonglong2 w = tw_ld(WL, i, md.twl_limit, md);
 #pragma unroll
     for (int k = 0; k < 4; ++k) ct_bfly<MODE>(x[k], x[k + 4], w, md);
   }
   {
-    const ulonglong2 w0 = __ldg(WL + oc + i), w1 = __ldg(WL + 2 * oc + i);
+    const ulonglong2 w0 = tw_ld(WL, oc + i, md.twl_limit, md), w1 = tw_ld(WL, 2 * oc + i, md.twl_limit, md);
     ct_bfly<MODE>(x[0], x[2], w0, md);
     ct_bfly<MODE>(x[1], x[3], w0, md);
     ct_bfly<MODE>(x[4], x[6], w1, md);
@@ -381,7 +424,7 @@ __device__ __forceinline__ void fwd_octet_last(u64 (&x)[8], const ulonglong2* __
   }
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
-    const ulonglong2 w = __ldg(WL + (3 + r) * oc + i);
+    const ulonglong2 w = tw_ld(WL, (3 + r) * oc + i, md.twl_limit, md);
     ct_bfly<MODE>(x[2 * r], x[2 * r + 1], w, md);
   }
 }
@@ -391,18 +434,18 @@ __device__ __forceinline__ void inv_octet_first(u64 (&x)[8], const ulonglong2* _
   const u64 c16 = md.fourp << 2, c32 = md.fourp << 3, c64 = md.fourp << 4;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
-    const ulonglong2 w = __ldg(IWL + (3 + r) * oc + i);
+    const ulonglong2 w = tw_ld(IWL, (3 + r) * oc + i, md.twl_limit, md);
     gs_bfly<MODE>(x[2 * r], x[2 * r + 1], w, md, c16);
   }
   {
-    const ulonglong2 w0 = __ldg(IWL + oc + i), w1 = __ldg(IWL + 2 * oc + i);
+    const ulonglong2 w0 = tw_ld(IWL, oc + i, md.twl_limit, md), w1 = tw_ld(IWL, 2 * oc + i, md.twl_limit, md);
     gs_bfly<MODE>(x[0], x[2], w0, md, c32);
     gs_bfly<MODE>(x[1], x[3], w0, md, c32);
     gs_bfly<MODE>(x[4], x[6], w1, md, c32);
     gs_bfly<MODE>(x[5], x[7], w1, md, c32);
   }
   {
-    const ulonglong2 w = __ldg(IWL + i);
+    const ulonglong2 w = tw_ld(IWL, i, md.twl_limit, md);
 #pragma unroll
     for (int k = 0; k < 4; ++k) gs_bfly<MODE>(x[k], x[k + 4], w, md, c64);
   }
@@ -419,19 +462,19 @@ __device__ __forceinline__ void inv_octet(u64 (&x)[8], const ulonglong2* __restr
   if (nst >= 3) {
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-      const ulonglong2 w = __ldg(IW + 4 * m + 4 * i + r);
+      const ulonglong2 w = tw_ld(IW, 4 * m + 4 * i + r, md.tw_limit, md);
       gs_bfly<MODE>(x[2 * r], x[2 * r + 1], w, md, c16);
     }
   }
   if (nst >= 2) {
-    const ulonglong2 w0 = __ldg(IW + 2 * m + 2 * i), w1 = __ldg(IW + 2 * m + 2 * i + 1);
+    const ulonglong2 w0 = tw_ld(IW, 2 * m + 2 * i, md.tw_limit, md), w1 = tw_ld(IW, 2 * m + 2 * i + 1, md.tw_limit, md);
     gs_bfly<MODE>(x[0], x[2], w0, md, c32);
     gs_bfly<MODE>(x[1], x[3], w0, md, c32);
     gs_bfly<MODE>(x[4], x[6], w1, md, c32);
     gs_bfly<MODE>(x[5], x[7], w1, md, c32);
   }
   {
-    const ulonglong2 w = __ldg(IW + m + i);
+    const ulonglong2 w = tw_ld(IW, m + i, md.tw_limit, md);
 #pragma unroll
     for (int k = 0; k < 4; ++k) gs_bfly<MODE>(x[k], x[k + 4], w, md, c64);
   }
@@ -542,6 +585,14 @@ struct OctAddr {
 __device__ __forceinline__ u64& sm_at(u64* sm, u32 byte_off) {
   return *reinterpret_cast<u64*>(reinterpret_cast<unsigned char*>(sm) + byte_off);
 }
+// the same through the checked build's test: byte_off must lie inside the polynomial and be a multiple of 8
+__device__ __forceinline__ u64 sm_get(u64* sm, u32 byte_off, u32 bytes, const Mod& m) {
+  if (!D2MHE_CHK(m.chk, byte_off | ((byte_off & 7u) ? 0x80000000u : 0u), bytes, SITE_SMEM)) return 0;
+  return sm_at(sm, byte_off);
+}
+__device__ __forceinline__ void sm_put(u64* sm, u32 byte_off, u64 v, u32 bytes, const Mod& m) {
+  if (D2MHE_CHK(m.chk, byte_off | ((byte_off & 7u) ? 0x80000000u : 0u), bytes, SITE_SMEM)) sm_at(sm, byte_off) = v;
+}
 
 // A transform of size N' = 2^logn can also be block `blk` of a larger transform whose first
 // `soff` stages were applied elsewhere (two-pass transforms for N > 16384): the block then
@@ -557,7 +608,10 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
   const NttGeom<LOGN, G> ge(logn_rt);
   const u32 T = ge.T, tid = threadIdx.x;
   constexpr int GB = ntt_group_bits(LOGN, WIDE);
-  const Mod md(lt);
+  Mod md(lt);
+  md.tw_limit = ge.n << soff;
+  md.twl_limit = 7u * ge.octets;
+  const u32 smb = ge.n << 3;  // bytes of the shared-memory polynomial
   const ulonglong2* __restrict__ W = lt.W;
   u64 x[8];
   __syncthreads();  // previous users of sm are done
@@ -571,10 +625,13 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
       if (LOGN || q < ge.octets) {
         const OctAddr ad(q, sh);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) x[k] = load(q + ((u32)k << sh));
+        for (int k = 0; k < 8; ++k) {
+          const u32 j = q + ((u32)k << sh);
+          x[k] = D2MHE_CHK(md.chk, j, ge.n, SITE_LOAD) ? load(j) : 0;
+        }
         fwd_octet<WIDE>(x, W, 1u << soff, blk, (int)ge.r0, md);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) sm_at(sm, ad.at(k, sh)) = x[k];
+        for (int k = 0; k < 8; ++k) sm_put(sm, ad.at(k, sh), x[k], smb, md);
       }
     }
     s = ge.r0;
@@ -595,20 +652,23 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
         const OctAddr ad(base, sh);
         if (from_load) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) x[k] = load(base + ((u32)k << sh));
+          for (int k = 0; k < 8; ++k) {
+            const u32 j = base + ((u32)k << sh);
+            x[k] = D2MHE_CHK(md.chk, j, ge.n, SITE_LOAD) ? load(j) : 0;
+          }
         } else {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
+          for (int k = 0; k < 8; ++k) x[k] = sm_get(sm, ad.at(k, sh), smb, md);
         }
         if (WIDE == MODE_PAIR && last && soff == 0)  // pays only where shared-memory wavefronts bind
           fwd_octet_last<WIDE>(x, lt.WL, ge.octets, i, md);
         else
           fwd_octet<WIDE>(x, W, m << soff, (blk << s) + i, 3, md);
         if (last) {
-          emit(g, q, x);
+          if (D2MHE_CHK(md.chk, q, ge.octets, SITE_OCTET)) emit(g, q, x);
         } else {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) sm_at(sm, ad.at(k, sh)) = x[k];
+          for (int k = 0; k < 8; ++k) sm_put(sm, ad.at(k, sh), x[k], smb, md);
         }
       }
     }
@@ -631,7 +691,10 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
   const NttGeom<LOGN, G> ge(logn_rt);
   const u32 T = ge.T, tid = threadIdx.x;
   constexpr int GB = ntt_group_bits(LOGN, WIDE);
-  const Mod md(lt);
+  Mod md(lt);
+  md.tw_limit = ge.n << soff;
+  md.twl_limit = 7u * ge.octets;
+  const u32 smb = ge.n << 3;  // bytes of the shared-memory polynomial
   const ulonglong2* __restrict__ IW = lt.IW;
   u64 x[8];
   __syncthreads();  // previous users of sm are done
@@ -650,10 +713,15 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
         const u32 base = ((i << 3) << sh) + o;
         const OctAddr ad(base, sh);
         if (from_fetch) {
-          fetch(g, q, x);
+          if (D2MHE_CHK(md.chk, q, ge.octets, SITE_OCTET)) {
+            fetch(g, q, x);
+          } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) x[k] = 0;
+          }
         } else {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
+          for (int k = 0; k < 8; ++k) x[k] = sm_get(sm, ad.at(k, sh), smb, md);
         }
         if (WIDE == MODE_PAIR && from_fetch && soff == 0)
           inv_octet_first<WIDE>(x, lt.IWL, ge.octets, i, md);
@@ -662,10 +730,13 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
         if (final_round) {
           finish_octet<WIDE>(x, 3, md);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) store(base + ((u32)k << sh), x[k]);
+          for (int k = 0; k < 8; ++k) {
+            const u32 j = base + ((u32)k << sh);
+            if (D2MHE_CHK(md.chk, j, ge.n, SITE_STORE)) store(j, x[k]);
+          }
         } else {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) sm_at(sm, ad.at(k, sh)) = x[k];
+          for (int k = 0; k < 8; ++k) sm_put(sm, ad.at(k, sh), x[k], smb, md);
         }
       }
     }
@@ -682,11 +753,14 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
       if (LOGN || q < ge.octets) {
         const OctAddr ad(q, sh);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) x[k] = sm_at(sm, ad.at(k, sh));
+        for (int k = 0; k < 8; ++k) x[k] = sm_get(sm, ad.at(k, sh), smb, md);
         inv_octet<WIDE>(x, IW, 1u << soff, blk, (int)ge.r0, md);
         finish_octet<WIDE>(x, (int)ge.r0, md);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) store(q + ((u32)k << sh), x[k]);
+        for (int k = 0; k < 8; ++k) {
+          const u32 j = q + ((u32)k << sh);
+          if (D2MHE_CHK(md.chk, j, ge.n, SITE_STORE)) store(j, x[k]);
+        }
       }
     }
   }

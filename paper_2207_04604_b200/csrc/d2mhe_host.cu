@@ -11,8 +11,8 @@
 
 typedef unsigned __int128 u128;
 
-// launcher of the context's kernel build
-#define L_(fn) d2mhe_launch::fn
+// launcher of the context's kernel build (plain, or with index checks in every kernel)
+#define L_(fn) (c->checked ? d2mhe_launch_chk::fn : d2mhe_launch::fn)
 
 namespace {
 
@@ -213,6 +213,12 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
 
   // q as a little-endian multi-word integer is never needed: everything about q that the
   // kernels use is a residue, computed limb by limb.
+  // check words of the checked kernel build: {site, index, limit, block}
+  c->view.chk = dev_alloc<u32>(c, 4, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  err = cudaMemset(c->view.chk, 0, 16);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+
   std::vector<LimbTab> limbs(L);
   // (q-1)/2 mod m and q mod m for a word-size m: q = prod q_l, so q mod m by repeated products;
   // (q-1)/2 mod m = (q-1) * 2^-1 mod m for odd m.
@@ -228,6 +234,7 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   for (u32 l = 0; l < L; ++l) {
     const u64 p = c->moduli[l];
     LimbTab& T = limbs[l];
+    T.chk = c->view.chk;
     T.p = p;
     T.twop = 2 * p;
     T.np = 0 - p;
@@ -457,7 +464,7 @@ d2mhe_status d2mhe_create(const d2mhe_params* P, d2mhe_ctx** out) {
   if (P->log2_n < 3 || P->log2_n > 16) return D2MHE_ERR_BAD_PARAMS;
   if (P->num_limbs < 1 || P->num_limbs > D2MHE_MAX_LIMBS) return D2MHE_ERR_BAD_PARAMS;
   if (P->num_parties < 1 || P->num_parties > 65535) return D2MHE_ERR_BAD_PARAMS;
-  if (P->gauss_bound != D2MHE_GAUSS_B || P->flags != 0) return D2MHE_ERR_BAD_PARAMS;
+  if (P->gauss_bound != D2MHE_GAUSS_B || (P->flags & ~(u32)D2MHE_FLAG_DEVICE_CHECKS) != 0) return D2MHE_ERR_BAD_PARAMS;
   const u64 t = P->plain_modulus, two_n = (u64)2 << P->log2_n;
   if (t < 3 || t >= ((u64)1 << 30) || !h_is_prime(t)) return D2MHE_ERR_BAD_PARAMS;
   for (u32 l = 0; l < P->num_limbs; ++l) {
@@ -477,6 +484,7 @@ d2mhe_status d2mhe_create(const d2mhe_params* P, d2mhe_ctx** out) {
   c->moduli.assign(P->moduli, P->moduli + P->num_limbs);
   c->params.moduli = reinterpret_cast<const uint64_t*>(c->moduli.data());
   c->device = P->device;
+  c->checked = (P->flags & D2MHE_FLAG_DEVICE_CHECKS) != 0;
   c->can_pack = (t - 1) % two_n == 0;
   c->narrow = true;
   for (u32 l = 0; l < P->num_limbs; ++l)
@@ -539,11 +547,38 @@ d2mhe_status d2mhe_sync(d2mhe_ctx* c) {
   u32 flag = 0;
   e = cudaMemcpy(&flag, c->view.range_flag, sizeof(u32), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return fail_cuda(c, e);
+  if (c->checked) {
+    u32 words[4] = {0, 0, 0, 0};
+    e = cudaMemcpy(words, c->view.chk, sizeof(words), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    if (words[0]) {
+      std::memcpy(c->last_check, words, sizeof(words));
+      e = cudaMemset(c->view.chk, 0, sizeof(words));
+      if (e != cudaSuccess) return fail_cuda(c, e);
+      if (flag) (void)cudaMemset(c->view.range_flag, 0, sizeof(u32));
+      return D2MHE_ERR_DEVICE_CHECK;
+    }
+  }
   if (flag) {
     e = cudaMemset(c->view.range_flag, 0, sizeof(u32));
     if (e != cudaSuccess) return fail_cuda(c, e);
     return D2MHE_ERR_RANGE;
   }
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_debug_last_device_check(const d2mhe_ctx* c, uint32_t info[4]) {
+  if (!c || !info) return D2MHE_ERR_INVALID_ARG;
+  std::memcpy(info, c->last_check, sizeof(c->last_check));
+  return D2MHE_OK;
+}
+
+d2mhe_status d2mhe_debug_check_selftest(d2mhe_ctx* c) {
+  if (!c) return D2MHE_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  cudaError_t e = L_(check_selftest)(c->view, c->stream);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
   return D2MHE_OK;
 }
 
@@ -557,7 +592,7 @@ d2mhe_status d2mhe_keygen_share(d2mhe_ctx* c, const u32* parties, u32 n_parties)
   const u32* arrays[1] = {parties};
   const size_t counts[1] = {n_parties};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::keygen(c->view, c->limb_params, c->stream, sg.dev[0], n_parties);
+  cudaError_t e = L_(keygen)(c->view, c->limb_params, c->stream, sg.dev[0], n_parties);
   if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
   for (u32 i = 0; i < n_parties; ++i) c->has_share[parties[i]] = true;
@@ -576,7 +611,7 @@ d2mhe_status d2mhe_collective_pk(d2mhe_ctx* c, const u32* parties, u32 n_parties
   const u32* arrays[1] = {parties};
   const size_t counts[1] = {n_parties};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::collective_pk(c->view, c->limb_params, c->stream, sg.dev[0], n_parties,
+  cudaError_t e = L_(collective_pk)(c->view, c->limb_params, c->stream, sg.dev[0], n_parties,
                                               reinterpret_cast<u64*>(pk_shares_dev));
   if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
@@ -595,7 +630,7 @@ d2mhe_status d2mhe_encode(d2mhe_ctx* c, const int32_t* values_dev, u32 n_cts, u3
   if (!aligned16(values_dev) || !aligned16(plain_dev)) return D2MHE_ERR_INVALID_ARG;
   if (!c->can_pack || c->params.log2_n > 15) return D2MHE_ERR_UNSUPPORTED;
   DeviceGuard guard(c->device);
-  cudaError_t e = d2mhe_launch::encode(c->view, c->stream, values_dev, n_cts, plain_dev);
+  cudaError_t e = L_(encode)(c->view, c->stream, values_dev, n_cts, plain_dev);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
   return D2MHE_OK;
@@ -606,7 +641,7 @@ d2mhe_status d2mhe_decode(d2mhe_ctx* c, const u32* plain_dev, u32 n_cts, int32_t
   if (!aligned16(values_dev) || !aligned16(plain_dev)) return D2MHE_ERR_INVALID_ARG;
   if (!c->can_pack || c->params.log2_n > 15) return D2MHE_ERR_UNSUPPORTED;
   DeviceGuard guard(c->device);
-  cudaError_t e = d2mhe_launch::decode(c->view, c->stream, plain_dev, n_cts, values_dev);
+  cudaError_t e = L_(decode)(c->view, c->stream, plain_dev, n_cts, values_dev);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
   return D2MHE_OK;
@@ -629,7 +664,7 @@ d2mhe_status d2mhe_encrypt(d2mhe_ctx* c, const u32* parties, u32 n_parties, u32 
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
   // u, e_0, e_1 are sampled ahead into the context's scratch, batch by batch
   u32 launched = 0;
-  cudaError_t e = d2mhe_launch::encrypt(c->view, c->limb_params, c->stream, sg.dev[0], n_parties, ct_first, n_cts,
+  cudaError_t e = L_(encrypt)(c->view, c->limb_params, c->stream, sg.dev[0], n_parties, ct_first, n_cts,
                                         plain_dev, reinterpret_cast<u64*>(ct_dev), c->noise_scratch,
                                         c->noise_scratch_bytes, &launched);
   if (e != cudaSuccess) return fail_staged(c, sg, e);
@@ -660,7 +695,7 @@ d2mhe_status d2mhe_aggregate(d2mhe_ctx* c, const uint64_t* ct_dev, u32 n_rows, u
   const size_t counts[2] = {(size_t)n_out + 1, nnz ? (size_t)nnz : 1};
   d2mhe_status st = stage_indices(c, arrays, counts, 2, &sg);
   if (st != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::aggregate(c->view, c->stream, reinterpret_cast<const u64*>(ct_dev), n_cts,
+  cudaError_t e = L_(aggregate)(c->view, c->stream, reinterpret_cast<const u64*>(ct_dev), n_cts,
                                           sg.dev[0], sg.dev[1], n_out, reinterpret_cast<u64*>(agg_dev));
   if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
@@ -687,7 +722,7 @@ d2mhe_status d2mhe_partial_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev, const 
   if ((size_t)n_parties * c->view.n > c->noise_scratch_bytes) return D2MHE_ERR_UNSUPPORTED;
   if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
   u32 launched = 0;
-  cudaError_t e = d2mhe_launch::partial_decrypt_scratch(
+  cudaError_t e = L_(partial_decrypt_scratch)(
       c->view, c->limb_params, c->stream, reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1], n_parties,
       ct_first, n_cts, reinterpret_cast<u64*>(shares_dev), c->noise_scratch, c->noise_scratch_bytes, &launched);
   if (e != cudaSuccess) return fail_staged(c, sg, e);
@@ -706,7 +741,7 @@ d2mhe_status d2mhe_combine_decrypt(d2mhe_ctx* c, const uint64_t* agg_dev,
   if (n_shares != c->pk_parties.size()) return D2MHE_ERR_INVALID_ARG;
   if ((u64)n_rec * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
-  cudaError_t e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
+  cudaError_t e = L_(combine)(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
                                         reinterpret_cast<const u64*>(shares_dev), n_rec, n_shares, 1, n_cts,
                                         plain_dev);
   if (e != cudaSuccess) return fail_cuda(c, e);
@@ -720,7 +755,7 @@ static d2mhe_status ntt_common(d2mhe_ctx* c, u64* polys_dev, u32 batch, bool inv
   if ((u64)batch * c->view.L * (c->params.log2_n > D2MHE_MAX_SMEM_LOGN ? 16u : 1u) > 0x7fffffffull)
     return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
-  cudaError_t e = d2mhe_launch::ntt(c->view, c->limb_params, c->stream, polys_dev, batch, inverse);
+  cudaError_t e = L_(ntt)(c->view, c->limb_params, c->stream, polys_dev, batch, inverse);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += c->params.log2_n > D2MHE_MAX_SMEM_LOGN ? 2 : 1;
   return D2MHE_OK;
@@ -738,7 +773,7 @@ static d2mhe_status ntt32_common(d2mhe_ctx* c, u32* polys_dev, u32 batch, bool i
   if (!c->narrow || !protocol_ok(c)) return D2MHE_ERR_UNSUPPORTED;
   if ((u64)batch * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
-  cudaError_t e = d2mhe_launch::ntt32(c->view, c->limb_params, c->stream, polys_dev, batch, inverse);
+  cudaError_t e = L_(ntt32)(c->view, c->limb_params, c->stream, polys_dev, batch, inverse);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
   return D2MHE_OK;
@@ -755,7 +790,7 @@ d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* c, const uint32_t* a, const uint32_t
   if (!aligned16(a) || !aligned16(b) || !aligned16(cc) || !aligned16(d)) return D2MHE_ERR_INVALID_ARG;
   if (!c->narrow) return D2MHE_ERR_UNSUPPORTED;
   DeviceGuard guard(c->device);
-  cudaError_t e = d2mhe_launch::muladd32(c->view, c->stream, a, b, cc, d, batch);
+  cudaError_t e = L_(muladd32)(c->view, c->stream, a, b, cc, d, batch);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
   return D2MHE_OK;
@@ -766,7 +801,7 @@ d2mhe_status d2mhe_poly_muladd(d2mhe_ctx* c, const uint64_t* a, const uint64_t* 
   if (!c || !a || !b || !cc || !d || batch == 0) return D2MHE_ERR_INVALID_ARG;
   if (!aligned16(a) || !aligned16(b) || !aligned16(cc) || !aligned16(d)) return D2MHE_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
-  cudaError_t e = d2mhe_launch::muladd(c->view, c->stream, reinterpret_cast<const u64*>(a),
+  cudaError_t e = L_(muladd)(c->view, c->stream, reinterpret_cast<const u64*>(a),
                                        reinterpret_cast<const u64*>(b), reinterpret_cast<const u64*>(cc),
                                        reinterpret_cast<u64*>(d), batch);
   if (e != cudaSuccess) return fail_cuda(c, e);
@@ -787,7 +822,7 @@ d2mhe_status d2mhe_user_keygen(d2mhe_ctx* c, const u32* users, u32 n_users, uint
   const u32* arrays[1] = {users};
   const size_t counts[1] = {n_users};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::user_keygen(c->view, c->limb_params, c->stream, sg.dev[0], n_users);
+  cudaError_t e = L_(user_keygen)(c->view, c->limb_params, c->stream, sg.dev[0], n_users);
   if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
   const size_t pk_words = 2 * (size_t)c->view.L * c->view.n;
@@ -820,12 +855,16 @@ d2mhe_status d2mhe_convert_share(d2mhe_ctx* c, const uint64_t* agg_dev, const u3
   Staged sg;
   const u32* arrays[2] = {recipients, parties};
   const size_t counts[2] = {n_rec, n_parties};
+  // mu_k, e_{0,k}, e_{1,k} are sampled ahead into the context's scratch, batch by batch
+  if ((size_t)n_parties * 3 * c->view.n > c->noise_scratch_bytes) return D2MHE_ERR_UNSUPPORTED;
   if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::convert_share(c->view, c->limb_params, c->stream,
-                                              reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1],
-                                              n_parties, ct_first, n_cts, reinterpret_cast<u64*>(shares_dev));
+  u32 launched = 0;
+  cudaError_t e = L_(convert_share)(c->view, c->limb_params, c->stream, reinterpret_cast<const u64*>(agg_dev),
+                                    sg.dev[0], n_rec, sg.dev[1], n_parties, ct_first, n_cts,
+                                    reinterpret_cast<u64*>(shares_dev), c->noise_scratch, c->noise_scratch_bytes,
+                                    &launched);
   if (e != cudaSuccess) return fail_staged(c, sg, e);
-  c->launches += 1;
+  c->launches += launched;
   return release_slot(c, sg);
 }
 
@@ -837,7 +876,7 @@ d2mhe_status d2mhe_convert_combine(d2mhe_ctx* c, const uint64_t* agg_dev, const 
   if (n_shares != c->pk_parties.size()) return D2MHE_ERR_INVALID_ARG;
   if ((u64)n_rec * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
   DeviceGuard guard(c->device);
-  cudaError_t e = d2mhe_launch::convert_combine(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
+  cudaError_t e = L_(convert_combine)(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
                                                 reinterpret_cast<const u64*>(shares_dev), n_rec, n_shares, n_cts,
                                                 reinterpret_cast<u64*>(ct_out_dev));
   if (e != cudaSuccess) return fail_cuda(c, e);
@@ -860,12 +899,12 @@ d2mhe_status d2mhe_decrypt(d2mhe_ctx* c, const u32* users, u32 n_users, const ui
   const u32* arrays[1] = {users};
   const size_t counts[1] = {n_users};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::secret_product(c->view, c->limb_params, c->stream,
+  cudaError_t e = L_(secret_product)(c->view, c->limb_params, c->stream,
                                                reinterpret_cast<const u64*>(ct_dev), sg.dev[0], n_users, n_cts,
                                                reinterpret_cast<u64*>(scratch_dev));
   if (e != cudaSuccess) return fail_staged(c, sg, e);
   // [c_0 + c_1 sk_i]_q then the exact scale-and-round: the product plays the role of one share
-  e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(ct_dev),
+  e = L_(combine)(c->view, c->stream, reinterpret_cast<const u64*>(ct_dev),
                             reinterpret_cast<const u64*>(scratch_dev), n_users, 1, 1, n_cts, plain_dev);
   if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 2;
@@ -890,12 +929,16 @@ d2mhe_status d2mhe_bootstrap_share(d2mhe_ctx* c, const uint64_t* agg_dev, const 
   Staged sg;
   const u32* arrays[2] = {recipients, parties};
   const size_t counts[2] = {n_rec, n_parties};
+  // e_{0,k}, e_{1,k} and the masks M_k are sampled ahead into the context's scratch, batch by batch
+  if ((size_t)n_parties * 6 * c->view.n > c->noise_scratch_bytes) return D2MHE_ERR_UNSUPPORTED;
   if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::boot_share(c->view, c->limb_params, c->stream,
-                                           reinterpret_cast<const u64*>(agg_dev), sg.dev[0], n_rec, sg.dev[1],
-                                           n_parties, ct_first, n_cts, reinterpret_cast<u64*>(shares_dev));
+  u32 launched = 0;
+  cudaError_t e = L_(boot_share)(c->view, c->limb_params, c->stream, reinterpret_cast<const u64*>(agg_dev),
+                                 sg.dev[0], n_rec, sg.dev[1], n_parties, ct_first, n_cts,
+                                 reinterpret_cast<u64*>(shares_dev), c->noise_scratch, c->noise_scratch_bytes,
+                                 &launched);
   if (e != cudaSuccess) return fail_staged(c, sg, e);
-  c->launches += 1;
+  c->launches += launched;
   return release_slot(c, sg);
 }
 
@@ -916,11 +959,11 @@ d2mhe_status d2mhe_bootstrap_combine(d2mhe_ctx* c, const uint64_t* agg_dev, cons
   const u32* arrays[1] = {recipients};
   const size_t counts[1] = {n_rec};
   if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
-  cudaError_t e = d2mhe_launch::combine(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
+  cudaError_t e = L_(combine)(c->view, c->stream, reinterpret_cast<const u64*>(agg_dev),
                                         reinterpret_cast<const u64*>(shares_dev), n_rec, n_shares, 2, n_cts,
                                         plain_scratch_dev);
   if (e != cudaSuccess) return fail_staged(c, sg, e);
-  e = d2mhe_launch::boot_finish(c->view, c->stream, plain_scratch_dev, reinterpret_cast<const u64*>(shares_dev),
+  e = L_(boot_finish)(c->view, c->stream, plain_scratch_dev, reinterpret_cast<const u64*>(shares_dev),
                                 sg.dev[0], n_rec, n_shares, ct_first, n_cts, reinterpret_cast<u64*>(ct_out_dev));
   if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 2;
@@ -1121,7 +1164,7 @@ static d2mhe_status export_key(d2mhe_ctx* c, const u64* key_dev, int8_t* s_host)
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&tmp), L * n);
   if (e != cudaSuccess) return fail_cuda(c, e);
   std::vector<signed char> host(L * n);
-  e = d2mhe_launch::export_secret(c->view, c->limb_params, c->stream, key_dev, tmp);
+  e = L_(export_secret)(c->view, c->limb_params, c->stream, key_dev, tmp);
   if (e == cudaSuccess) {
     c->launches += 1;
     e = cudaMemcpyAsync(host.data(), tmp, L * n, cudaMemcpyDeviceToHost, c->stream);

@@ -50,6 +50,7 @@ struct DevView {
   u64* upk_mont;  // [K][2][L][N]  NTT(p_{0,i}), NTT(p_{1,i}) * N^-1 (Montgomery form)
   u64* upk_coef;  // [K][2][L][N]  pk_i, coefficient domain
   u32* range_flag;
+  u32* chk;       // four check words {site, index, limit, block} of the checked build
 };
 
 // ---- host-side context (shared by the translation units that implement the C ABI) ----
@@ -103,53 +104,72 @@ struct d2mhe_ctx {
   unsigned char* noise_scratch = nullptr;  // device: noise bytes of the shares of one d2mhe_partial_decrypt batch
   size_t noise_scratch_bytes = 0;
   cudaError_t last_cuda = cudaSuccess;
+  bool checked = false;             // launches the checked kernel build
+  u32 last_check[4] = {};           // the last violation that d2mhe_sync reported
 };
 
+// The kernel translation units are compiled twice: as they are into namespace d2mhe_launch, and
+// with D2MHE_CHECKED (index checks in every kernel, see d2mhe_device.cuh) into d2mhe_launch_chk.
+// A context created with D2MHE_FLAG_DEVICE_CHECKS launches the second set.
+#ifdef D2MHE_CHECKED
+#define D2MHE_LAUNCH_NS d2mhe_launch_chk
+#else
+#define D2MHE_LAUNCH_NS d2mhe_launch
+#endif
+
+// Launchers (one per kernel or kernel sequence).  Notes: encrypt and partial_decrypt_scratch sample
+// u, e_0, e_1 / the shares' noise ahead into caller-lent scratch (at least 3 N / n_parties N bytes)
+// and report their number of launches, and so do convert_share (n_parties 3 N bytes) and boot_share
+// (n_parties 6 N bytes); combine sums the first of share_comps polynomials per
+// (recipient, party, ciphertext); int_probe synchronises the stream; export_secret turns key rows
+// [L][N] (transform domain, Montgomery form) into int8 coefficients [L][N] (127 = not ternary);
+// check_selftest makes one thread of the checked build raise SITE_SELFTEST (no memory access).
+#define D2MHE_LAUNCHER_DECLS \
+cudaError_t keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties); \
+cudaError_t collective_pk(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties, \
+                          u64* shares_out); \
+cudaError_t int_probe(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 kind, u32 iters, u32* sink, \
+                      float* ms, double* lane_ops); \
+cudaError_t export_secret(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* key, signed char* out); \
+cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain); \
+cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values); \
+cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties, \
+                    u32 ct_first, u32 n_cts, const u32* plain, u64* ct, void* scratch, size_t scratch_bytes, \
+                    u32* launches); \
+cudaError_t aggregate(const DevView& v, cudaStream_t s, const u64* ct, u32 n_cts, \
+                      const u32* offsets_dev, const u32* rows_dev, u32 n_out, u64* agg); \
+cudaError_t partial_decrypt_scratch(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg, \
+                                    const u32* recipients_dev, u32 n_rec, const u32* parties_dev, \
+                                    u32 n_parties, u32 ct_first, u32 n_cts, u64* shares, void* scratch, \
+                                    size_t scratch_bytes, u32* launches); \
+cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec, \
+                    u32 n_shares, u32 share_comps, u32 n_cts, u32* plain); \
+cudaError_t boot_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg, \
+                       const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties, \
+                       u32 ct_first, u32 n_cts, u64* shares, void* scratch, size_t scratch_bytes, u32* launches); \
+cudaError_t boot_finish(const DevView& v, cudaStream_t s, const u32* x, const u64* shares, \
+                        const u32* recipients_dev, u32 n_rec, u32 n_shares, u32 ct_first, u32 n_cts, u64* out); \
+cudaError_t ntt(const DevView& v, const LimbParams& lp, cudaStream_t s, u64* polys, u32 batch, bool inverse); \
+cudaError_t ntt32(const DevView& v, const LimbParams& lp, cudaStream_t s, u32* polys, u32 batch, bool inverse); \
+cudaError_t muladd32(const DevView& v, cudaStream_t s, const u32* a, const u32* b, const u32* c, u32* d, \
+                     u32 batch); \
+cudaError_t user_keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* users_dev, \
+                        u32 n_users); \
+cudaError_t convert_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg, \
+                          const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties, \
+                          u32 ct_first, u32 n_cts, u64* shares, void* scratch, size_t scratch_bytes, u32* launches); \
+cudaError_t convert_combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec, \
+                            u32 n_shares, u32 n_cts, u64* out); \
+cudaError_t secret_product(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* ct, \
+                           const u32* users_dev, u32 n_users, u32 n_cts, u64* prod); \
+cudaError_t muladd(const DevView& v, cudaStream_t s, const u64* a, const u64* b, const u64* c, \
+                   u64* d, u32 batch); \
+cudaError_t check_selftest(const DevView& v, cudaStream_t s);
+
 namespace d2mhe_launch {
-cudaError_t keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties);
-cudaError_t collective_pk(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
-                          u64* shares_out);
-// measurement hook: register-only integer loops (kern_probe.cu); synchronises the stream
-cudaError_t int_probe(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 kind, u32 iters, u32* sink,
-                      float* ms, double* lane_ops);
-// test hook: key rows [L][N] (transform domain, Montgomery form) -> int8 coefficients [L][N] (127 = not ternary)
-cudaError_t export_secret(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* key, signed char* out);
-cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain);
-cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values);
-// u, e_0, e_1 are sampled ahead into caller-lent scratch (at least 3 N bytes)
-cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties,
-                    u32 ct_first, u32 n_cts, const u32* plain, u64* ct, void* scratch, size_t scratch_bytes,
-                    u32* launches);
-cudaError_t aggregate(const DevView& v, cudaStream_t s, const u64* ct, u32 n_cts,
-                      const u32* offsets_dev, const u32* rows_dev, u32 n_out, u64* agg);
-// decryption shares; their noise is sampled ahead into caller-lent scratch (at least n_parties * N bytes)
-cudaError_t partial_decrypt_scratch(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
-                                    const u32* recipients_dev, u32 n_rec, const u32* parties_dev,
-                                    u32 n_parties, u32 ct_first, u32 n_cts, u64* shares, void* scratch,
-                                    size_t scratch_bytes, u32* launches);
-// shares hold share_comps polynomials per (recipient, party, ciphertext); the first one is summed
-cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
-                    u32 n_shares, u32 share_comps, u32 n_cts, u32* plain);
-cudaError_t boot_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
-                       const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties,
-                       u32 ct_first, u32 n_cts, u64* shares);
-cudaError_t boot_finish(const DevView& v, cudaStream_t s, const u32* x, const u64* shares,
-                        const u32* recipients_dev, u32 n_rec, u32 n_shares, u32 ct_first, u32 n_cts, u64* out);
-cudaError_t ntt(const DevView& v, const LimbParams& lp, cudaStream_t s, u64* polys, u32 batch, bool inverse);
-// 32-bit-word variants (every prime below 2^30)
-cudaError_t ntt32(const DevView& v, const LimbParams& lp, cudaStream_t s, u32* polys, u32 batch, bool inverse);
-cudaError_t muladd32(const DevView& v, cudaStream_t s, const u32* a, const u32* b, const u32* c, u32* d,
-                     u32 batch);
-cudaError_t user_keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* users_dev,
-                        u32 n_users);
-cudaError_t convert_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
-                          const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties,
-                          u32 ct_first, u32 n_cts, u64* shares);
-cudaError_t convert_combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
-                            u32 n_shares, u32 n_cts, u64* out);
-cudaError_t secret_product(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* ct,
-                           const u32* users_dev, u32 n_users, u32 n_cts, u64* prod);
-cudaError_t muladd(const DevView& v, cudaStream_t s, const u64* a, const u64* b, const u64* c,
-                   u64* d, u32 batch);
-// number of kernel launches the call above performed (for bookkeeping)
-}  // namespace d2mhe_launch
+D2MHE_LAUNCHER_DECLS
+}
+namespace d2mhe_launch_chk {
+D2MHE_LAUNCHER_DECLS
+}
+

@@ -1,7 +1,7 @@
 // MBFV.Convert to a recipient's own key pair (Sec. 4.2 item 3, Eq. 2-3) and BFV.Decrypt under it.
-#include "d2mhe_kernels_common.cuh"
+#include <algorithm>
 
-namespace cg = cooperative_groups;
+#include "d2mhe_kernels_common.cuh"
 
 namespace {
 
@@ -19,6 +19,7 @@ template <int LOGN, int G, bool WIDE>
 __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
     k_user_keygen(DevView v, const __grid_constant__ LimbParams lp, const u32* __restrict__ users) {
   const u32 l = blockIdx.x % v.L, user = users[blockIdx.x / v.L];
+  if (!D2MHE_CHK(v.chk, user, v.K, SITE_PARTY)) return;
   const LimbTab& lt = lp.limbs[l];
   GaussTab* gt = gauss_smem();
   load_gauss(gt, v.gauss);
@@ -71,22 +72,47 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
       [&](int, u32 q, u64(&x)[8]) { store_octet_mont(pkm0 + 8 * (size_t)q, x, lt); });
 }
 
+// mu_k, e_{0,k}, e_{1,k} of a conversion share do not depend on the limb: like the noise of the
+// decryption shares they are sampled once per share by a kernel of its own, one byte per
+// coefficient, into scratch memory that the caller of the launcher lends ([mu | e_0 | e_1], N bytes
+// each, per (recipient, ciphertext) unit and party), so the share kernel needs no clusters.
+// grid = ceil(n_units * n_parties * 3 * N / 4 / 256); one thread = four samples = one packed word.
+__global__ void __launch_bounds__(256)
+    k_sample_convert_noise(DevView v, const u32* __restrict__ recipients, const u32* __restrict__ parties,
+                           u32 n_parties, u32 ct_first, u32 n_cts, u32 unit_first, u32 n_units,
+                           u32* __restrict__ out) {
+  __shared__ GaussTab gt;
+  load_gauss(&gt, v.gauss);
+  const u32 words = v.n >> 2;
+  const size_t total = (size_t)n_units * n_parties * 3 * words;
+  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;  // the last block is ragged
+  const u32 w = (u32)(e % words), which = (u32)((e / words) % 3);
+  const size_t share = e / (3 * (size_t)words);
+  const u32 a = (u32)(share % n_parties), unit = unit_first + (u32)(share / n_parties);
+  const u32 party = parties[a], recipient = recipients[unit / n_cts];
+  if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY) || !D2MHE_CHK(v.chk, recipient, v.K, SITE_PARTY)) return;
+  const Stream st(v.seed, which == 0 ? TAG_CONV_MU : which == 1 ? TAG_CONV_E0 : TAG_CONV_E1, ct_first + unit % n_cts,
+                  party, recipient);
+  u32 pack = 0;
+#pragma unroll
+  for (u32 b = 0; b < 4; ++b) pack |= ((u32)gauss_from_r(gt, st.draw64(4 * w + b)) & 0xffu) << (8 * b);
+  out[e] = pack;
+}
+
 // Conversion shares (Eq. 2): (h_0, h_1) = (s_k c_1 + mu_k p_{0,i} + e_{0,k}, mu_k p_{1,i} + e_{1,k}).
-// grid = n_rec * n_cts * L in clusters over limbs (mu, e_0, e_1 are sampled once per cluster).
+// grid = n_units * L; units unit_first .. unit_first + n_units - 1 of the (recipient, ciphertext) grid.
 // NTT(c_1) is parked in the h_0 row of the last share, NTT(mu_k) in the h_1 row of its own share.
 template <int LOGN, int G, bool WIDE>
 __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
     k_convert_share(DevView v, const __grid_constant__ LimbParams lp, const u64* __restrict__ agg,
                     const u32* __restrict__ recipients, const u32* __restrict__ parties, u32 n_parties,
-                    u32 ct_first, u32 n_cts, u64* shares) {
-  cg::cluster_group cluster = cg::this_cluster();
-  const u32 cs = cluster.num_blocks(), rank = cluster.block_rank();
-  const u32 l = blockIdx.x % v.L, unit = blockIdx.x / v.L;
-  const u32 irec = unit / n_cts, cl = unit % n_cts, c = ct_first + cl;
+                    u32 n_cts, u32 unit_first, const u32* __restrict__ sampled, u64* shares) {
+  const u32 l = blockIdx.x % v.L, ulocal = blockIdx.x / v.L, unit = unit_first + ulocal;
+  const u32 irec = unit / n_cts, cl = unit % n_cts;
   const u32 recipient = recipients[irec];
+  if (!D2MHE_CHK(v.chk, recipient, v.K, SITE_PARTY)) return;
   const LimbTab& lt = lp.limbs[l];
-  GaussTab* gt = gauss_smem();
-  load_gauss(gt, v.gauss);
   signed char* small = bytes_smem();  // mu, e_0, e_1: N bytes each
   u64* sm = poly_smem(3 * v.n);
   const size_t row = (size_t)l * v.n, poly = (size_t)v.L * v.n;
@@ -99,23 +125,12 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 #pragma unroll 1
   for (int a = -1; a < (int)n_parties; ++a) {
     const u32 party = a < 0 ? 0u : parties[a];
+    if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY)) continue;
     if (a >= 0) {
-      cluster.sync();  // every CTA is done with the previous share's samples
-      const Stream sm_(v.seed, TAG_CONV_MU, c, party, recipient);
-      const Stream s0(v.seed, TAG_CONV_E0, c, party, recipient);
-      const Stream s1(v.seed, TAG_CONV_E1, c, party, recipient);
-      const u32 quarter = v.n >> 2;
-      // words 0..N/4-1: mu, N/4..N/2-1: e_0, N/2..3N/4-1: e_1 (four samples per word)
-#pragma unroll 1
-      for (u32 w = rank + cs * threadIdx.x; w < 3 * quarter; w += cs * blockDim.x) {
-        const u32 which = w / quarter, j0 = 4 * (w - which * quarter);
-        const Stream& st = which == 0 ? sm_ : which == 1 ? s0 : s1;
-        u32 pack = 0;
-#pragma unroll
-        for (u32 b = 0; b < 4; ++b) pack |= ((u32)gauss_from_r(*gt, st.draw64(j0 + b)) & 0xffu) << (8 * b);
-        for (u32 r = 0; r < cs; ++r) cluster.map_shared_rank(reinterpret_cast<u32*>(small), r)[w] = pack;
-      }
-      cluster.sync();  // all samples of this share have landed everywhere
+      __syncthreads();  // every thread is done with the previous share's samples
+      const u32* src = sampled + ((size_t)ulocal * n_parties + a) * 3 * (v.n >> 2);
+      for (u32 w = threadIdx.x; w < 3 * (v.n >> 2); w += blockDim.x) reinterpret_cast<u32*>(small)[w] = __ldg(src + w);
+      // the barrier that opens the forward transform publishes the copy
     }
     u64* h0 = a < 0 ? park : shares + ((((size_t)irec * n_parties + a) * n_cts + cl) * 2) * poly + row;
     u64* h1 = h0 + poly;
@@ -150,7 +165,6 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
           [&](u32 j, u64 val) { out[j] = add_small_canon<WIDE>(val, (int)e[j], lt); });
     }
   }
-  cluster.sync();
 }
 
 // ct' = (c_0 + sum_k h_{0,k}, sum_k h_{1,k}).  grid = (n_rec * n_cts, chunks); two residues per thread.
@@ -164,6 +178,7 @@ __global__ void __launch_bounds__(256)
   for (size_t e = (size_t)blockIdx.y * blockDim.x + threadIdx.x; e < ct_pairs;
        e += (size_t)gridDim.y * blockDim.x) {
     const u32 l = (u32)(((e * 2) >> v.logn) % v.L);
+    if (!D2MHE_CHK(v.chk, e, ct_pairs, SITE_ELEMENT)) continue;
     const u64 p = v.limbs[l].p;
     ulonglong2 acc = (e < ct_pairs / 2) ? __ldg(in0 + e) : make_ulonglong2(0, 0);  // c_0 only
     for (u32 k = 0; k < n_shares; ++k) {
@@ -184,6 +199,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
                      const u32* __restrict__ users, u32 n_cts, u64* prod) {
   const u32 l = blockIdx.x % v.L, unit = blockIdx.x / v.L;
   const u32 user = users[unit / n_cts];
+  if (!D2MHE_CHK(v.chk, user, v.K, SITE_PARTY)) return;
   const LimbTab& lt = lp.limbs[l];
   u64* sm = poly_smem();
   const size_t row = (size_t)l * v.n, poly = (size_t)v.L * v.n;
@@ -207,18 +223,43 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 
 }  // namespace
 
-namespace d2mhe_launch {
+namespace D2MHE_LAUNCH_NS {
 
 cudaError_t user_keygen(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* users_dev,
                         u32 n_users) {
   D2MHE_DISPATCH(k_user_keygen, v, n_users * v.L, s, v, lp, users_dev);
 }
 
+static cudaError_t convert_share_units(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
+                                       const u32* recipients_dev, const u32* parties_dev, u32 n_parties, u32 n_cts,
+                                       u32 unit_first, u32 n_units, const u32* sampled, u64* shares) {
+  D2MHE_DISPATCH_EX(k_convert_share, v, n_units * v.L, s, 3 * (size_t)v.n, 1, v, lp, agg, recipients_dev, parties_dev,
+                    n_parties, n_cts, unit_first, sampled, shares);
+}
+
+// scratch: at least n_parties * 3 N bytes; (recipient, ciphertext) units are processed in batches of as
+// many as it holds.
 cudaError_t convert_share(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
                           const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties,
-                          u32 ct_first, u32 n_cts, u64* shares) {
-  D2MHE_DISPATCH_EX(k_convert_share, v, n_rec * n_cts * v.L, s, 3 * (size_t)v.n, cluster_size_for(v.L, v.logn), v,
-                    lp, agg, recipients_dev, parties_dev, n_parties, ct_first, n_cts, shares);
+                          u32 ct_first, u32 n_cts, u64* shares, void* scratch, size_t scratch_bytes, u32* launches) {
+  const size_t per_unit = (size_t)n_parties * 3 * v.n;
+  const u32 n_units = n_rec * n_cts;
+  const u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
+  if (launches) *launches = 0;
+  if (per_batch == 0) return cudaErrorInvalidValue;
+  for (u32 first = 0; first < n_units; first += per_batch) {
+    const u32 nu = std::min(per_batch, n_units - first);
+    const size_t words = (size_t)nu * per_unit / 4;
+    k_sample_convert_noise<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(
+        v, recipients_dev, parties_dev, n_parties, ct_first, n_cts, first, nu, reinterpret_cast<u32*>(scratch));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    e = convert_share_units(v, lp, s, agg, recipients_dev, parties_dev, n_parties, n_cts, first, nu,
+                            reinterpret_cast<const u32*>(scratch), shares);
+    if (e != cudaSuccess) return e;
+    if (launches) *launches += 2;
+  }
+  return cudaSuccess;
 }
 
 cudaError_t convert_combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
@@ -236,4 +277,4 @@ cudaError_t secret_product(const DevView& v, const LimbParams& lp, cudaStream_t 
   D2MHE_DISPATCH(k_secret_product, v, n_users * n_cts * v.L, s, v, lp, ct, users_dev, n_cts, prod);
 }
 
-}  // namespace d2mhe_launch
+}  // namespace D2MHE_LAUNCH_NS

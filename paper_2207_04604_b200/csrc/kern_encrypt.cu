@@ -21,6 +21,7 @@ __global__ void __launch_bounds__(256)
   if (e >= total) return;
   const u32 w = (u32)(e % words), which = (u32)((e / words) % 3), unit = unit_first + (u32)(e / (3 * (size_t)words));
   const u32 party = parties[unit / n_cts], c = ct_first + unit % n_cts;
+  if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY)) return;
   const Stream st(v.seed, which == 0 ? TAG_ENC_U : which == 1 ? TAG_ENC_E0 : TAG_ENC_E1, c, party, 0);
   u32 pack = 0;
   if (which == 0) {
@@ -83,7 +84,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 
 }  // namespace
 
-namespace d2mhe_launch {
+namespace D2MHE_LAUNCH_NS {
 
 static cudaError_t encrypt_units(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 unit_first, u32 n_units,
                                  const u32* sampled, const u32* plain, u64* ct) {
@@ -113,4 +114,4 @@ cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, cons
   return cudaSuccess;
 }
 
-}  // namespace d2mhe_launch
+}  // namespace D2MHE_LAUNCH_NS

@@ -8,6 +8,7 @@ template <int LOGN, int G, bool WIDE>
 __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
     k_keygen(DevView v, const __grid_constant__ LimbParams lp, const u32* __restrict__ parties) {
   const u32 l = blockIdx.x % v.L, party = parties[blockIdx.x / v.L];
+  if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY)) return;
   const LimbTab& lt = lp.limbs[l];
   const Stream st(v.seed, TAG_SECRET, 0, party, 0);
   u64* out = v.s_mont + ((size_t)party * v.L + l) * v.n;
@@ -57,6 +58,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
   }
   for (u32 a = 0; a < n_parties; ++a) {
     const u32 party = parties[a];
+    if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY)) continue;
     const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
     const Stream se(v.seed, TAG_PK_ERR, 0, party, 0);
     u64* share = shares_out ? shares_out + ((size_t)a * v.L + l) * v.n : nullptr;
@@ -107,9 +109,18 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
       });
 }
 
+// Test hook of the checked build: the index test on an index equal to its limit.  Touches no memory
+// beyond the check words; compiles to an empty kernel without D2MHE_CHECKED.
+__global__ void k_check_selftest(DevView v) { (void)D2MHE_CHK(v.chk, 1, 1, SITE_SELFTEST); }
+
 }  // namespace
 
-namespace d2mhe_launch {
+namespace D2MHE_LAUNCH_NS {
+
+cudaError_t check_selftest(const DevView& v, cudaStream_t s) {
+  k_check_selftest<<<1, 1, 0, s>>>(v);
+  return cudaGetLastError();
+}
 
 cudaError_t export_secret(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* key, signed char* out) {
   D2MHE_DISPATCH(k_export_secret, v, v.L, s, v, lp, key, out);
@@ -124,4 +135,4 @@ cudaError_t collective_pk(const DevView& v, const LimbParams& lp, cudaStream_t s
   D2MHE_DISPATCH(k_collective_pk, v, v.L, s, v, lp, parties_dev, n_parties, shares_out);
 }
 
-}  // namespace d2mhe_launch
+}  // namespace D2MHE_LAUNCH_NS

@@ -55,6 +55,7 @@ __global__ void __launch_bounds__(256)
   const Mod md(lt);
   const u32 o = (blockIdx.x & 15u) * blockDim.x + threadIdx.x;  // < 4096
   u64* row = polys + (size_t)r * v.n + o;
+  if (!D2MHE_CHK(v.chk, (size_t)o + ((size_t)(R - 1) << 12), v.n, SITE_LOAD)) return;
   u64 x[R];
 #pragma unroll
   for (int k = 0; k < R; ++k) x[k] = row[(size_t)k << 12];
@@ -127,7 +128,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 
 }  // namespace
 
-namespace d2mhe_launch {
+namespace D2MHE_LAUNCH_NS {
 
 static cudaError_t ntt_two_pass(const DevView& v, const LimbParams& lp, cudaStream_t s, u64* polys,
                                 u32 batch, bool inverse) {
@@ -165,4 +166,4 @@ cudaError_t ntt(const DevView& v, const LimbParams& lp, cudaStream_t s, u64* pol
   }
 }
 
-}  // namespace d2mhe_launch
+}  // namespace D2MHE_LAUNCH_NS

@@ -84,6 +84,7 @@ __global__ void __launch_bounds__(256) k_muladd32(DevView v, const u32* __restri
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_quads; e += stride) {
     const u32 l = (u32)(((e * 4) >> v.logn) % v.L);
+    if (!D2MHE_CHK(v.chk, e, n_quads, SITE_ELEMENT) || !D2MHE_CHK(v.chk, l, v.L, SITE_LIMB)) continue;
     const LimbTab* lt = v.limbs + l;
     const u64 p = lt->p, one_sh = lt->one_sh;
     const uint4 av = reinterpret_cast<const uint4*>(a)[e];
@@ -110,7 +111,7 @@ cudaError_t launch_ntt32(const DevView& v, const LimbParams& lp, cudaStream_t s,
 
 }  // namespace
 
-namespace d2mhe_launch {
+namespace D2MHE_LAUNCH_NS {
 
 cudaError_t ntt32(const DevView& v, const LimbParams& lp, cudaStream_t s, u32* polys, u32 batch, bool inverse) {
   switch (v.logn) {
@@ -132,4 +133,4 @@ cudaError_t muladd32(const DevView& v, cudaStream_t s, const u32* a, const u32* 
   return cudaGetLastError();
 }
 
-}  // namespace d2mhe_launch
+}  // namespace D2MHE_LAUNCH_NS

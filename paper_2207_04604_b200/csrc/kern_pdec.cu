@@ -27,7 +27,9 @@ __global__ void __launch_bounds__(256)
   const u32 w = (u32)(e % words);
   const size_t share = e / words;
   const u32 a = (u32)(share % n_parties), unit = unit_first + (u32)(share / n_parties);
-  const Stream se(v.seed, TAG_DEC_ERR, ct_first + unit % n_cts, parties[a], recipients[unit / n_cts]);
+  const u32 party = parties[a], recipient = recipients[unit / n_cts];
+  if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY) || !D2MHE_CHK(v.chk, recipient, v.K, SITE_PARTY)) return;
+  const Stream se(v.seed, TAG_DEC_ERR, ct_first + unit % n_cts, party, recipient);
   u32 pack = 0;
 #pragma unroll
   for (u32 b = 0; b < 4; ++b) pack |= ((u32)gauss_from_r(gt, se.draw64(4 * w + b)) & 0xffu) << (8 * b);
@@ -53,7 +55,9 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
       [&](int, u32 q, u64(&x)[8]) { store_octet(park + 8 * (size_t)q, x); });
 #pragma unroll 1
   for (u32 a = 0; a < n_parties; ++a) {
-    const u64* sk = v.s_mont + ((size_t)parties[a] * v.L + l) * v.n;
+    const u32 party = parties[a];
+    if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY)) continue;
+    const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
     // Buffer a & 1 was last read in the final round of share a - 2, which every thread left before
     // it passed the barrier that opens the transform of share a - 1; the barrier that opens this
     // share's transform publishes the copy.
@@ -78,7 +82,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 
 }  // namespace
 
-namespace d2mhe_launch {
+namespace D2MHE_LAUNCH_NS {
 
 static cudaError_t pdec_pre_units(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
                                   const u32* parties_dev, u32 n_parties, u32 n_cts, u32 unit_first,
@@ -114,4 +118,4 @@ cudaError_t partial_decrypt_scratch(const DevView& v, const LimbParams& lp, cuda
   return cudaSuccess;
 }
 
-}  // namespace d2mhe_launch
+}  // namespace D2MHE_LAUNCH_NS

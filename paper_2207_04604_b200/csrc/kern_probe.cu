@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(256, 4)
 
 }  // namespace
 
-namespace d2mhe_launch {
+namespace D2MHE_LAUNCH_NS {
 
 // Runs the loop `kind` for `iters` iterations between two events on stream s and returns the
 // elapsed milliseconds and the number of lane operations (kind 0-2: multiply instructions x 32
@@ -113,4 +113,4 @@ cudaError_t int_probe(const DevView& v, const LimbParams& lp, cudaStream_t s, u3
   return e;
 }
 
-}  // namespace d2mhe_launch
+}  // namespace D2MHE_LAUNCH_NS

@@ -11,6 +11,7 @@ __global__ void __launch_bounds__(256) k_muladd(DevView v, const u64* __restrict
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_pairs; e += stride) {
     const u32 l = (u32)(((e * 2) >> v.logn) % v.L);
+    if (!D2MHE_CHK(v.chk, e, n_pairs, SITE_ELEMENT) || !D2MHE_CHK(v.chk, l, v.L, SITE_LIMB)) continue;
     const LimbTab* lt = v.limbs + l;
     const u64 p = lt->p, pinv = lt->pinv, r = lt->rmod, rs = lt->rmod_sh;
     const ulonglong2 av = reinterpret_cast<const ulonglong2*>(a)[e];
@@ -39,6 +40,7 @@ __global__ void __launch_bounds__(256)
     // block-uniform index so that the division runs on the uniform datapath
     const size_t e_row = v.n >= 512 ? e - threadIdx.x : e;
     const u32 l = (u32)(((e_row * 2) >> v.logn) % v.L);
+    if (!D2MHE_CHK(v.chk, e, ct_pairs, SITE_ELEMENT) || !D2MHE_CHK(v.chk, l, v.L, SITE_LIMB)) continue;
     const u64 p = v.limbs[l].p;
     ulonglong2 acc = make_ulonglong2(0, 0);
     for (u32 a = beg; a < end; ++a) {
@@ -69,6 +71,7 @@ __global__ void __launch_bounds__(256, LMAX <= 8 ? 8 : 3)
   const u32 j = blockIdx.y * blockDim.x + threadIdx.x;
   if (j >= v.n) return;
   const u32 L = v.L;
+  if (!D2MHE_CHK(v.chk, L, (u32)LMAX + 1u, SITE_LIMB)) return;
   const size_t poly = (size_t)L * v.n;
   const u64* c0 = agg + (size_t)unit * 2 * poly;
   const bool lazy = v.wide != 0 && n_shares < 120;
@@ -157,7 +160,8 @@ __global__ void __launch_bounds__(1024)
     bad |= (val > (int32_t)pt.half) || (val < -(int32_t)pt.half);
     int32_t r = val % (int32_t)t;
     if (r < 0) r += (int32_t)t;
-    sm[__brev(j) >> (32 - logn)] = (u32)r;
+    const u32 pos = __brev(j) >> (32 - logn);
+    if (D2MHE_CHK(v.chk, pos, n, SITE_STAGED)) sm[pos] = (u32)r;
   }
   if (bad) atomicOr(v.range_flag, 1u);
   __syncthreads();
@@ -167,6 +171,7 @@ __global__ void __launch_bounds__(1024)
     for (u32 b = threadIdx.x; b < (n >> 2); b += blockDim.x) {
       const u32 i2 = b >> lt, jj = b & (span - 1);
       const u32 base = (i2 << (lt + 2)) + jj;
+      if (!D2MHE_CHK(v.chk, base + 3 * span, n, SITE_STAGED) || !D2MHE_CHK(v.chk, m + 2 * i2 + 1, n, SITE_TWIDDLE)) continue;
       u32 x0 = sm[base], x1 = sm[base + span], x2 = sm[base + 2 * span], x3 = sm[base + 3 * span];
       gs32(x0, x1, __ldg(pt.IW + m + 2 * i2), t, twot);
       gs32(x2, x3, __ldg(pt.IW + m + 2 * i2 + 1), t, twot);
@@ -225,6 +230,7 @@ __global__ void __launch_bounds__(1024)
     for (u32 b = threadIdx.x; b < (n >> 2); b += blockDim.x) {
       const u32 i2 = b >> (lt - 1), jj = b & (span - 1);
       const u32 base = (i2 << (lt + 1)) + jj;
+      if (!D2MHE_CHK(v.chk, base + 3 * span, n, SITE_STAGED) || !D2MHE_CHK(v.chk, 2 * m2 + 2 * i2 + 1, n, SITE_TWIDDLE)) continue;
       u32 x0 = sm[base], x1 = sm[base + span], x2 = sm[base + 2 * span], x3 = sm[base + 3 * span];
       const uint2 w = __ldg(pt.W + m2 + i2);
       ct32(x0, x2, w, t, twot);
@@ -239,14 +245,16 @@ __global__ void __launch_bounds__(1024)
     __syncthreads();
   }
   for (u32 j = threadIdx.x; j < n; j += blockDim.x) {
-    const u32 y = csub32(csub32(sm[__brev(j) >> (32 - logn)], twot), t);
+    const u32 pos = __brev(j) >> (32 - logn);
+    if (!D2MHE_CHK(v.chk, pos, n, SITE_STAGED)) continue;
+    const u32 y = csub32(csub32(sm[pos], twot), t);
     out[j] = y > pt.half ? (int32_t)y - (int32_t)t : (int32_t)y;
   }
 }
 
 }  // namespace
 
-namespace d2mhe_launch {
+namespace D2MHE_LAUNCH_NS {
 
 cudaError_t muladd(const DevView& v, cudaStream_t s, const u64* a, const u64* b, const u64* c,
                    u64* d, u32 batch) {
@@ -297,4 +305,4 @@ cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts
   return cudaGetLastError();
 }
 
-}  // namespace d2mhe_launch
+}  // namespace D2MHE_LAUNCH_NS

@@ -23,6 +23,7 @@ ERR_CUDA = -5
 ERR_RANGE = -6
 ERR_UNSUPPORTED = -7
 ERR_DEVICE_CHECK = -8
+FLAG_DEVICE_CHECKS = 1
 
 EXPORTS = [
     "d2mhe_create", "d2mhe_destroy", "d2mhe_set_stream", "d2mhe_sync", "d2mhe_strerror",
@@ -31,7 +32,8 @@ EXPORTS = [
     "d2mhe_ntt_inverse", "d2mhe_poly_muladd", "d2mhe_ntt32_forward", "d2mhe_ntt32_inverse",
     "d2mhe_poly_muladd32", "d2mhe_round_workspace_bytes", "d2mhe_round_plan", "d2mhe_round_device",
     "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_user_keygen", "d2mhe_convert_share",
-    "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_bootstrap_share", "d2mhe_bootstrap_combine", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_debug_int_throughput", "d2mhe_get_root", "d2mhe_get_plain_root",
+    "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_bootstrap_share", "d2mhe_bootstrap_combine", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_debug_int_throughput", "d2mhe_debug_last_device_check",
+    "d2mhe_debug_check_selftest", "d2mhe_get_root", "d2mhe_get_plain_root",
     "d2mhe_launch_count",
 ]
 
@@ -107,6 +109,8 @@ def load():
         lib.d2mhe_bootstrap_share.argtypes = [vp, vp, vp, u32, vp, u32, u32, u32, vp]
         lib.d2mhe_bootstrap_combine.argtypes = [vp, vp, vp, vp, u32, u32, u32, u32, vp, vp]
         lib.d2mhe_debug_int_throughput.argtypes = [vp, u32, u32, ctypes.POINTER(ctypes.c_double)]
+        lib.d2mhe_debug_last_device_check.argtypes = [vp, vp]
+        lib.d2mhe_debug_check_selftest.argtypes = [vp]
         lib.d2mhe_get_root.argtypes = [vp, u32, ctypes.POINTER(u64)]
         lib.d2mhe_get_plain_root.argtypes = [vp, ctypes.POINTER(u64)]
         lib.d2mhe_launch_count.argtypes = [vp]
@@ -156,7 +160,7 @@ U64 = torch.int64
 class Context:
     """d2mhe_ctx.  Methods are the C calls with the same names (without the prefix)."""
 
-    def __init__(self, log2_n, moduli, num_parties, seed, plain_modulus=65537, device=0, gauss_bound=19):
+    def __init__(self, log2_n, moduli, num_parties, seed, plain_modulus=65537, device=0, gauss_bound=19, flags=0):
         lib = load()
         self.log2_n, self.n = int(log2_n), 1 << int(log2_n)
         self.moduli = [int(m) for m in moduli]
@@ -169,7 +173,7 @@ class Context:
         p.log2_n, p.num_limbs, p.num_parties = self.log2_n, self.num_limbs, self.num_parties
         p.moduli = ctypes.cast(self._moduli_arr, ctypes.POINTER(ctypes.c_uint64))
         p.plain_modulus, p.seed = self.t, int(seed)
-        p.gauss_bound, p.flags, p.device = gauss_bound, 0, device
+        p.gauss_bound, p.flags, p.device = gauss_bound, flags, device
         self._params = p
         self._h = ctypes.c_void_p()
         st = lib.d2mhe_create(ctypes.byref(p), ctypes.byref(self._h))
@@ -347,6 +351,14 @@ class Context:
         self._check(load().d2mhe_debug_int_throughput(self._h, kind, iters, ctypes.byref(v)),
                     "d2mhe_debug_int_throughput")
         return float(v.value)
+
+    def debug_last_device_check(self):
+        out = (ctypes.c_uint32 * 4)()
+        self._check(load().d2mhe_debug_last_device_check(self._h, out), "d2mhe_debug_last_device_check")
+        return [int(x) for x in out]
+
+    def debug_check_selftest(self):
+        self._check(load().d2mhe_debug_check_selftest(self._h), "d2mhe_debug_check_selftest")
 
     def get_root(self, limb):
         v = ctypes.c_uint64()

@@ -941,3 +941,97 @@ def test_error_statuses(d2):
     assert status(big.keygen_share, [0]) == d2.ERR_UNSUPPORTED
     big.close()
     ctx.close()
+
+
+# ----------------------------------------------------------------------------------
+# the checked kernel build (D2MHE_FLAG_DEVICE_CHECKS)
+# ----------------------------------------------------------------------------------
+
+
+def test_checked_build_gives_the_same_messages_and_reports_nothing(d2):
+    """Every kernel of the checked build (index tests on coefficient, octet, shared-memory, twiddle and
+    party indices) on a small ring, on configuration 1, on the conversion and refresh calls and on the
+    stand-alone transforms: the same bit-exact messages, and no violation recorded."""
+    log2_n, K = 6, 3
+    moduli = small_moduli(log2_n, 54, 2)
+    ctx = d2.Context(log2_n, moduli, K, seed=5, flags=d2.FLAG_DEVICE_CHECKS)
+    o = make_oracle(log2_n, moduli, seed=5)
+    values = np.random.default_rng(2).integers(-3000, 3001, size=(K, 2, 1 << log2_n)).astype(np.int32)
+    offsets = np.array([0, K, K, K + 1], dtype=np.uint32)
+    rows = np.array(list(range(K)) + [K - 1], dtype=np.uint32)
+    _run_round(d2, ctx, o, K, list(range(K)), offsets, rows, values, ct_first=3)
+    ctx.sync()
+    ctx.close()
+
+    cfg = wl.round_config(1)
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, cfg.num_parties, seed=2, flags=d2.FLAG_DEVICE_CHECKS)
+    o = make_oracle(cfg.log2_n, cfg.moduli, seed=2)
+    offsets, rows = wl.regular_graph(cfg.num_parties, cfg.degree, 2)
+    values = wl.gradients(cfg, 2)
+    want = {}
+    parties = list(range(cfg.num_parties))
+    _run_round(d2, ctx, o, cfg.num_parties, parties, offsets, rows, values, 0, keep=want)
+    _check_whole_round_call(d2, ctx, cfg, offsets, rows, values, want)
+    K, L, n = cfg.num_parties, cfg.num_limbs, cfg.n
+    # conversion and refresh shares through the checked kernels
+    agg = d2.from_u64_numpy(want["agg"][:2, :1].copy(), ctx.device)
+    ctx.user_keygen([0, 1])
+    sh = ctx.empty_u64(2, K, 1, 2, L, n)
+    ctx.convert_share(agg, [0, 1], parties, 0, 1, sh)
+    pk_users = np.stack([o.user_pk(i) for i in (0, 1)])
+    assert np.array_equal(d2.to_u64_numpy(sh), o.convert_share(want["agg"][:2, :1], pk_users, [0, 1], parties, 0))
+    ctx.bootstrap_share(agg, [0, 1], parties, 0, 1, sh)
+    assert np.array_equal(d2.to_u64_numpy(sh), o.boot_share(want["agg"][:2, :1], [0, 1], parties, 0))
+    # stand-alone transforms and multiply-add
+    polys = wl.random_polys(cfg.moduli, cfg.log2_n, 3, seed=9)
+    dp = d2.from_u64_numpy(polys, ctx.device)
+    ctx.ntt_forward(dp, 3)
+    ctx.ntt_inverse(dp, 3)
+    assert np.array_equal(d2.to_u64_numpy(dp), polys)
+    ctx.poly_muladd(dp, dp, dp, dp, 3)
+    ctx.sync()  # D2MHE_ERR_DEVICE_CHECK would raise here
+    ctx.close()
+    # the two-pass transforms (N = 2^15) and the 32-bit-word calls
+    big = d2.Context(15, wl.ntt_primes(54, 1 << 16, 2), 1, seed=1, flags=d2.FLAG_DEVICE_CHECKS)
+    polys = wl.random_polys(big.moduli, 15, 2, seed=3)
+    dp = d2.from_u64_numpy(polys, big.device)
+    big.ntt_forward(dp, 2)
+    big.ntt_inverse(dp, 2)
+    assert np.array_equal(d2.to_u64_numpy(dp), polys)
+    big.sync()
+    big.close()
+    narrow = d2.Context(12, small_moduli(12, 30, 2), 1, seed=1, flags=d2.FLAG_DEVICE_CHECKS)
+    p32 = wl.random_polys(narrow.moduli, 12, 3, seed=4).astype(np.uint32)
+    d32 = d2.from_u32_numpy(p32, narrow.device)
+    narrow.ntt32_forward(d32, 3)
+    narrow.ntt32_inverse(d32, 3)
+    assert np.array_equal(d2.to_u32_numpy(d32), p32)
+    narrow.sync()
+    narrow.close()
+
+
+def test_checked_build_reports_a_violation_without_losing_the_context(d2):
+    """The self-test hook runs the index test on an index equal to its limit (no memory is touched):
+    the next sync reports it once, with its site, index and limit, and the context keeps working.
+    Without the flag the same hook does nothing."""
+    cfg = wl.round_config(1)
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, 2, seed=1, flags=d2.FLAG_DEVICE_CHECKS)
+    ctx.sync()
+    ctx.debug_check_selftest()
+    with pytest.raises(d2.D2mheError) as e:
+        ctx.sync()
+    assert e.value.status == d2.ERR_DEVICE_CHECK
+    assert ctx.debug_last_device_check() == [15, 1, 1, 0]
+    ctx.sync()  # reported once, then cleared
+    polys = wl.random_polys(cfg.moduli, cfg.log2_n, 2, seed=1)
+    dp = d2.from_u64_numpy(polys, ctx.device)
+    ctx.ntt_forward(dp, 2)
+    ctx.ntt_inverse(dp, 2)
+    assert np.array_equal(d2.to_u64_numpy(dp), polys)
+    ctx.sync()
+    ctx.close()
+    plain = d2.Context(cfg.log2_n, cfg.moduli, 2, seed=1)
+    plain.debug_check_selftest()
+    plain.sync()
+    assert plain.debug_last_device_check() == [0, 0, 0, 0]
+    plain.close()

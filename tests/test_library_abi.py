@@ -59,6 +59,21 @@ def test_create_rejects_bad_arguments_before_touching_the_device():
     p.plain_modulus = 65536
     assert lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h)) == d2mhe.ERR_BAD_PARAMS
     assert not h.value
+    # flags: bit 0 (device-side index checks) is accepted, every other bit is refused
+    p.plain_modulus = 65537
+    p.flags = 2
+    assert lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h)) == d2mhe.ERR_BAD_PARAMS
+    p.flags = d2mhe.FLAG_DEVICE_CHECKS | 4
+    assert lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h)) == d2mhe.ERR_BAD_PARAMS
+    p.flags = d2mhe.FLAG_DEVICE_CHECKS
+    st = lib.d2mhe_create(ctypes.byref(p), ctypes.byref(h))
+    import torch
+
+    if torch.cuda.is_available():
+        assert st == d2mhe.OK
+        lib.d2mhe_destroy(h)
+    else:
+        assert st == d2mhe.ERR_CUDA and not h.value  # the parameters passed validation; there is no device here
 
 
 def test_round_plan_invariants():
