@@ -554,6 +554,71 @@ def convert_bootstrap_bench(ctx, cfg, dev, stream, flush, offsets, rows, seed):
             "share_bytes": units * S * 2 * 8 * n * L}
 
 
+def narrow_round_bench(args, local_rank):
+    """The MNIST-shaped round on seven 30-bit limbs (log q = 210 against 216) through the 32-bit-word
+    protocol calls, call by call on one stream, and the same parameter set through the 64-bit-word
+    calls: a separate, labelled line (the benchmark configurations fix their 54-bit primes)."""
+    import torch
+
+    from paper_2207_04604_b200 import d2mhe
+
+    cfg = wl.narrow_round_config()
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream(dev)
+    K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, cfg.num_cts
+    parties = list(range(K))
+    offsets, rows = wl.regular_graph(K, cfg.degree, args.seed)
+    ctx = d2mhe.Context(cfg.log2_n, cfg.moduli, K, seed=args.seed, device=local_rank)
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    values = torch.from_numpy(wl.gradients(cfg, args.seed)).to(dev)
+    flush = torch.empty(384 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    idx = [torch.as_tensor(rows[offsets[i]:offsets[i + 1]].astype(np.int64), device=dev) for i in range(K)]
+    plain, out_plain = ctx.empty_u32(K, C, n), ctx.empty_u32(K, C, n)
+    sums = torch.empty((K, C, n), dtype=torch.int32, device=dev)
+    names = ["encode", "encrypt", "aggregate", "partial_decrypt", "combine_decrypt", "decode"]
+
+    def run(words32, reps=10):
+        mk = ctx.empty_u32 if words32 else ctx.empty_u64
+        ct, agg, sh = mk(K, C, 2, L, n), mk(K, C, 2, L, n), mk(K, K, C, L, n)
+        calls = [lambda: ctx.encode(values, K * C, plain),
+                 (lambda: ctx.encrypt32(parties, 0, C, plain, ct)) if words32 else (lambda: ctx.encrypt(parties, 0, C, plain, ct)),
+                 (lambda: ctx.aggregate32(ct, K, C, offsets, rows, agg)) if words32 else (lambda: ctx.aggregate(ct, K, C, offsets, rows, agg)),
+                 (lambda: ctx.partial_decrypt32(agg, parties, parties, 0, C, sh)) if words32 else (lambda: ctx.partial_decrypt(agg, parties, parties, 0, C, sh)),
+                 (lambda: ctx.combine_decrypt32(agg, sh, K, K, C, out_plain)) if words32 else (lambda: ctx.combine_decrypt(agg, sh, K, K, C, out_plain)),
+                 lambda: ctx.decode(out_plain, K * C, sums)]
+        per = [0.0] * len(calls)
+        total = 0.0
+        for it in range(reps + 3):
+            flush.zero_()
+            marks = [torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)]
+            marks[0].record(stream)
+            for i, fn in enumerate(calls):
+                fn()
+                marks[i + 1].record(stream)
+            torch.cuda.synchronize(dev)
+            if it == 0 and not all(bool(torch.equal(sums[i], values[idx[i]].sum(dim=0, dtype=torch.int32))) for i in range(K)):
+                raise RuntimeError("narrow round: decrypted sums differ from the plaintext sums")
+            if it >= 3:
+                total += marks[0].elapsed_time(marks[-1])
+                for i in range(len(calls)):
+                    per[i] += marks[i].elapsed_time(marks[i + 1])
+        return total / reps, {nm: t / reps for nm, t in zip(names, per)}
+
+    ms32, per32 = run(True)
+    ms64, per64 = run(False)
+    lo = max(ctx.debug_int_throughput(0, 4096) for _ in range(3))
+    t32 = 4 * (n // 2) * cfg.log2_n  # one high and two low multiplies per 32-bit butterfly
+    slots_pdec = K * C * (L * (t32 + K * (t32 + 4 * n)) + K * 40 * n)
+    coeffs = coeffs_of(cfg, 0, C)
+    ctx.close()
+    return {"config": config_dict(cfg), "note": "call by call on one stream; not the headline (its primes are not the benchmark's)",
+            "words32": {"ms_per_round": ms32, "value": coeffs / (ms32 * 1e-3), "unit": UNIT, "calls_ms": per32,
+                        "partial_decrypt_alu_frac": slots_pdec / (per32["partial_decrypt"] * 1e-3) / lo,
+                        "slots_per_butterfly": 4},
+            "words64_same_primes": {"ms_per_round": ms64, "value": coeffs / (ms64 * 1e-3), "unit": UNIT, "calls_ms": per64}}
+
+
 def run_cuda(args, cfg):
     import torch
 
@@ -583,6 +648,11 @@ def run_cuda(args, cfg):
                                "unit": UNIT, "steps": 10, "warmup": 3, "sub_chunks": r2["sub_chunks"],
                                "round_hbm_frac": sum(algorithmic_bytes(c2, c2.num_cts).values()) / 1e9
                                / (r2["ms_per_step"] * 1e-3) / measured_peaks()[0]}
+
+    narrow = None
+    if rank == 0 and world == 1 and not args.no_other_configs and not args.cts:
+        torch.cuda.empty_cache()
+        narrow = narrow_round_bench(args, local_rank)
 
     if rank == 0:
         K, L, n, C = cfg.num_parties, cfg.num_limbs, cfg.n, res["C"]
@@ -673,6 +743,7 @@ def run_cuda(args, cfg):
             "ntt": ntt,
             "convert_bootstrap": cb,
             "other_configs": others,
+            "narrow_words": narrow,
             "init_ms": res["init_ms"],
             "wall_ms_per_step_incl_flush": res["wall_ms_per_step_incl_flush"],
             "cpu_baseline": cpu_baseline(cfg, args.seed) if world == 1 and not args.no_cpu_baseline else None,

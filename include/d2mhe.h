@@ -252,6 +252,29 @@ d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* ctx, const uint32_t* a_dev, const ui
                                  const uint32_t* c_dev, uint32_t* d_dev, uint32_t batch);
 
 /*
+ * The protocol calls on 32-bit words, for the same parameter sets (every prime below 2^30,
+ * log2_n <= 14; D2MHE_ERR_UNSUPPORTED otherwise): ciphertexts, neighbour sums and decryption shares
+ * are uint32 arrays of the shapes given above, residues in [0, q_l).  Keys come from
+ * d2mhe_keygen_share and d2mhe_collective_pk as before; plaintexts from d2mhe_encode and to
+ * d2mhe_decode.  Streams, samples and every result equal those of the 64-bit calls on the same
+ * context (BFV.Encrypt, Sec. 3.2 item 3; BFV.Add, item 4; decryption shares and their combination,
+ * Sec. 4.2 item 3 and Sec. 3.2 item 5).  Two units share a thread block, so even counts of
+ * (party, ciphertext) and (recipient, ciphertext) pairs use the GPU best.
+ */
+d2mhe_status d2mhe_encrypt32(d2mhe_ctx* ctx, const uint32_t* parties, uint32_t n_parties,
+                             uint32_t ct_first, uint32_t n_cts, const uint32_t* plain_dev,
+                             uint32_t* ct_dev);
+d2mhe_status d2mhe_aggregate32(d2mhe_ctx* ctx, const uint32_t* ct_dev, uint32_t n_rows, uint32_t n_cts,
+                               const uint32_t* nbr_offsets, const uint32_t* nbr_rows, uint32_t n_out,
+                               uint32_t* agg_dev);
+d2mhe_status d2mhe_partial_decrypt32(d2mhe_ctx* ctx, const uint32_t* agg_dev, const uint32_t* recipients,
+                                     uint32_t n_rec, const uint32_t* parties, uint32_t n_parties,
+                                     uint32_t ct_first, uint32_t n_cts, uint32_t* shares_dev);
+d2mhe_status d2mhe_combine_decrypt32(d2mhe_ctx* ctx, const uint32_t* agg_dev, const uint32_t* shares_dev,
+                                     uint32_t n_rec, uint32_t n_shares, uint32_t n_cts,
+                                     uint32_t* plain_dev);
+
+/*
  * One whole private gradient update for ciphertext indices ct_first .. ct_first+n_cts-1
  * of all K parties (Algorithm 2 from encryption to decryption, without the model update): encode,
  * encrypt, neighbour sums, shares from every share holder, combine, decode.  Ciphertext

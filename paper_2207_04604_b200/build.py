@@ -7,7 +7,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libd2mhe.so")
-SOURCES = ["kern_pdec.cu", "kern_encrypt.cu", "kern_ntt.cu", "kern_ntt32.cu", "kern_keys.cu", "kern_stream.cu", "kern_convert.cu", "kern_bootstrap.cu", "kern_probe.cu", "d2mhe_host.cu",
+SOURCES = ["kern_pdec.cu", "kern_encrypt.cu", "kern_ntt.cu", "kern_ntt32.cu", "kern_keys.cu", "kern_stream.cu", "kern_convert.cu", "kern_bootstrap.cu", "kern_probe.cu", "kern_proto32.cu", "d2mhe_host.cu",
            "d2mhe_round_static.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

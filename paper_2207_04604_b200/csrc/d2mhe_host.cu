@@ -396,6 +396,12 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   if (err != cudaSuccess) return fail_cuda(c, err);
   c->view.upk_coef = dev_alloc<u64>(c, (size_t)P.num_parties * 2 * poly, &err);
   if (err != cudaSuccess) return fail_cuda(c, err);
+  if (c->narrow && P.log2_n <= D2MHE_MAX_SMEM_LOGN) {
+    c->view.s32 = dev_alloc<u64>(c, (size_t)P.num_parties * poly, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    c->view.pk32 = dev_alloc<u64>(c, 2 * poly, &err);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+  }
   c->noise_scratch_bytes = kNoiseScratchBytes;
   c->noise_scratch = dev_alloc<unsigned char>(c, c->noise_scratch_bytes, &err);
   if (err != cudaSuccess) return fail_cuda(c, err);
@@ -595,6 +601,15 @@ d2mhe_status d2mhe_keygen_share(d2mhe_ctx* c, const u32* parties, u32 n_parties)
   cudaError_t e = L_(keygen)(c->view, c->limb_params, c->stream, sg.dev[0], n_parties);
   if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
+  if (c->view.s32) {  // the same key shares in the form the 32-bit-word calls read
+    const size_t poly = (size_t)c->view.L * c->view.n;
+    for (u32 i = 0; i < n_parties; ++i) {
+      e = L_(make_tab32)(c->view, c->stream, c->view.s_mont + parties[i] * poly, c->view.s32 + parties[i] * poly,
+                         c->view.L);
+      if (e != cudaSuccess) return fail_staged(c, sg, e);
+      c->launches += 1;
+    }
+  }
   for (u32 i = 0; i < n_parties; ++i) c->has_share[parties[i]] = true;
   return release_slot(c, sg);
 }
@@ -615,6 +630,11 @@ d2mhe_status d2mhe_collective_pk(d2mhe_ctx* c, const u32* parties, u32 n_parties
                                               reinterpret_cast<u64*>(pk_shares_dev));
   if (e != cudaSuccess) return fail_staged(c, sg, e);
   c->launches += 1;
+  if (c->view.pk32) {
+    e = L_(make_tab32)(c->view, c->stream, c->view.pk_mont, c->view.pk32, 2 * (size_t)c->view.L);
+    if (e != cudaSuccess) return fail_staged(c, sg, e);
+    c->launches += 1;
+  }
   if (pk_dev) {
     e = cudaMemcpyAsync(pk_dev, c->view.pk_coef, 2 * (size_t)c->view.L * c->view.n * sizeof(u64),
                         cudaMemcpyDeviceToDevice, c->stream);
@@ -791,6 +811,104 @@ d2mhe_status d2mhe_poly_muladd32(d2mhe_ctx* c, const uint32_t* a, const uint32_t
   if (!c->narrow) return D2MHE_ERR_UNSUPPORTED;
   DeviceGuard guard(c->device);
   cudaError_t e = L_(muladd32)(c->view, c->stream, a, b, cc, d, batch);
+  if (e != cudaSuccess) return fail_cuda(c, e);
+  c->launches += 1;
+  return D2MHE_OK;
+}
+
+// ---- the protocol calls on 32-bit words (every prime below 2^30) ------------------------
+
+static bool proto32_ok(const d2mhe_ctx* c) { return c->narrow && protocol_ok(c) && c->view.s32 && c->view.pk32; }
+
+d2mhe_status d2mhe_encrypt32(d2mhe_ctx* c, const u32* parties, u32 n_parties, u32 ct_first, u32 n_cts,
+                             const u32* plain_dev, uint32_t* ct_dev) {
+  if (!c || !plain_dev || !ct_dev || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(plain_dev) || !aligned16(ct_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!proto32_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  if (!c->has_pk) return D2MHE_ERR_STATE;
+  d2mhe_status st = check_party_list(c, parties, n_parties, false, false);
+  if (st != D2MHE_OK) return st;
+  if ((u64)ct_first + n_cts > 0x100000000ull) return D2MHE_ERR_RANGE;
+  if ((u64)n_parties * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[1] = {parties};
+  const size_t counts[1] = {n_parties};
+  if ((st = stage_indices(c, arrays, counts, 1, &sg)) != D2MHE_OK) return st;
+  u32 launched = 0;
+  cudaError_t e = L_(encrypt32)(c->view, c->limb_params, c->stream, sg.dev[0], n_parties, ct_first, n_cts, plain_dev,
+                                ct_dev, c->noise_scratch, c->noise_scratch_bytes, &launched);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
+  c->launches += launched;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_aggregate32(d2mhe_ctx* c, const uint32_t* ct_dev, u32 n_rows, u32 n_cts, const u32* nbr_offsets,
+                               const u32* nbr_rows, u32 n_out, uint32_t* agg_dev) {
+  if (!c || !ct_dev || !agg_dev || !nbr_offsets || n_rows == 0 || n_cts == 0 || n_out == 0)
+    return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(ct_dev) || !aligned16(agg_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!c->narrow || c->params.log2_n < 1) return D2MHE_ERR_UNSUPPORTED;
+  if (n_out > 65536) return D2MHE_ERR_RANGE;
+  if (nbr_offsets[0] != 0) return D2MHE_ERR_INVALID_ARG;
+  for (u32 i = 0; i < n_out; ++i)
+    if (nbr_offsets[i + 1] < nbr_offsets[i]) return D2MHE_ERR_INVALID_ARG;
+  const u32 nnz = nbr_offsets[n_out];
+  if (nnz > 1048576) return D2MHE_ERR_RANGE;
+  if (nnz && !nbr_rows) return D2MHE_ERR_INVALID_ARG;
+  for (u32 a = 0; a < nnz; ++a)
+    if (nbr_rows[a] >= n_rows) return D2MHE_ERR_RANGE;
+  if ((u64)n_out * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32 dummy = 0;
+  const u32* arrays[2] = {nbr_offsets, nnz ? nbr_rows : &dummy};
+  const size_t counts[2] = {(size_t)n_out + 1, nnz ? (size_t)nnz : 1};
+  d2mhe_status st = stage_indices(c, arrays, counts, 2, &sg);
+  if (st != D2MHE_OK) return st;
+  cudaError_t e = L_(aggregate32)(c->view, c->stream, ct_dev, n_cts, sg.dev[0], sg.dev[1], n_out, agg_dev);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
+  c->launches += 1;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_partial_decrypt32(d2mhe_ctx* c, const uint32_t* agg_dev, const u32* recipients, u32 n_rec,
+                                     const u32* parties, u32 n_parties, u32 ct_first, u32 n_cts,
+                                     uint32_t* shares_dev) {
+  if (!c || !agg_dev || !shares_dev || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(agg_dev) || !aligned16(shares_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!proto32_ok(c)) return D2MHE_ERR_UNSUPPORTED;
+  d2mhe_status st = check_party_list(c, recipients, n_rec, false, false);
+  if (st != D2MHE_OK) return st;
+  st = check_party_list(c, parties, n_parties, true, true);
+  if (st != D2MHE_OK) return st;
+  if ((u64)ct_first + n_cts > 0x100000000ull) return D2MHE_ERR_RANGE;
+  if ((u64)n_rec * n_cts * c->view.L > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  if ((size_t)n_parties * c->view.n > c->noise_scratch_bytes) return D2MHE_ERR_UNSUPPORTED;
+  DeviceGuard guard(c->device);
+  Staged sg;
+  const u32* arrays[2] = {recipients, parties};
+  const size_t counts[2] = {n_rec, n_parties};
+  if ((st = stage_indices(c, arrays, counts, 2, &sg)) != D2MHE_OK) return st;
+  u32 launched = 0;
+  cudaError_t e = L_(partial_decrypt32)(c->view, c->limb_params, c->stream, agg_dev, sg.dev[0], n_rec, sg.dev[1],
+                                        n_parties, ct_first, n_cts, shares_dev, c->noise_scratch,
+                                        c->noise_scratch_bytes, &launched);
+  if (e != cudaSuccess) return fail_staged(c, sg, e);
+  c->launches += launched;
+  return release_slot(c, sg);
+}
+
+d2mhe_status d2mhe_combine_decrypt32(d2mhe_ctx* c, const uint32_t* agg_dev, const uint32_t* shares_dev, u32 n_rec,
+                                     u32 n_shares, u32 n_cts, u32* plain_dev) {
+  if (!c || !agg_dev || !shares_dev || !plain_dev || n_rec == 0 || n_cts == 0) return D2MHE_ERR_INVALID_ARG;
+  if (!aligned16(agg_dev) || !aligned16(shares_dev) || !aligned16(plain_dev)) return D2MHE_ERR_INVALID_ARG;
+  if (!c->narrow) return D2MHE_ERR_UNSUPPORTED;
+  if (!c->has_pk) return D2MHE_ERR_STATE;
+  if (n_shares != c->pk_parties.size()) return D2MHE_ERR_INVALID_ARG;
+  if ((u64)n_rec * n_cts > 0x7fffffffull) return D2MHE_ERR_RANGE;
+  DeviceGuard guard(c->device);
+  cudaError_t e = L_(combine32)(c->view, c->stream, agg_dev, shares_dev, n_rec, n_shares, n_cts, plain_dev);
   if (e != cudaSuccess) return fail_cuda(c, e);
   c->launches += 1;
   return D2MHE_OK;

@@ -49,6 +49,10 @@ struct DevView {
   u64* usk_mont;  // [K][L][N]     NTT(sk_i) * N^-1 (Montgomery form) of the users' own keys
   u64* upk_mont;  // [K][2][L][N]  NTT(p_{0,i}), NTT(p_{1,i}) * N^-1 (Montgomery form)
   u64* upk_coef;  // [K][2][L][N]  pk_i, coefficient domain
+  // only when every prime is below 2^30 (the 32-bit-word protocol calls): the same keys as words
+  // {residue out of Montgomery form, its 32-bit Shoup companion}
+  u64* s32;       // [K][L][N]
+  u64* pk32;      // [2][L][N]
   u32* range_flag;
   u32* chk;       // four check words {site, index, limit, block} of the checked build
 };
@@ -164,7 +168,23 @@ cudaError_t secret_product(const DevView& v, const LimbParams& lp, cudaStream_t 
                            const u32* users_dev, u32 n_users, u32 n_cts, u64* prod); \
 cudaError_t muladd(const DevView& v, cudaStream_t s, const u64* a, const u64* b, const u64* c, \
                    u64* d, u32 batch); \
-cudaError_t check_selftest(const DevView& v, cudaStream_t s);
+cudaError_t check_selftest(const DevView& v, cudaStream_t s); \
+cudaError_t sample_encrypt_noise(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 ct_first, u32 n_cts, \
+                                 u32 unit_first, u32 n_units, u32* out); \
+cudaError_t sample_share_noise(const DevView& v, cudaStream_t s, const u32* recipients_dev, const u32* parties_dev, \
+                               u32 n_parties, u32 ct_first, u32 n_cts, u32 unit_first, u32 n_units, u32* out); \
+cudaError_t make_tab32(const DevView& v, cudaStream_t s, const u64* src, u64* dst, size_t rows); \
+cudaError_t encrypt32(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties, \
+                      u32 ct_first, u32 n_cts, const u32* plain, u32* ct, void* scratch, size_t scratch_bytes, \
+                      u32* launches); \
+cudaError_t aggregate32(const DevView& v, cudaStream_t s, const u32* ct, u32 n_cts, const u32* offsets_dev, \
+                        const u32* rows_dev, u32 n_out, u32* agg); \
+cudaError_t partial_decrypt32(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* agg, \
+                              const u32* recipients_dev, u32 n_rec, const u32* parties_dev, u32 n_parties, \
+                              u32 ct_first, u32 n_cts, u32* shares, void* scratch, size_t scratch_bytes, \
+                              u32* launches); \
+cudaError_t combine32(const DevView& v, cudaStream_t s, const u32* agg, const u32* shares, u32 n_rec, u32 n_shares, \
+                      u32 n_cts, u32* plain);
 
 namespace d2mhe_launch {
 D2MHE_LAUNCHER_DECLS

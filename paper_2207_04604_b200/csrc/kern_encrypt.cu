@@ -86,6 +86,15 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 
 namespace D2MHE_LAUNCH_NS {
 
+// u, e_0, e_1 of units unit_first .. unit_first + n_units - 1 into out ([u | e_0 | e_1], N bytes each, per unit)
+cudaError_t sample_encrypt_noise(const DevView& v, cudaStream_t s, const u32* parties_dev, u32 ct_first, u32 n_cts,
+                                 u32 unit_first, u32 n_units, u32* out) {
+  const size_t words = (size_t)n_units * 3 * v.n / 4;
+  k_sample_encrypt_noise<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(v, parties_dev, ct_first, n_cts, unit_first,
+                                                                        n_units, out);
+  return cudaGetLastError();
+}
+
 static cudaError_t encrypt_units(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 unit_first, u32 n_units,
                                  const u32* sampled, const u32* plain, u64* ct) {
   D2MHE_DISPATCH_EX(k_encrypt, v, n_units * v.L, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain, ct);
@@ -102,10 +111,7 @@ cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, cons
   if (per_batch == 0) return cudaErrorInvalidValue;
   for (u32 first = 0; first < n_units; first += per_batch) {
     const u32 nu = std::min(per_batch, n_units - first);
-    const size_t words = (size_t)nu * per_unit / 4;
-    k_sample_encrypt_noise<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(v, parties_dev, ct_first, n_cts, first, nu,
-                                                                          reinterpret_cast<u32*>(scratch));
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = sample_encrypt_noise(v, s, parties_dev, ct_first, n_cts, first, nu, reinterpret_cast<u32*>(scratch));
     if (e != cudaSuccess) return e;
     e = encrypt_units(v, lp, s, first, nu, reinterpret_cast<const u32*>(scratch), plain, ct);
     if (e != cudaSuccess) return e;

@@ -84,6 +84,15 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 
 namespace D2MHE_LAUNCH_NS {
 
+// the noise of the shares of units unit_first .. unit_first + n_units - 1: N bytes per (unit, party)
+cudaError_t sample_share_noise(const DevView& v, cudaStream_t s, const u32* recipients_dev, const u32* parties_dev,
+                               u32 n_parties, u32 ct_first, u32 n_cts, u32 unit_first, u32 n_units, u32* out) {
+  const size_t words = (size_t)n_units * n_parties * v.n / 4;
+  k_sample_share_noise<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(v, recipients_dev, parties_dev, n_parties,
+                                                                      ct_first, n_cts, unit_first, n_units, out);
+  return cudaGetLastError();
+}
+
 static cudaError_t pdec_pre_units(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
                                   const u32* parties_dev, u32 n_parties, u32 n_cts, u32 unit_first,
                                   u32 n_units, const signed char* noise, u64* shares) {
@@ -105,10 +114,8 @@ cudaError_t partial_decrypt_scratch(const DevView& v, const LimbParams& lp, cuda
   if (per_batch == 0) return cudaErrorInvalidValue;
   for (u32 first = 0; first < n_units; first += per_batch) {
     const u32 nu = std::min(per_batch, n_units - first);
-    const size_t words = (size_t)nu * per_unit / 4;
-    k_sample_share_noise<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(
-        v, recipients_dev, parties_dev, n_parties, ct_first, n_cts, first, nu, reinterpret_cast<u32*>(scratch));
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = sample_share_noise(v, s, recipients_dev, parties_dev, n_parties, ct_first, n_cts, first, nu,
+                                       reinterpret_cast<u32*>(scratch));
     if (e != cudaSuccess) return e;
     e = pdec_pre_units(v, lp, s, agg, parties_dev, n_parties, n_cts, first, nu,
                        reinterpret_cast<const signed char*>(scratch), shares);

@@ -63,9 +63,10 @@ __global__ void __launch_bounds__(256)
 // Up to 8 limbs the kernel is held to 32 registers (a few spilled words) so that 8 CTAs = 2048 threads
 // are resident per SM: the share streams need the loads in flight more than the registers
 // (measured: -13 % at N = 16384, L = 8, 20 shares; -2 % at N = 8192, L = 4, 10 shares).
-template <int LMAX>
+// W = u64, or u32 for the 32-bit-word messages (same arithmetic on the loaded residues).
+template <int LMAX, class W>
 __global__ void __launch_bounds__(256, LMAX <= 8 ? 8 : 3)
-    k_combine(DevView v, const u64* __restrict__ agg, const u64* __restrict__ shares, u32 n_shares,
+    k_combine(DevView v, const W* __restrict__ agg, const W* __restrict__ shares, u32 n_shares,
               u32 share_comps, u32 n_cts, u32* __restrict__ plain) {
   const u32 unit = blockIdx.x, irec = unit / n_cts, cl = unit % n_cts;
   const u32 j = blockIdx.y * blockDim.x + threadIdx.x;
@@ -73,8 +74,8 @@ __global__ void __launch_bounds__(256, LMAX <= 8 ? 8 : 3)
   const u32 L = v.L;
   if (!D2MHE_CHK(v.chk, L, (u32)LMAX + 1u, SITE_LIMB)) return;
   const size_t poly = (size_t)L * v.n;
-  const u64* c0 = agg + (size_t)unit * 2 * poly;
-  const bool lazy = v.wide != 0 && n_shares < 120;
+  const W* c0 = agg + (size_t)unit * 2 * poly;
+  const bool lazy = (v.wide != 0 || sizeof(W) == 4) && n_shares < 120;
   u64 d[LMAX];
 #pragma unroll
   for (int l = 0; l < LMAX; ++l) {
@@ -82,7 +83,7 @@ __global__ void __launch_bounds__(256, LMAX <= 8 ? 8 : 3)
       const LimbTab* lt = v.limbs + l;
       const u64 p = lt->p;
       u64 acc = __ldg(c0 + (size_t)l * v.n + j);
-      const u64* sh = shares + ((size_t)irec * n_shares * n_cts + cl) * share_comps * poly + (size_t)l * v.n + j;
+      const W* sh = shares + ((size_t)irec * n_shares * n_cts + cl) * share_comps * poly + (size_t)l * v.n + j;
       const size_t kstride = (size_t)n_cts * share_comps * poly;
       if (lazy) {
         // primes below 2^57 and fewer than 120 shares: the plain 64-bit sum cannot overflow and the
@@ -275,16 +276,25 @@ cudaError_t aggregate(const DevView& v, cudaStream_t s, const u64* ct, u32 n_cts
   return cudaGetLastError();
 }
 
-cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
-                    u32 n_shares, u32 share_comps, u32 n_cts, u32* plain) {
+template <class W>
+static cudaError_t combine_words(const DevView& v, cudaStream_t s, const W* agg, const W* shares, u32 n_rec,
+                                 u32 n_shares, u32 share_comps, u32 n_cts, u32* plain) {
   dim3 grid(n_rec * n_cts, (v.n + 255) / 256);
   if (v.L <= 4)
-    k_combine<4><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, share_comps, n_cts, plain);
+    k_combine<4, W><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, share_comps, n_cts, plain);
   else if (v.L <= 8)
-    k_combine<8><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, share_comps, n_cts, plain);
+    k_combine<8, W><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, share_comps, n_cts, plain);
   else
-    k_combine<D2MHE_MAX_LIMBS><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, share_comps, n_cts, plain);
+    k_combine<D2MHE_MAX_LIMBS, W><<<grid, 256, 0, s>>>(v, agg, shares, n_shares, share_comps, n_cts, plain);
   return cudaGetLastError();
+}
+cudaError_t combine(const DevView& v, cudaStream_t s, const u64* agg, const u64* shares, u32 n_rec,
+                    u32 n_shares, u32 share_comps, u32 n_cts, u32* plain) {
+  return combine_words<u64>(v, s, agg, shares, n_rec, n_shares, share_comps, n_cts, plain);
+}
+cudaError_t combine32(const DevView& v, cudaStream_t s, const u32* agg, const u32* shares, u32 n_rec, u32 n_shares,
+                      u32 n_cts, u32* plain) {
+  return combine_words<u32>(v, s, agg, shares, n_rec, n_shares, 1, n_cts, plain);
 }
 
 cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain) {

@@ -30,7 +30,8 @@ EXPORTS = [
     "d2mhe_keygen_share", "d2mhe_collective_pk", "d2mhe_encode", "d2mhe_decode", "d2mhe_encrypt",
     "d2mhe_aggregate", "d2mhe_partial_decrypt", "d2mhe_combine_decrypt", "d2mhe_ntt_forward",
     "d2mhe_ntt_inverse", "d2mhe_poly_muladd", "d2mhe_ntt32_forward", "d2mhe_ntt32_inverse",
-    "d2mhe_poly_muladd32", "d2mhe_round_workspace_bytes", "d2mhe_round_plan", "d2mhe_round_device",
+    "d2mhe_poly_muladd32", "d2mhe_encrypt32", "d2mhe_aggregate32", "d2mhe_partial_decrypt32",
+    "d2mhe_combine_decrypt32", "d2mhe_round_workspace_bytes", "d2mhe_round_plan", "d2mhe_round_device",
     "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_user_keygen", "d2mhe_convert_share",
     "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_bootstrap_share", "d2mhe_bootstrap_combine", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_debug_int_throughput", "d2mhe_debug_last_device_check",
     "d2mhe_debug_check_selftest", "d2mhe_get_root", "d2mhe_get_plain_root",
@@ -93,6 +94,10 @@ def load():
         lib.d2mhe_ntt32_forward.argtypes = [vp, vp, u32]
         lib.d2mhe_ntt32_inverse.argtypes = [vp, vp, u32]
         lib.d2mhe_poly_muladd32.argtypes = [vp, vp, vp, vp, vp, u32]
+        lib.d2mhe_encrypt32.argtypes = [vp, vp, u32, u32, u32, vp, vp]
+        lib.d2mhe_aggregate32.argtypes = [vp, vp, u32, u32, vp, vp, u32, vp]
+        lib.d2mhe_partial_decrypt32.argtypes = [vp, vp, vp, u32, vp, u32, u32, u32, vp]
+        lib.d2mhe_combine_decrypt32.argtypes = [vp, vp, vp, u32, u32, u32, vp]
         lib.d2mhe_round_plan.argtypes = [u32, ctypes.c_uint64, vp, u32, vp]
         lib.d2mhe_round_plan.restype = ctypes.c_uint32
         lib.d2mhe_round_workspace_bytes.argtypes = [vp, u32]
@@ -270,6 +275,28 @@ class Context:
     def poly_muladd32(self, a, b, c, d, batch):
         self._check(load().d2mhe_poly_muladd32(self._h, _dev(a, U32), _dev(b, U32), _dev(c, U32), _dev(d, U32), batch),
                     "d2mhe_poly_muladd32")
+
+    # ---- the protocol calls on 32-bit words ----
+    def encrypt32(self, parties, ct_first, n_cts, plain, ct):
+        arr, ptr = _host_u32(parties)
+        self._check(load().d2mhe_encrypt32(self._h, ptr, arr.size, ct_first, n_cts, _dev(plain, U32), _dev(ct, U32)),
+                    "d2mhe_encrypt32")
+
+    def aggregate32(self, ct, n_rows, n_cts, nbr_offsets, nbr_rows, agg):
+        off, offp = _host_u32(nbr_offsets)
+        rows, rowsp = _host_u32(nbr_rows)
+        self._check(load().d2mhe_aggregate32(self._h, _dev(ct, U32), n_rows, n_cts, offp, rowsp, off.size - 1,
+                                             _dev(agg, U32)), "d2mhe_aggregate32")
+
+    def partial_decrypt32(self, agg, recipients, parties, ct_first, n_cts, shares):
+        rec, recp = _host_u32(recipients)
+        par, parp = _host_u32(parties)
+        self._check(load().d2mhe_partial_decrypt32(self._h, _dev(agg, U32), recp, rec.size, parp, par.size, ct_first,
+                                                   n_cts, _dev(shares, U32)), "d2mhe_partial_decrypt32")
+
+    def combine_decrypt32(self, agg, shares, n_rec, n_shares, n_cts, plain):
+        self._check(load().d2mhe_combine_decrypt32(self._h, _dev(agg, U32), _dev(shares, U32), n_rec, n_shares, n_cts,
+                                                   _dev(plain, U32)), "d2mhe_combine_decrypt32")
 
     def round_workspace_bytes(self, chunk_cts):
         return int(load().d2mhe_round_workspace_bytes(self._h, chunk_cts))

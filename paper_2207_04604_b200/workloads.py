@@ -113,6 +113,13 @@ def round_config(index: int) -> RoundConfig:
     raise ValueError("round configs are 1..4")
 
 
+def narrow_round_config() -> RoundConfig:
+    """The MNIST-shaped configuration on 30-bit limbs (for the 32-bit-word protocol calls): same K,
+    graph, N, gradient and plaintext modulus; seven primes below 2^30 give log q = 210 against the 216
+    of four 54-bit primes."""
+    return RoundConfig("mnist-mlp-784-128-10-K10-30bit-limbs", 10, 4, 13, 30, 7, 101770, 1e-2)
+
+
 SWEEP_LOG2_N = (12, 13, 14, 15, 16)
 SWEEP_LIMBS = (1, 4, 8, 16, 24)
 SWEEP_BATCH = (1, 64, 1024, 4096)

@@ -944,6 +944,111 @@ def test_error_statuses(d2):
 
 
 # ----------------------------------------------------------------------------------
+# the protocol calls on 32-bit words (every prime below 2^30)
+# ----------------------------------------------------------------------------------
+
+
+def _run_round32(d2, ctx, o, parties, offsets, rows, values, ct_first, also_64=True):
+    """encrypt32 -> aggregate32 -> partial_decrypt32 -> combine_decrypt32 against the oracle, message
+    by message, and against the 64-bit calls of the same context."""
+    K, n_cts = len(parties), values.shape[1]
+    L, n = o.num_limbs, o.n
+    dev = ctx.device
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    want_pk = o.collective_pk(parties)
+    dv = torch.from_numpy(values).to(dev)
+    plain = ctx.empty_u32(K, n_cts, n)
+    ctx.encode(dv, K * n_cts, plain)
+    want_plain = o.encode(values)
+    ct = ctx.empty_u32(K, n_cts, 2, L, n)
+    ctx.encrypt32(parties, ct_first, n_cts, plain, ct)
+    want_ct = o.encrypt(want_pk, parties, ct_first, want_plain)
+    assert np.array_equal(d2.to_u32_numpy(ct).astype(np.uint64), want_ct)
+    n_out = len(offsets) - 1
+    agg = ctx.empty_u32(n_out, n_cts, 2, L, n)
+    ctx.aggregate32(ct, K, n_cts, offsets, rows, agg)
+    want_agg = o.aggregate(want_ct, offsets, rows)
+    assert np.array_equal(d2.to_u32_numpy(agg).astype(np.uint64), want_agg)
+    recipients = [i % K for i in range(n_out)]
+    shares = ctx.empty_u32(n_out, K, n_cts, L, n)
+    ctx.partial_decrypt32(agg, recipients, parties, ct_first, n_cts, shares)
+    want_shares = o.partial_decrypt(want_agg, recipients, parties, ct_first)
+    assert np.array_equal(d2.to_u32_numpy(shares).astype(np.uint64), want_shares)
+    out_plain = ctx.empty_u32(n_out, n_cts, n)
+    ctx.combine_decrypt32(agg, shares, n_out, K, n_cts, out_plain)
+    want_out = o.combine(want_agg, want_shares)
+    assert np.array_equal(d2.to_u32_numpy(out_plain), want_out)
+    sums = torch.empty((n_out, n_cts, n), dtype=torch.int32, device=dev)
+    ctx.decode(out_plain, n_out * n_cts, sums)
+    ctx.sync()
+    got = sums.cpu().numpy()
+    for i in range(n_out):
+        lst = rows[offsets[i]:offsets[i + 1]]
+        assert np.array_equal(got[i], values[lst].astype(np.int64).sum(axis=0))
+    if also_64:
+        ct64 = ctx.empty_u64(K, n_cts, 2, L, n)
+        ctx.encrypt(parties, ct_first, n_cts, plain, ct64)
+        assert np.array_equal(d2.to_u64_numpy(ct64), want_ct)
+        sh64 = ctx.empty_u64(n_out, K, n_cts, L, n)
+        ctx.partial_decrypt(d2.from_u64_numpy(want_agg, dev), recipients, parties, ct_first, n_cts, sh64)
+        assert np.array_equal(d2.to_u64_numpy(sh64), want_shares)
+
+
+@pytest.mark.parametrize("log2_n,bits,L,K,n_cts", [
+    (4, 24, 2, 3, 1),    # odd numbers of units: the last thread block holds one
+    (6, 30, 3, 2, 3),
+    (10, 30, 5, 3, 2),
+    (12, 29, 3, 4, 2),
+    (13, 30, 2, 3, 1),
+    (14, 30, 2, 2, 2),
+])
+def test_protocol_on_32_bit_words_every_message(d2, log2_n, bits, L, K, n_cts):
+    moduli = wl.ntt_primes(bits, 2 << log2_n, L)
+    seed = 200 + log2_n
+    ctx = d2.Context(log2_n, moduli, K, seed=seed)
+    o = make_oracle(log2_n, moduli, seed=seed)
+    n = 1 << log2_n
+    half = (T - 1) // 2 // K
+    values = np.random.default_rng(log2_n).integers(-half, half + 1, size=(K, n_cts, n)).astype(np.int32)
+    values[0, 0, :2] = [half, -half]
+    offsets = np.array([0, K, K, K + 1], dtype=np.uint32)  # an empty list in the middle, three recipients
+    rows = np.array(list(range(K)) + [K - 1], dtype=np.uint32)
+    _run_round32(d2, ctx, o, list(range(K)), offsets, rows, values, ct_first=9)
+    ctx.close()
+
+
+def test_mnist_shaped_round_on_30_bit_limbs_every_message(d2):
+    """The MNIST-shaped configuration with seven 30-bit limbs (log q = 210) through the 32-bit-word
+    calls: every ciphertext, sum, share and plaintext of all 13 indices against the oracle."""
+    cfg = wl.narrow_round_config()
+    assert max(cfg.moduli) < 1 << 30 and len(cfg.moduli) == 7
+    seed = 1
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, cfg.num_parties, seed=seed)
+    o = make_oracle(cfg.log2_n, cfg.moduli, seed=seed)
+    offsets, rows = wl.regular_graph(cfg.num_parties, cfg.degree, seed)
+    values = wl.gradients(cfg, seed)
+    _run_round32(d2, ctx, o, list(range(cfg.num_parties)), offsets, rows, values, 0, also_64=False)
+    ctx.close()
+
+
+def test_32_bit_protocol_calls_refuse_wide_primes(d2):
+    cfg = wl.round_config(1)
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, 2, seed=1)
+    ctx.keygen_share([0, 1])
+    ctx.collective_pk([0, 1])
+    plain = ctx.empty_u32(2, 1, cfg.n)
+    ct = ctx.empty_u32(2, 1, 2, cfg.num_limbs, cfg.n)
+    with pytest.raises(d2.D2mheError) as e:
+        ctx.encrypt32([0, 1], 0, 1, plain, ct)
+    assert e.value.status == d2.ERR_UNSUPPORTED
+    with pytest.raises(d2.D2mheError) as e:
+        ctx.partial_decrypt32(ct, [0], [0, 1], 0, 1, ct)
+    assert e.value.status == d2.ERR_UNSUPPORTED
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------------
 # the checked kernel build (D2MHE_FLAG_DEVICE_CHECKS)
 # ----------------------------------------------------------------------------------
 
