@@ -440,7 +440,8 @@ def measure_round(cfg, args, steps, warmup, rank, local_rank, world, detailed, s
 
     # transform / multiply-add micro-benchmark on this configuration's ring (batch > L2), and the
     # conversion / refresh calls (the paper's own decryption path and its bootstrap) on a few indices
-    if rank == 0:
+    res["ntt"] = res["convert_bootstrap"] = None
+    if rank == 0 and not args.no_extras:
         del ws
         torch.cuda.empty_cache()
         res["ntt"] = ntt_microbench(ctx, cfg, dev, stream, flush)
@@ -670,12 +671,12 @@ def run_cuda(args, cfg):
         total_ms = sum(per_call.values())
         slots = algorithmic_mad_slots(cfg, C)
         ntt = res["ntt"]
-        for k_ in ("forward", "inverse", "muladd"):
+        for k_ in ("forward", "inverse", "muladd") if ntt else ():
             ntt[k_ + "_frac_of_hbm"] = ntt[k_ + "_GBps"] / peak
-        for k_ in ("forward", "inverse"):
+        for k_ in ("forward", "inverse") if ntt else ():
             ntt[k_ + "_alu_frac"] = ntt[k_ + "_butterflies_per_s"] * SLOTS_PER_BUTTERFLY / imad_peak
         cb = res["convert_bootstrap"]
-        for k_ in ("convert", "bootstrap"):
+        for k_ in ("convert", "bootstrap") if cb else ():
             cb[k_ + "_share_alu_frac"] = cb[k_ + "_share_slots"] / (cb[k_ + "_share_ms"] * 1e-3) / imad_peak
             cb[k_ + "_share_GBps"] = cb["share_bytes"] / 1e9 / (cb[k_ + "_share_ms"] * 1e-3)
         kernels = {}
@@ -846,6 +847,10 @@ def main():
     ap.add_argument("--cts", type=int, default=0,
                     help="run only the first CTS ciphertext indices of the workload (a labelled slice, for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the transform micro-benchmark and the conversion / refresh calls")
+    ap.add_argument("--narrow", action="store_true",
+                    help="run only the MNIST-shaped round on 30-bit limbs (32-bit-word calls) and print its line")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the short passes over the other round configurations")
     ap.add_argument("--sweep-bits", type=int, default=60, choices=[30, 50, 60])
@@ -853,6 +858,13 @@ def main():
     args = ap.parse_args()
     if args.config == 5:
         return run_sweep(args)
+    if args.narrow:
+        from paper_2207_04604_b200 import build
+
+        build.build()
+        line = narrow_round_bench(args, 0)
+        line.update(metric=METRIC, unit=UNIT, dtype="u32", data="synthetic")
+        return print(json.dumps(line))
     cfg = wl.round_config(args.config)
     if args.impl == "reference":
         run_reference(args, cfg)

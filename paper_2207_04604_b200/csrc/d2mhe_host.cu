@@ -410,6 +410,12 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   err = cudaMemset(c->view.range_flag, 0, 16);
   if (err != cudaSuccess) return fail_cuda(c, err);
 
+  {
+    int sms = 0;
+    err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    c->view.sms = sms > 0 ? (u32)sms : 1u;
+  }
   c->view.seed = P.seed;
   c->view.logn = logn;
   c->view.n = n;

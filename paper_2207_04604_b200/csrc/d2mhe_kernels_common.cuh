@@ -116,6 +116,19 @@ constexpr u32 ntt_threads_ct(int logn, int g) {
   return logn == 0 ? 1024u : (((1u << logn) / 8u / (u32)g) < 32u ? 32u : ((1u << logn) / 8u / (u32)g));
 }
 
+// Thread blocks of a transform kernel that the device holds at once.
+inline u32 resident_ctas(const DevView& v) { return v.sms * (u32)ntt_minb_ct((int)v.logn); }
+// A call that must be cut into batches (its scratch holds `cap` of its `n_units` units, each unit
+// ctas_per_unit thread blocks) takes batches of whole waves of thread blocks when a batch is at least
+// one wave: a batch that ends part-way through a wave leaves SMs idle until its last blocks finish.
+inline u32 whole_wave_batch(const DevView& v, u32 cap, u32 n_units, u32 ctas_per_unit) {
+  if (cap >= n_units) return n_units;
+  const u32 res = resident_ctas(v), ctas = cap * ctas_per_unit;
+  if (ctas < res) return cap;
+  const u32 whole = (ctas / res) * res / ctas_per_unit;
+  return whole ? whole : cap;
+}
+
 inline size_t poly_bytes(u32 n, size_t extra_bytes = 0) {
   return D2MHE_GAUSS_BYTES + extra_bytes + (size_t)n * sizeof(u64);
 }

@@ -244,9 +244,10 @@ cudaError_t convert_share(const DevView& v, const LimbParams& lp, cudaStream_t s
                           u32 ct_first, u32 n_cts, u64* shares, void* scratch, size_t scratch_bytes, u32* launches) {
   const size_t per_unit = (size_t)n_parties * 3 * v.n;
   const u32 n_units = n_rec * n_cts;
-  const u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
+  u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
   if (launches) *launches = 0;
   if (per_batch == 0) return cudaErrorInvalidValue;
+  per_batch = whole_wave_batch(v, per_batch, n_units, v.L);
   for (u32 first = 0; first < n_units; first += per_batch) {
     const u32 nu = std::min(per_batch, n_units - first);
     const size_t words = (size_t)nu * per_unit / 4;

@@ -34,14 +34,17 @@ __global__ void __launch_bounds__(256)
   small[e] = pack;
 }
 
-// grid = n_units * L; units unit_first .. unit_first + n_units - 1 of the (party, ciphertext) grid.
+// grid = n_units * L * split; units unit_first .. unit_first + n_units - 1 of the (party, ciphertext) grid.
 // NTT(u) is parked in the output row of c_1 (re-read for both components, overwritten by
 // c_1 at the very end), so no registers are held across the two inverse transforms.
+// split = 2 (chosen by the launcher when the grid would otherwise leave most SMs idle) gives the two
+// components to two thread blocks; each transforms u for itself and parks it in its own output row.
 template <int LOGN, int G, bool WIDE>
 __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
     k_encrypt(DevView v, const __grid_constant__ LimbParams lp, u32 unit_first, const u32* __restrict__ sampled,
-              const u32* __restrict__ plain, u64* ct) {
-  const u32 l = blockIdx.x % v.L, ulocal = blockIdx.x / v.L, unit = unit_first + ulocal;
+              const u32* __restrict__ plain, u64* ct, u32 split) {
+  const u32 part = blockIdx.x % split, rest = blockIdx.x / split;
+  const u32 l = rest % v.L, ulocal = rest / v.L, unit = unit_first + ulocal;
   const LimbTab& lt = lp.limbs[l];
   signed char* small = bytes_smem();  // u, e_0, e_1: N bytes each
   u64* sm = poly_smem(3 * v.n);
@@ -52,12 +55,12 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
     for (u32 w = threadIdx.x; w < 3 * (v.n >> 2); w += blockDim.x) reinterpret_cast<u32*>(small)[w] = __ldg(src + w);
   }
   // the barrier that opens the forward transform publishes the copy
-  u64* park = ct + ((size_t)unit * 2 + 1) * poly + row;
+  u64* park = ct + ((size_t)unit * 2 + (split > 1 ? part : 1u)) * poly + row;
   ntt_forward<LOGN, G, WIDE>(
       sm, lt, v.logn, [&](u32 j) { return lift_small((int)small[j], lt.p); },
       [&](int, u32 q, u64(&x)[8]) { store_octet(park + 8 * (size_t)q, x); });
 #pragma unroll 1
-  for (u32 comp = 0; comp < 2; ++comp) {
+  for (u32 comp = split > 1 ? part : 0u; comp < (split > 1 ? part + 1u : 2u); ++comp) {
     const u64* pkh = v.pk_mont + comp * poly + row;
     u64* out = ct + ((size_t)unit * 2 + comp) * poly + row;
     const signed char* e = small + (comp + 1) * v.n;
@@ -97,7 +100,11 @@ cudaError_t sample_encrypt_noise(const DevView& v, cudaStream_t s, const u32* pa
 
 static cudaError_t encrypt_units(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 unit_first, u32 n_units,
                                  const u32* sampled, const u32* plain, u64* ct) {
-  D2MHE_DISPATCH_EX(k_encrypt, v, n_units * v.L, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain, ct);
+  // a small call (at most half of the thread blocks that the GPU holds at once) uses one block per component
+  const u32 resident = resident_ctas(v);
+  const u32 split = n_units * v.L * 2 <= resident ? 2u : 1u;
+  D2MHE_DISPATCH_EX(k_encrypt, v, n_units * v.L * split, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain, ct,
+                    split);
 }
 
 // scratch: at least 3 N bytes; (party, ciphertext) units are processed in batches of as many as it holds.
@@ -106,9 +113,10 @@ cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, cons
                     u32* launches) {
   const size_t per_unit = 3 * (size_t)v.n;
   const u32 n_units = n_parties * n_cts;
-  const u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
+  u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
   if (launches) *launches = 0;
   if (per_batch == 0) return cudaErrorInvalidValue;
+  per_batch = whole_wave_batch(v, per_batch, n_units, v.L);
   for (u32 first = 0; first < n_units; first += per_batch) {
     const u32 nu = std::min(per_batch, n_units - first);
     cudaError_t e = sample_encrypt_noise(v, s, parties_dev, ct_first, n_cts, first, nu, reinterpret_cast<u32*>(scratch));

@@ -36,32 +36,38 @@ __global__ void __launch_bounds__(256)
   noise[e] = pack;
 }
 
-// grid = n_units * L; units unit_first .. unit_first + n_units - 1 of the (recipient, ciphertext) grid.
+// grid = n_units * L * split; units unit_first .. unit_first + n_units - 1 of the (recipient, ciphertext)
+// grid.  split > 1 (chosen by the launcher when the grid would otherwise leave most SMs idle) gives the
+// parties of a unit's list to `split` thread blocks, party a to block a mod split; each of them
+// transforms c_1 for itself and parks it in the row of the last share that it writes.
 template <int LOGN, int G, bool WIDE>
 __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
     k_partial_decrypt_pre(DevView v, const __grid_constant__ LimbParams lp, const u64* __restrict__ agg,
                           const u32* __restrict__ parties, u32 n_parties, u32 n_cts, u32 unit_first,
-                          const signed char* __restrict__ noise, u64* shares) {
-  const u32 l = blockIdx.x % v.L, ulocal = blockIdx.x / v.L, unit = unit_first + ulocal;
+                          const signed char* __restrict__ noise, u64* shares, u32 split) {
+  const u32 part = blockIdx.x % split, rest = blockIdx.x / split;
+  const u32 l = rest % v.L, ulocal = rest / v.L, unit = unit_first + ulocal;
+  if (part >= n_parties) return;
+  const u32 a_last = part + split * ((n_parties - 1 - part) / split);  // the last party of this block
   const u32 irec = unit / n_cts, cl = unit % n_cts;
   const LimbTab& lt = lp.limbs[l];
   signed char* staged = bytes_smem();  // two buffers of N bytes: the noise of this share and of the next
   u64* sm = poly_smem(2 * v.n);
   const size_t row = (size_t)l * v.n, poly = (size_t)v.L * v.n;
   const u64* c1 = agg + ((size_t)unit * 2 + 1) * poly + row;
-  u64* park = shares + (((size_t)irec * n_parties + (n_parties - 1)) * n_cts + cl) * poly + row;
+  u64* park = shares + (((size_t)irec * n_parties + a_last) * n_cts + cl) * poly + row;
   ntt_forward<LOGN, G, WIDE>(
       sm, lt, v.logn, [&](u32 j) { return __ldg(c1 + j); },
       [&](int, u32 q, u64(&x)[8]) { store_octet(park + 8 * (size_t)q, x); });
 #pragma unroll 1
-  for (u32 a = 0; a < n_parties; ++a) {
+  for (u32 a = part, it = 0; a < n_parties; a += split, ++it) {
     const u32 party = parties[a];
     if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY)) continue;
     const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
-    // Buffer a & 1 was last read in the final round of share a - 2, which every thread left before
-    // it passed the barrier that opens the transform of share a - 1; the barrier that opens this
-    // share's transform publishes the copy.
-    signed char* e = staged + (a & 1u) * v.n;
+    // The buffer of iteration it was last read in the final round of iteration it - 2, which every
+    // thread left before it passed the barrier that opens the transform of iteration it - 1; the
+    // barrier that opens this share's transform publishes the copy.
+    signed char* e = staged + (it & 1u) * v.n;
     {
       const u32* src = reinterpret_cast<const u32*>(noise + ((size_t)ulocal * n_parties + a) * v.n);
       for (u32 w = threadIdx.x; w < (v.n >> 2); w += blockDim.x) reinterpret_cast<u32*>(e)[w] = __ldg(src + w);
@@ -96,8 +102,13 @@ cudaError_t sample_share_noise(const DevView& v, cudaStream_t s, const u32* reci
 static cudaError_t pdec_pre_units(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
                                   const u32* parties_dev, u32 n_parties, u32 n_cts, u32 unit_first,
                                   u32 n_units, const signed char* noise, u64* shares) {
-  D2MHE_DISPATCH_EX(k_partial_decrypt_pre, v, n_units * v.L, s, 2 * (size_t)v.n, 1, v, lp, agg, parties_dev, n_parties,
-                    n_cts, unit_first, noise, shares);
+  // A small call (fewer thread blocks than the GPU holds at once) spreads each unit's parties over
+  // several blocks: the latency of the call is then that of a few transforms, not of the whole list.
+  const u32 resident = resident_ctas(v);
+  u32 split = 1;
+  if (n_units * v.L * 2 <= resident) split = std::min(n_parties, resident / (n_units * v.L));
+  D2MHE_DISPATCH_EX(k_partial_decrypt_pre, v, n_units * v.L * split, s, 2 * (size_t)v.n, 1, v, lp, agg, parties_dev,
+                    n_parties, n_cts, unit_first, noise, shares, split);
 }
 
 // Shares with the noise sampled ahead into `scratch` (scratch_bytes >= n_parties * N), in batches of
@@ -109,9 +120,10 @@ cudaError_t partial_decrypt_scratch(const DevView& v, const LimbParams& lp, cuda
                                     size_t scratch_bytes, u32* launches) {
   const size_t per_unit = (size_t)n_parties * v.n;
   const u32 n_units = n_rec * n_cts;
-  const u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
+  u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
   if (launches) *launches = 0;
   if (per_batch == 0) return cudaErrorInvalidValue;
+  per_batch = whole_wave_batch(v, per_batch, n_units, v.L);
   for (u32 first = 0; first < n_units; first += per_batch) {
     const u32 nu = std::min(per_batch, n_units - first);
     cudaError_t e = sample_share_noise(v, s, recipients_dev, parties_dev, n_parties, ct_first, n_cts, first, nu,

@@ -306,9 +306,11 @@ cudaError_t partial_decrypt32(const DevView& v, const LimbParams& lp, cudaStream
   const size_t per_unit = (size_t)n_parties * v.n;
   const u32 n_units = n_rec * n_cts;
   u32 per_batch = (u32)std::min<size_t>(scratch_bytes / per_unit, n_units);
-  if (per_batch > 1) per_batch &= ~1u;  // whole pairs per batch
   if (launches) *launches = 0;
   if (per_batch == 0) return cudaErrorInvalidValue;
+  if (per_batch < n_units && per_batch > 1) {
+    per_batch = 2 * whole_wave_batch(v, per_batch / 2, (n_units + 1) / 2, v.L);  // whole pairs, whole waves
+  }
   for (u32 first = 0; first < n_units; first += per_batch) {
     const u32 nu = std::min(per_batch, n_units - first);
     cudaError_t e = sample_share_noise(v, s, recipients_dev, parties_dev, n_parties, ct_first, n_cts, first, nu,
