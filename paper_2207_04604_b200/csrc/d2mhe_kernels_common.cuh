@@ -1,6 +1,5 @@
 // Shared pieces of the kernel translation units: shared-memory layout, octet I/O, dispatch.
 #pragma once
-#include <cooperative_groups.h>
 #include <cstdlib>
 
 #include "d2mhe_internal.h"
@@ -137,28 +136,10 @@ inline u32 ntt_threads(u32 n, int g) {
   return t < 32 ? 32 : t;
 }
 
-// Largest divisor of L that is a portable thread-block-cluster size, at most `cap` (the conversion
-// and bootstrap share kernels sample their noise inside the kernel, each CTA of a cluster a part of
-// it).  At N = 16384 a CTA fills an SM, a cluster must sit inside one GPC, and clusters of 8 leave the
-// SMs of every GPC beyond a multiple of 8 idle (120 of 148 SMs were busy when the decryption-share
-// kernel still ran that way).  Measured there (L = 8): clusters of 2 beat 4, 8 and 1 although each
-// CTA then samples half of the noise itself; at N = 8192 (two CTAs per SM, L = 4) clusters of 4 beat
-// 2 and 1.
-#ifndef D2MHE_CS_CAP14
-#define D2MHE_CS_CAP14 2
-#endif
-#ifndef D2MHE_CS_CAP
-#define D2MHE_CS_CAP 8
-#endif
-inline u32 cluster_size_for(u32 L, u32 logn) {
-  const u32 cap = logn >= 14 ? D2MHE_CS_CAP14 : D2MHE_CS_CAP;
-  for (u32 cs = cap; cs > 1; --cs)
-    if (L % cs == 0) return cs;
-  return 1;
-}
-
-// Launch with a thread-block cluster of `cs` CTAs along x (cs = 1: plain launch).  Falls back
-// to cs = 1 when the device cannot co-schedule such a cluster for this kernel.
+// Launch with a thread-block cluster of `cs` CTAs along x (cs = 1: plain launch, which is what every
+// kernel of the library uses: kernels that sampled inside clusters were measured slower than
+// sampling ahead of the kernel).  Falls back to cs = 1 when the device cannot co-schedule such a
+// cluster for this kernel.
 template <class... KArgs, class... Args>
 cudaError_t launch_clustered(void (*kernel)(KArgs...), u32 grid, u32 threads, size_t smem,
                              cudaStream_t stream, u32 cs, Args... args) {
