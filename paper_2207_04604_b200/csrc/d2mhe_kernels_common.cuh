@@ -170,9 +170,12 @@ cudaError_t launch_clustered(void (*kernel)(KArgs...), u32 grid, u32 threads, si
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// D2MHE_EXTRA_TARGS: further template arguments of the kernel (", true"), empty by default; a
+// translation unit redefines it around the launcher that needs them.
+#define D2MHE_EXTRA_TARGS
 #define D2MHE_LAUNCH_ONE(KERNEL, LOGN_, G_, WIDE_, grid, stream, cs, ...)                      \
   do {                                                                                         \
-    cudaError_t e_ = launch_clustered(KERNEL<LOGN_, G_, WIDE_>, grid, ntt_threads(n_, G_),     \
+    cudaError_t e_ = launch_clustered(KERNEL<LOGN_, G_, WIDE_ D2MHE_EXTRA_TARGS>, grid, ntt_threads(n_, G_), \
                                       smem_, stream, cs, __VA_ARGS__);                         \
     if (e_ != cudaSuccess) return e_;                                                          \
   } while (0)

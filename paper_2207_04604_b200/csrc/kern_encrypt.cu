@@ -39,11 +39,12 @@ __global__ void __launch_bounds__(256)
 // c_1 at the very end), so no registers are held across the two inverse transforms.
 // split = 2 (chosen by the launcher when the grid would otherwise leave most SMs idle) gives the two
 // components to two thread blocks; each transforms u for itself and parks it in its own output row.
-template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
-    k_encrypt(DevView v, const __grid_constant__ LimbParams lp, u32 unit_first, const u32* __restrict__ sampled,
-              const u32* __restrict__ plain, u64* ct, u32 split) {
-  const u32 part = blockIdx.x % split, rest = blockIdx.x / split;
+// (The split is a template switch: as a run-time argument it cost the common, unsplit case registers.)
+template <int LOGN, int G, bool WIDE, bool SPLIT>
+__device__ __forceinline__ void encrypt_body(const DevView& v, const LimbParams& lp, u32 unit_first,
+                                             const u32* __restrict__ sampled, const u32* __restrict__ plain, u64* ct) {
+  const u32 split = SPLIT ? 2u : 1u;
+  const u32 part = SPLIT ? blockIdx.x % 2u : 0u, rest = SPLIT ? blockIdx.x / 2u : blockIdx.x;
   const u32 l = rest % v.L, ulocal = rest / v.L, unit = unit_first + ulocal;
   const LimbTab& lt = lp.limbs[l];
   signed char* small = bytes_smem();  // u, e_0, e_1: N bytes each
@@ -85,6 +86,19 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
   }
 }
 
+template <int LOGN, int G, bool WIDE>
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+    k_encrypt(DevView v, const __grid_constant__ LimbParams lp, u32 unit_first, const u32* __restrict__ sampled,
+              const u32* __restrict__ plain, u64* ct) {
+  encrypt_body<LOGN, G, WIDE, false>(v, lp, unit_first, sampled, plain, ct);
+}
+template <int LOGN, int G, bool WIDE>
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+    k_encrypt_split(DevView v, const __grid_constant__ LimbParams lp, u32 unit_first, const u32* __restrict__ sampled,
+                    const u32* __restrict__ plain, u64* ct) {
+  encrypt_body<LOGN, G, WIDE, true>(v, lp, unit_first, sampled, plain, ct);
+}
+
 }  // namespace
 
 namespace D2MHE_LAUNCH_NS {
@@ -102,9 +116,11 @@ static cudaError_t encrypt_units(const DevView& v, const LimbParams& lp, cudaStr
                                  const u32* sampled, const u32* plain, u64* ct) {
   // a small call (at most half of the thread blocks that the GPU holds at once) uses one block per component
   const u32 resident = resident_ctas(v);
-  const u32 split = n_units * v.L * 2 <= resident ? 2u : 1u;
-  D2MHE_DISPATCH_EX(k_encrypt, v, n_units * v.L * split, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain, ct,
-                    split);
+  if (n_units * v.L * 2 <= resident) {
+    D2MHE_DISPATCH_EX(k_encrypt_split, v, n_units * v.L * 2, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain,
+                      ct);
+  }
+  D2MHE_DISPATCH_EX(k_encrypt, v, n_units * v.L, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain, ct);
 }
 
 // scratch: at least 3 N bytes; (party, ciphertext) units are processed in batches of as many as it holds.

@@ -40,15 +40,17 @@ __global__ void __launch_bounds__(256)
 // grid.  split > 1 (chosen by the launcher when the grid would otherwise leave most SMs idle) gives the
 // parties of a unit's list to `split` thread blocks, party a to block a mod split; each of them
 // transforms c_1 for itself and parks it in the row of the last share that it writes.
-template <int LOGN, int G, bool WIDE>
+// (The split is a template switch: as a run-time argument it cost the common, unsplit case registers.)
+template <int LOGN, int G, bool WIDE, bool SPLIT>
 __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
     k_partial_decrypt_pre(DevView v, const __grid_constant__ LimbParams lp, const u64* __restrict__ agg,
                           const u32* __restrict__ parties, u32 n_parties, u32 n_cts, u32 unit_first,
-                          const signed char* __restrict__ noise, u64* shares, u32 split) {
-  const u32 part = blockIdx.x % split, rest = blockIdx.x / split;
+                          const signed char* __restrict__ noise, u64* shares, u32 split_arg) {
+  const u32 split = SPLIT ? split_arg : 1u;
+  const u32 part = SPLIT ? blockIdx.x % split : 0u, rest = SPLIT ? blockIdx.x / split : blockIdx.x;
   const u32 l = rest % v.L, ulocal = rest / v.L, unit = unit_first + ulocal;
-  if (part >= n_parties) return;
-  const u32 a_last = part + split * ((n_parties - 1 - part) / split);  // the last party of this block
+  if (SPLIT && part >= n_parties) return;
+  const u32 a_last = SPLIT ? part + split * ((n_parties - 1 - part) / split) : n_parties - 1;  // the last party of this block
   const u32 irec = unit / n_cts, cl = unit % n_cts;
   const LimbTab& lt = lp.limbs[l];
   signed char* staged = bytes_smem();  // two buffers of N bytes: the noise of this share and of the next
@@ -60,7 +62,8 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
       sm, lt, v.logn, [&](u32 j) { return __ldg(c1 + j); },
       [&](int, u32 q, u64(&x)[8]) { store_octet(park + 8 * (size_t)q, x); });
 #pragma unroll 1
-  for (u32 a = part, it = 0; a < n_parties; a += split, ++it) {
+  for (u32 a = part; a < n_parties; a += split) {
+    const u32 it = SPLIT ? (a - part) / split : a;  // iteration number of this block
     const u32 party = parties[a];
     if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY)) continue;
     const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
@@ -99,6 +102,25 @@ cudaError_t sample_share_noise(const DevView& v, cudaStream_t s, const u32* reci
   return cudaGetLastError();
 }
 
+#undef D2MHE_EXTRA_TARGS
+#define D2MHE_EXTRA_TARGS , false
+static cudaError_t pdec_units_plain(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
+                                    const u32* parties_dev, u32 n_parties, u32 n_cts, u32 unit_first, u32 n_units,
+                                    const signed char* noise, u64* shares) {
+  D2MHE_DISPATCH_EX(k_partial_decrypt_pre, v, n_units * v.L, s, 2 * (size_t)v.n, 1, v, lp, agg, parties_dev, n_parties,
+                    n_cts, unit_first, noise, shares, 1u);
+}
+#undef D2MHE_EXTRA_TARGS
+#define D2MHE_EXTRA_TARGS , true
+static cudaError_t pdec_units_split(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
+                                    const u32* parties_dev, u32 n_parties, u32 n_cts, u32 unit_first, u32 n_units,
+                                    const signed char* noise, u64* shares, u32 split) {
+  D2MHE_DISPATCH_EX(k_partial_decrypt_pre, v, n_units * v.L * split, s, 2 * (size_t)v.n, 1, v, lp, agg, parties_dev,
+                    n_parties, n_cts, unit_first, noise, shares, split);
+}
+#undef D2MHE_EXTRA_TARGS
+#define D2MHE_EXTRA_TARGS
+
 static cudaError_t pdec_pre_units(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* agg,
                                   const u32* parties_dev, u32 n_parties, u32 n_cts, u32 unit_first,
                                   u32 n_units, const signed char* noise, u64* shares) {
@@ -107,8 +129,8 @@ static cudaError_t pdec_pre_units(const DevView& v, const LimbParams& lp, cudaSt
   const u32 resident = resident_ctas(v);
   u32 split = 1;
   if (n_units * v.L * 2 <= resident) split = std::min(n_parties, resident / (n_units * v.L));
-  D2MHE_DISPATCH_EX(k_partial_decrypt_pre, v, n_units * v.L * split, s, 2 * (size_t)v.n, 1, v, lp, agg, parties_dev,
-                    n_parties, n_cts, unit_first, noise, shares, split);
+  if (split > 1) return pdec_units_split(v, lp, s, agg, parties_dev, n_parties, n_cts, unit_first, n_units, noise, shares, split);
+  return pdec_units_plain(v, lp, s, agg, parties_dev, n_parties, n_cts, unit_first, n_units, noise, shares);
 }
 
 // Shares with the noise sampled ahead into `scratch` (scratch_bytes >= n_parties * N), in batches of

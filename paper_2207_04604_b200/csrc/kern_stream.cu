@@ -33,6 +33,7 @@ __global__ void __launch_bounds__(256)
   const u32 unit = blockIdx.x, i = unit / n_cts, c = unit % n_cts;
   const size_t ct_pairs = (size_t)v.L * v.n;  // 2*L*N residues = L*N pairs
   const u32 beg = offsets[i], end = offsets[i + 1];
+  const bool lazy = v.wide != 0 && end - beg < 64;
   ulonglong2* out = reinterpret_cast<ulonglong2*>(agg) + (size_t)unit * ct_pairs;
   for (size_t e = (size_t)blockIdx.y * blockDim.x + threadIdx.x; e < ct_pairs;
        e += (size_t)gridDim.y * blockDim.x) {
@@ -43,11 +44,27 @@ __global__ void __launch_bounds__(256)
     if (!D2MHE_CHK(v.chk, e, ct_pairs, SITE_ELEMENT) || !D2MHE_CHK(v.chk, l, v.L, SITE_LIMB)) continue;
     const u64 p = v.limbs[l].p;
     ulonglong2 acc = make_ulonglong2(0, 0);
-    for (u32 a = beg; a < end; ++a) {
-      const ulonglong2 x =
-          __ldg(reinterpret_cast<const ulonglong2*>(ct) + ((size_t)rows[a] * n_cts + c) * ct_pairs + e);
-      acc.x = addmod(acc.x, x.x, p);
-      acc.y = addmod(acc.y, x.y, p);
+    if (lazy) {
+      // primes below 2^57 and fewer than 64 addends: the plain 64-bit sums cannot overflow, so the
+      // loads are independent (several in flight per thread) and one reduction at the end replaces
+      // one per addend
+#pragma unroll 4
+      for (u32 a = beg; a < end; ++a) {
+        const ulonglong2 x =
+            __ldg(reinterpret_cast<const ulonglong2*>(ct) + ((size_t)rows[a] * n_cts + c) * ct_pairs + e);
+        acc.x += x.x;
+        acc.y += x.y;
+      }
+      const u64 one_sh = v.limbs[l].one_sh;
+      acc.x = shoup_full(acc.x, 1, one_sh, p);
+      acc.y = shoup_full(acc.y, 1, one_sh, p);
+    } else {
+      for (u32 a = beg; a < end; ++a) {
+        const ulonglong2 x =
+            __ldg(reinterpret_cast<const ulonglong2*>(ct) + ((size_t)rows[a] * n_cts + c) * ct_pairs + e);
+        acc.x = addmod(acc.x, x.x, p);
+        acc.y = addmod(acc.y, x.y, p);
+      }
     }
     out[e] = acc;
   }

@@ -861,7 +861,8 @@ def test_ciphertext_index_shards_reproduce_the_whole(d2):
 
 def test_sample_batches_of_one_call_reproduce_separate_calls(d2):
     """d2mhe_encrypt and d2mhe_partial_decrypt draw their samples into the context's 64 MiB scratch,
-    as many (party, ciphertext) or (recipient, ciphertext) units per pair of launches as fit.  A call
+    as many (party, ciphertext) or (recipient, ciphertext) units per pair of launches as fit (rounded
+    down to whole waves of thread blocks).  A call
     large enough to need several batches must produce, unit for unit, what one small call per slice
     of the index range produces (every sample is addressed by its counters, not by its batch)."""
     cfg = wl.round_config(1)
@@ -879,8 +880,11 @@ def test_sample_batches_of_one_call_reproduce_separate_calls(d2):
     ctx.encrypt(parties, 7, C, plain, whole)
     shares = ctx.empty_u64(K, K, C, 1, n)
     ctx.partial_decrypt(whole, parties, parties, 7, C, shares)
-    # batches end after 5461 encryption units (party 3, index 853) and after 4096 share units (recipient 2, index 1024)
-    for first, cnt in ((0, 3), (851, 5), (1022, 5), (C - 3, 3)):
+    # The scratch holds 5461 encryption units and 4096 share units; batches are cut to whole waves of
+    # thread blocks (592 resident blocks on a 148-SM device): 5328 encryption units (the first batch ends
+    # inside party 3 at index 720) and 3552 share units (inside recipient 2 at index 480).  The slices
+    # straddle those boundaries and the ones a cut at the scratch size would give.
+    for first, cnt in ((0, 3), (478, 5), (718, 5), (851, 5), (1022, 5), (C - 3, 3)):
         part = ctx.empty_u64(K, cnt, 2, 1, n)
         ctx.encrypt(parties, 7 + first, cnt, plain[:, first:first + cnt].contiguous(), part)
         assert torch.equal(part, whole[:, first:first + cnt])
