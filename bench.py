@@ -773,6 +773,7 @@ def run_sweep(args):
     flush = torch.empty(384 * 1024 * 1024, dtype=torch.uint8, device=dev)
     free_b, _ = torch.cuda.mem_get_info(dev)
     rows = []
+    imad_peak = None  # the mad.lo rate of this GPU, measured with the first context
     only = [int(x) for x in args.sweep_point.split(",")] if args.sweep_point else None  # N, L, batch
     for log2_n in wl.SWEEP_LOG2_N:
         n = 1 << log2_n
@@ -783,7 +784,10 @@ def run_sweep(args):
                 continue
             moduli = wl.sweep_moduli(args.sweep_bits, L)
             ctx = d2mhe.Context(log2_n, moduli, 1, seed=args.seed)
+            if imad_peak is None:
+                imad_peak = max(ctx.debug_int_throughput(0, 4096) for _ in range(3))
             narrow = args.sweep_bits <= 30
+            slots_per_bfly = 4 if narrow else SLOTS_PER_BUTTERFLY
             word = 4 if narrow else 8
             host_tile = wl.random_polys(moduli, log2_n, 1, args.seed)
             tile = torch.from_numpy(host_tile.astype(np.uint32).view(np.int32) if narrow else host_tile.view(np.int64)).to(dev)
@@ -825,12 +829,19 @@ def run_sweep(args):
                 for k_ in ("forward", "inverse", "muladd"):
                     if k_ + "_GBps" in row:
                         row[k_ + "_frac_of_hbm"] = row[k_ + "_GBps"] / peak
+                for k_ in ("forward", "inverse"):
+                    if k_ + "_GBps" in row:  # butterflies/s x slots per butterfly / measured mad.lo rate
+                        bfly = row[k_ + "_GBps"] * 1e9 / (2 * word) * log2_n / 2
+                        row[k_ + "_alu_frac"] = bfly * slots_per_bfly / imad_peak
                 rows.append(row)
                 del polys
                 torch.cuda.empty_cache()
             ctx.close()
     print(json.dumps({"metric": METRIC, "unit": "GB/s", "config": {"workload": "kernel-sweep", "prime_bits": args.sweep_bits},
                       "hbm_peak_GBps": peak, "peak_source": "of " + peak_kind,
+                      "integer_peak_slots_per_s": imad_peak,
+                      "integer_peak_source": "mad.lo.u32 rate measured in this run (d2mhe_debug_int_throughput); a "
+                                             "butterfly counts %d slots" % (4 if args.sweep_bits <= 30 else SLOTS_PER_BUTTERFLY),
                       "dtype": "u32" if args.sweep_bits <= 30 else "u64", "data": "synthetic", "rows": rows}))
 
 
