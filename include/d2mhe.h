@@ -76,8 +76,10 @@ typedef struct {
 } d2mhe_params;
 
 /* Validates params, builds all tables on `device` and allocates the context's device memory (tables,
- * key storage, index staging, and 64 MiB of scratch for the samples that d2mhe_encrypt and
- * d2mhe_partial_decrypt draw ahead of their kernels).  *out is NULL on failure. */
+ * key storage, index staging, and the scratch for the samples that d2mhe_encrypt,
+ * d2mhe_partial_decrypt, d2mhe_convert_share and d2mhe_bootstrap_share draw ahead of their kernels:
+ * 64 MiB, or what two waves of thread blocks of the share kernels need for this parameter set, at
+ * most 512 MiB; d2mhe_sample_scratch_bytes reports it).  *out is NULL on failure. */
 d2mhe_status d2mhe_create(const d2mhe_params* params, d2mhe_ctx** out);
 void d2mhe_destroy(d2mhe_ctx* ctx);
 /* Stream (a cudaStream_t passed as void*) on which later calls are enqueued; NULL = default. */
@@ -150,9 +152,10 @@ d2mhe_status d2mhe_aggregate(d2mhe_ctx* ctx, const uint64_t* ct_dev, uint32_t n_
  * e from chi on the stream (party k, recipient recipients[i], ciphertext index ct_first + c).
  * agg_dev: [n_rec, n_cts, 2, L, N];  shares_dev: out [n_rec, n_parties, n_cts, L, N].
  * recipients, parties: HOST arrays of indices < K.
- * The noise of the shares is sampled by a kernel of its own into a 64 MiB scratch buffer that the
+ * The noise of the shares is sampled by a kernel of its own into the scratch buffer that the
  * context owns (one byte per share coefficient; as many (recipient, ciphertext) pairs per launch as
- * fit), so the call is one or more pairs of launches on the context's stream.
+ * fit, rounded down to whole waves of thread blocks), so the call is one or more pairs of launches
+ * on the context's stream.
  * D2MHE_ERR_UNSUPPORTED if n_parties * N exceeds that buffer (d2mhe_convert_share and
  * d2mhe_bootstrap_share work the same way with 3 and 6 bytes per share coefficient).
  */
@@ -381,6 +384,9 @@ d2mhe_status d2mhe_get_root(const d2mhe_ctx* ctx, uint32_t limb, uint64_t* psi);
 d2mhe_status d2mhe_get_plain_root(const d2mhe_ctx* ctx, uint64_t* psi_t);
 /* Number of kernels this context has launched since creation. */
 uint64_t d2mhe_launch_count(const d2mhe_ctx* ctx);
+/* Bytes of the context's sample scratch (see d2mhe_create): a single call whose samples need more
+ * runs as several batches. */
+size_t d2mhe_sample_scratch_bytes(const d2mhe_ctx* ctx);
 
 #ifdef __cplusplus
 }

@@ -402,7 +402,16 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
     c->view.pk32 = dev_alloc<u64>(c, 2 * poly, &err);
     if (err != cudaSuccess) return fail_cuda(c, err);
   }
-  c->noise_scratch_bytes = kNoiseScratchBytes;
+  {
+    // two waves of thread blocks = 2 * resident / L (recipient, ciphertext) units of K shares each
+    int sms = 0;
+    err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+    if (err != cudaSuccess) return fail_cuda(c, err);
+    const size_t per_sm = logn == 12 ? 4 : logn == 13 ? 2 : 1;  // resident blocks of the transform kernels
+    const size_t units = (2 * (size_t)sms * per_sm + L - 1) / L;
+    const size_t want = units * P.num_parties * 6 * n;
+    c->noise_scratch_bytes = std::min(kNoiseScratchMaxBytes, std::max(kNoiseScratchBytes, (want + 255) / 256 * 256));
+  }
   c->noise_scratch = dev_alloc<unsigned char>(c, c->noise_scratch_bytes, &err);
   if (err != cudaSuccess) return fail_cuda(c, err);
   c->view.range_flag = dev_alloc<u32>(c, 4, &err);
@@ -1353,5 +1362,7 @@ d2mhe_status d2mhe_get_plain_root(const d2mhe_ctx* c, uint64_t* psi_t) {
 }
 
 uint64_t d2mhe_launch_count(const d2mhe_ctx* c) { return c ? c->launches : 0; }
+
+size_t d2mhe_sample_scratch_bytes(const d2mhe_ctx* c) { return c ? c->noise_scratch_bytes : 0; }
 
 }  // extern "C"

@@ -65,7 +65,10 @@ struct DevView {
 
 static const size_t kIdxSlotWords = (size_t)1 << 21;  // u32 words per staging slot (8 MiB)
 static const int kIdxSlots = 4;
-static const size_t kNoiseScratchBytes = (size_t)64 << 20;  // per context, for the single calls
+// Sample scratch of a context (for the single calls): 64 MiB, or what two waves of thread blocks of
+// the share kernel with the largest samples (MBFV.Bootstrap: 6 N bytes per share) need, up to 512 MiB.
+static const size_t kNoiseScratchBytes = (size_t)64 << 20;
+static const size_t kNoiseScratchMaxBytes = (size_t)512 << 20;
 #ifndef D2MHE_ROUND_LANES
 #define D2MHE_ROUND_LANES 2
 #endif

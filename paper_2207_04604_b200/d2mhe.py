@@ -35,7 +35,7 @@ EXPORTS = [
     "d2mhe_round_host", "d2mhe_round_device_static", "d2mhe_user_keygen", "d2mhe_convert_share",
     "d2mhe_convert_combine", "d2mhe_decrypt", "d2mhe_bootstrap_share", "d2mhe_bootstrap_combine", "d2mhe_debug_export_user_secret", "d2mhe_debug_export_secret", "d2mhe_debug_int_throughput", "d2mhe_debug_last_device_check",
     "d2mhe_debug_check_selftest", "d2mhe_get_root", "d2mhe_get_plain_root",
-    "d2mhe_launch_count",
+    "d2mhe_launch_count", "d2mhe_sample_scratch_bytes",
 ]
 
 
@@ -120,6 +120,8 @@ def load():
         lib.d2mhe_get_plain_root.argtypes = [vp, ctypes.POINTER(u64)]
         lib.d2mhe_launch_count.argtypes = [vp]
         lib.d2mhe_launch_count.restype = u64
+        lib.d2mhe_sample_scratch_bytes.argtypes = [vp]
+        lib.d2mhe_sample_scratch_bytes.restype = sz
         for name in EXPORTS:
             fn = getattr(lib, name)
             if fn.restype is ctypes.c_int:  # default: every remaining entry returns d2mhe_status
@@ -211,6 +213,9 @@ class Context:
 
     def launch_count(self):
         return int(load().d2mhe_launch_count(self._h))
+
+    def sample_scratch_bytes(self):
+        return int(load().d2mhe_sample_scratch_bytes(self._h))
 
     # ---- allocation helpers (torch is the allocator) ----
     def empty_u64(self, *shape):

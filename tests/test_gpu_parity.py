@@ -872,19 +872,24 @@ def test_sample_batches_of_one_call_reproduce_separate_calls(d2):
     parties = list(range(K))
     ctx.keygen_share(parties)
     ctx.collective_pk(parties)
-    C = 1536  # encrypt: 4 * 1536 units of 3 N bytes = 72 MiB; shares: 4 * 1536 units of 4 N bytes = 96 MiB
-    assert K * C * 3 * n > 64 << 20
+    scratch = ctx.sample_scratch_bytes()
+    assert scratch >= 64 << 20
+    cap_enc, cap_sh = scratch // (3 * n), scratch // (K * n)  # units that the scratch holds
+    C = -(-(cap_enc + 600) // K)  # enough indices that both calls need more than one batch
+    assert K * C > cap_enc > cap_sh
     gen = torch.Generator().manual_seed(3)
     plain = torch.randint(0, T, (K, C, n), dtype=torch.int32, generator=gen).to(ctx.device)
     whole = ctx.empty_u64(K, C, 2, 1, n)
     ctx.encrypt(parties, 7, C, plain, whole)
     shares = ctx.empty_u64(K, K, C, 1, n)
     ctx.partial_decrypt(whole, parties, parties, 7, C, shares)
-    # The scratch holds 5461 encryption units and 4096 share units; batches are cut to whole waves of
-    # thread blocks (592 resident blocks on a 148-SM device): 5328 encryption units (the first batch ends
-    # inside party 3 at index 720) and 3552 share units (inside recipient 2 at index 480).  The slices
-    # straddle those boundaries and the ones a cut at the scratch size would give.
-    for first, cnt in ((0, 3), (478, 5), (718, 5), (851, 5), (1022, 5), (C - 3, 3)):
+    # Batches are cut to whole waves of thread blocks (592 resident blocks of this kernel on a 148-SM
+    # device, one block per unit here).  The slices straddle the ends of the first batches under that
+    # rule and the ones a cut at the scratch size would give.
+    wave = 592
+    edges = {cap_enc // wave * wave, cap_enc, cap_sh // wave * wave, cap_sh}
+    firsts = sorted({0, C - 3} | {max(0, min(C - 5, e % C - 2)) for e in edges})
+    for first, cnt in [(f, 3 if f in (0, C - 3) else 5) for f in firsts]:
         part = ctx.empty_u64(K, cnt, 2, 1, n)
         ctx.encrypt(parties, 7 + first, cnt, plain[:, first:first + cnt].contiguous(), part)
         assert torch.equal(part, whole[:, first:first + cnt])
