@@ -1,6 +1,7 @@
 // Decryption shares: h = s_k c_1 + e for every listed share holder.
 #include <algorithm>
 
+#define D2MHE_SHIFT_AS_MULTIPLY 1  // see shoup_approx_sf: measured faster in this kernel only
 #include "d2mhe_kernels_common.cuh"
 
 namespace {
