@@ -1114,6 +1114,14 @@ def test_checked_build_gives_the_same_messages_and_reports_nothing(d2):
     assert np.array_equal(d2.to_u64_numpy(dp), polys)
     big.sync()
     big.close()
+    # the protocol calls on 32-bit words
+    n32_moduli = wl.ntt_primes(30, 2 << 10, 3)
+    n32 = d2.Context(10, n32_moduli, 3, seed=6, flags=d2.FLAG_DEVICE_CHECKS)
+    vals = np.random.default_rng(4).integers(-2000, 2001, size=(3, 3, 1 << 10)).astype(np.int32)
+    _run_round32(d2, n32, make_oracle(10, n32_moduli, seed=6), [0, 1, 2], np.array([0, 3, 3, 4], dtype=np.uint32),
+                 np.array([0, 1, 2, 2], dtype=np.uint32), vals, ct_first=1, also_64=False)
+    n32.sync()
+    n32.close()
     narrow = d2.Context(12, small_moduli(12, 30, 2), 1, seed=1, flags=d2.FLAG_DEVICE_CHECKS)
     p32 = wl.random_polys(narrow.moduli, 12, 3, seed=4).astype(np.uint32)
     d32 = d2.from_u32_numpy(p32, narrow.device)
