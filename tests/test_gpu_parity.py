@@ -1041,6 +1041,49 @@ def test_mnist_shaped_round_on_30_bit_limbs_every_message(d2):
     ctx.close()
 
 
+def test_32_bit_calls_in_several_batches_reproduce_separate_calls(d2):
+    """d2mhe_encrypt32 / d2mhe_partial_decrypt32 with more units than the sample scratch holds run as
+    several batches (whole pairs of units, whole waves of thread blocks); an odd total leaves the last
+    thread block with one unit.  Unit for unit they must equal small calls on slices of the index range."""
+    log2_n, K = 12, 3
+    n = 1 << log2_n
+    moduli = wl.ntt_primes(30, 2 << log2_n, 1)
+    ctx = d2.Context(log2_n, moduli, K, seed=11)
+    parties = list(range(K))
+    ctx.keygen_share(parties)
+    ctx.collective_pk(parties)
+    scratch = ctx.sample_scratch_bytes()
+    cap_enc, cap_sh = scratch // (3 * n), scratch // (K * n)
+    C = -(-(cap_sh + 700) // K) | 1  # odd, so that K * C is odd too: the last pair is a single unit
+    assert K * C > max(cap_sh, cap_enc) and (K * C) % 2 == 1
+    gen = torch.Generator().manual_seed(5)
+    plain = torch.randint(0, T, (K, C, n), dtype=torch.int32, generator=gen).to(ctx.device)
+    whole = ctx.empty_u32(K, C, 2, 1, n)
+    ctx.encrypt32(parties, 3, C, plain, whole)
+    shares = ctx.empty_u32(K, K, C, 1, n)
+    ctx.partial_decrypt32(whole, parties, parties, 3, C, shares)
+    wave = 592  # resident thread blocks of this kernel on a 148-SM device; one block per pair of units
+    edges = {2 * (cap_enc // 2 // wave * wave), cap_enc, 2 * (cap_sh // 2 // wave * wave), cap_sh}
+    firsts = sorted({0, C - 3} | {max(0, min(C - 5, e % C - 2)) for e in edges})
+    for first in firsts:
+        cnt = 3 if first in (0, C - 3) else 5
+        part = ctx.empty_u32(K, cnt, 2, 1, n)
+        ctx.encrypt32(parties, 3 + first, cnt, plain[:, first:first + cnt].contiguous(), part)
+        assert torch.equal(part, whole[:, first:first + cnt])
+        sh = ctx.empty_u32(K, K, cnt, 1, n)
+        ctx.partial_decrypt32(part, parties, parties, 3 + first, cnt, sh)
+        assert torch.equal(sh, shares[:, :, first:first + cnt])
+    # and against the oracle on the last (single-unit) pair
+    o = make_oracle(log2_n, moduli, seed=11)
+    pk = o.collective_pk(parties)
+    last = C - 1
+    want_ct = o.encrypt(pk, parties, 3 + last, d2.to_u32_numpy(plain[:, last:last + 1].contiguous()))
+    assert np.array_equal(d2.to_u32_numpy(whole[:, last:last + 1].contiguous()).astype(np.uint64), want_ct)
+    want_sh = o.partial_decrypt(want_ct, parties, parties, 3 + last)
+    assert np.array_equal(d2.to_u32_numpy(shares[:, :, last:last + 1].contiguous()).astype(np.uint64), want_sh)
+    ctx.close()
+
+
 def test_32_bit_protocol_calls_refuse_wide_primes(d2):
     cfg = wl.round_config(1)
     ctx = d2.Context(cfg.log2_n, cfg.moduli, 2, seed=1)
