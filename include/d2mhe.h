@@ -288,8 +288,8 @@ d2mhe_status d2mhe_combine_decrypt32(d2mhe_ctx* ctx, const uint32_t* agg_dev, co
  * and memory-bound kernels overlap another's arithmetic; the internal streams start after
  * the work already queued on the context's stream, and the context's stream continues
  * after they have finished (so the call behaves like one operation on that stream).
- *   values:  int32 [K, n_cts, N]   in
- *   sums:    int32 [K, n_cts, N]   out: sums[i] = sum over list(i) of the values
+ *   values:  int32 [K, n_cts, N]   in (d2mhe_round_device reads it in place, sub-chunk by sub-chunk)
+ *   sums:    int32 [K, n_cts, N]   out: sums[i] = sum over list(i) of the values (written in place)
  *   nbr_offsets / nbr_rows: HOST CSR lists over parties, K lists.
  *   workspace_dev / workspace_bytes: device scratch, at least
  *   d2mhe_round_workspace_bytes(ctx, 1); d2mhe_round_workspace_bytes(ctx, n_cts) holds
@@ -308,8 +308,8 @@ size_t d2mhe_round_workspace_bytes(const d2mhe_ctx* ctx, uint32_t chunk_cts);
  * (may be NULL) and the number of internal streams used to *lanes_out (may be NULL); returns the
  * number of sub-chunks, 0 for n_cts == 0 or cap_cts == 0.  Sub-chunk i runs on stream i mod
  * lanes; sizes differ by at most one, larger ones first; the sizes of the first `lanes`
- * sub-chunks add up to at most cap_cts.  (d2mhe_round_host cuts by the same rule over three
- * streams.)
+ * sub-chunks add up to at most cap_cts.  Fewer than four indices run on one stream.
+ * (d2mhe_round_host cuts by the same rule over three streams.)
  */
 uint32_t d2mhe_round_plan(uint32_t n_cts, uint64_t cap_cts, uint32_t* sizes, uint32_t max_out,
                           uint32_t* lanes_out);

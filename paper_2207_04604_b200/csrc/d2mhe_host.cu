@@ -444,6 +444,12 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
     if (err != cudaSuccess) return fail_cuda(c, err);
     c->idx_event_valid[i] = false;
   }
+  err = cudaMallocHost(reinterpret_cast<void**>(&c->round_lists_host), kIdxSlotWords * sizeof(u32));
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  c->round_lists_dev = dev_alloc<u32>(c, kIdxSlotWords, &err);
+  if (err != cudaSuccess) return fail_cuda(c, err);
+  err = cudaEventCreateWithFlags(&c->round_lists_event, cudaEventDisableTiming);
+  if (err != cudaSuccess) return fail_cuda(c, err);
   // lanes of the whole-round entry points
   for (int i = 0; i < kRoundLanes; ++i) {
     err = cudaStreamCreateWithFlags(&c->lane_stream[i], cudaStreamNonBlocking);
@@ -544,6 +550,8 @@ void d2mhe_destroy(d2mhe_ctx* c) {
   cudaDeviceSynchronize();
   for (void* p : c->allocs) cudaFree(p);
   if (c->idx_host) cudaFreeHost(c->idx_host);
+  if (c->round_lists_host) cudaFreeHost(c->round_lists_host);
+  if (c->round_lists_event) cudaEventDestroy(c->round_lists_event);
   for (int i = 0; i < kIdxSlots; ++i)
     if (c->idx_event[i]) cudaEventDestroy(c->idx_event[i]);
   for (int i = 0; i < kRoundLanes; ++i) {
@@ -1131,6 +1139,8 @@ struct RoundPlan {
 };
 static RoundPlan plan_round(u32 n_cts, size_t cap, size_t max_sub, int max_lanes) {
   RoundPlan pl;
+  // fewer than four indices: one stream (the fork and join of a second one cost more than they hide)
+  if (n_cts < 4) max_lanes = 1;
   pl.lanes = (u32)std::min<size_t>(std::min<size_t>(max_lanes, cap), n_cts);
   u32 n_sub = pl.lanes;
   for (;; n_sub += pl.lanes) {
@@ -1192,11 +1202,36 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
 
   DeviceGuard guard(c->device);
   const u32 dummy = 0;
-  Staged sg;  // the four index lists of every sub-chunk, staged once
+  // The four index lists of every sub-chunk.  They rarely change from one round to the next, so they
+  // stay on the device and are uploaded (stream-ordered after the earlier rounds that read them) only
+  // when they differ from what is there.
+  Staged sg;
   const u32* arrays[4] = {c->all_parties.data(), c->pk_parties.data(), nbr_offsets, nnz ? nbr_rows : &dummy};
   const size_t counts[4] = {K, S, (size_t)K + 1, nnz ? (size_t)nnz : 1};
-  d2mhe_status st = stage_indices(c, arrays, counts, 4, &sg);
-  if (st != D2MHE_OK) return st;
+  d2mhe_status st = D2MHE_OK;
+  {
+    size_t off[5] = {0, 0, 0, 0, 0};
+    for (int i = 0; i < 4; ++i) off[i + 1] = off[i] + ((counts[i] + 3) & ~(size_t)3);
+    if (off[4] > kIdxSlotWords) return D2MHE_ERR_RANGE;
+    bool same = c->round_lists_valid && c->round_lists_cache.size() == off[4];
+    for (int i = 0; same && i < 4; ++i)
+      same = std::memcmp(c->round_lists_cache.data() + off[i], arrays[i], counts[i] * sizeof(u32)) == 0;
+    if (!same) {
+      cudaError_t e2 = c->round_lists_valid ? cudaEventSynchronize(c->round_lists_event) : cudaSuccess;  // the pinned source is free again
+      if (e2 != cudaSuccess) return fail_cuda(c, e2);
+      c->round_lists_valid = false;
+      c->round_lists_cache.assign(off[4], 0u);
+      for (int i = 0; i < 4; ++i)
+        std::memcpy(c->round_lists_cache.data() + off[i], arrays[i], counts[i] * sizeof(u32));
+      std::memcpy(c->round_lists_host, c->round_lists_cache.data(), off[4] * sizeof(u32));
+      e2 = cudaMemcpyAsync(c->round_lists_dev, c->round_lists_host, off[4] * sizeof(u32), cudaMemcpyHostToDevice,
+                           c->stream);
+      if (e2 == cudaSuccess) e2 = cudaEventRecord(c->round_lists_event, c->stream);
+      if (e2 != cudaSuccess) return fail_cuda(c, e2);
+      c->round_lists_valid = true;
+    }
+    for (int i = 0; i < 4; ++i) sg.dev[i] = c->round_lists_dev + off[i];
+  }
   unsigned char* base = reinterpret_cast<unsigned char*>(ws);
   // Everything between the fork and the join; a failure stops issuing, and the join below still runs,
   // so that the context's stream stays ordered after whatever the lanes were given.
@@ -1217,13 +1252,21 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
       u64* ct = reinterpret_cast<u64*>(lane_base + (size_t)K * cc * n * sizeof(u32));
       u64* agg = ct + (size_t)K * cc * 2 * polyw;
       u64* shares = agg + (size_t)K * cc * 2 * polyw;
-      int32_t* vals_dev = reinterpret_cast<int32_t*>(plain);  // encode and decode run in place
-      // values are [K, n_cts, N]: one strided copy, K rows of cc*N values, rows n_cts*N apart
-      e = cudaMemcpy2DAsync(vals_dev, (size_t)cc * n * sizeof(int32_t), values + (size_t)done * n,
-                            (size_t)n_cts * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
-                            host_io ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice, s);
-      if (e != cudaSuccess) return e;
-      if ((e = L_(encode)(c->view, s, vals_dev, K * cc, plain)) != cudaSuccess) return e;
+      int32_t* vals_dev = reinterpret_cast<int32_t*>(plain);  // with host buffers encode and decode run in place
+      // values are [K, n_cts, N]: the sub-chunk is K groups of cc rows, groups n_cts*N apart.  Device
+      // buffers are read and written in place by the packing kernels; host buffers go through one
+      // strided copy each way.
+      if (host_io) {
+        e = cudaMemcpy2DAsync(vals_dev, (size_t)cc * n * sizeof(int32_t), values + (size_t)done * n,
+                              (size_t)n_cts * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
+                              cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return e;
+        if ((e = L_(encode)(c->view, s, vals_dev, K * cc, plain)) != cudaSuccess) return e;
+      } else {
+        if ((e = L_(encode_strided)(c->view, s, values + (size_t)done * n, K, cc, (size_t)n_cts * n, plain)) !=
+            cudaSuccess)
+          return e;
+      }
       unsigned char* noise = reinterpret_cast<unsigned char*>(shares + (size_t)K * S * cc * polyw);
       const size_t noise_bytes = round_noise_bytes_per_ct(c) * cc;  // first u, e_0, e_1, later the shares' noise
       u32 enc_launches = 0;
@@ -1237,12 +1280,18 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
           cudaSuccess)
         return e;
       if ((e = L_(combine)(c->view, s, agg, shares, K, S, 1, cc, plain)) != cudaSuccess) return e;
-      if ((e = L_(decode)(c->view, s, plain, K * cc, vals_dev)) != cudaSuccess) return e;
       c->launches += 4 + enc_launches + pdec_launches;
-      e = cudaMemcpy2DAsync(sums + (size_t)done * n, (size_t)n_cts * n * sizeof(int32_t), vals_dev,
-                            (size_t)cc * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
-                            host_io ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice, s);
-      if (e != cudaSuccess) return e;
+      if (host_io) {
+        if ((e = L_(decode)(c->view, s, plain, K * cc, vals_dev)) != cudaSuccess) return e;
+        e = cudaMemcpy2DAsync(sums + (size_t)done * n, (size_t)n_cts * n * sizeof(int32_t), vals_dev,
+                              (size_t)cc * n * sizeof(int32_t), (size_t)cc * n * sizeof(int32_t), K,
+                              cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return e;
+      } else {
+        if ((e = L_(decode_strided)(c->view, s, plain, K, cc, (size_t)n_cts * n, sums + (size_t)done * n)) !=
+            cudaSuccess)
+          return e;
+      }
       done += cc;
     }
     return cudaSuccess;
@@ -1255,8 +1304,7 @@ static d2mhe_status round_impl(d2mhe_ctx* c, const int32_t* values, bool host_io
       if (e == cudaSuccess) e = j;
     }
   }
-  if (e != cudaSuccess) return fail_staged(c, sg, e);
-  if ((st = release_slot(c, sg)) != D2MHE_OK) return st;
+  if (e != cudaSuccess) return fail_cuda(c, e);
   if (host_io) {
     // the call returns when the sums are in host memory, so it can also report values that
     // d2mhe_encode found out of range (the flag is cleared, as d2mhe_sync does)

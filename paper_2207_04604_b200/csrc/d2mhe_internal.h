@@ -106,6 +106,13 @@ struct d2mhe_ctx {
   cudaEvent_t idx_event[kIdxSlots] = {};
   bool idx_event_valid[kIdxSlots] = {};
   int idx_next = 0;
+  // the four index lists of the whole-round calls: kept on the device from one call to the next and
+  // uploaded again only when they change
+  u32* round_lists_host = nullptr;        // pinned
+  u32* round_lists_dev = nullptr;
+  std::vector<u32> round_lists_cache;     // what round_lists_dev holds
+  cudaEvent_t round_lists_event = nullptr;  // after the last upload
+  bool round_lists_valid = false;
   cudaStream_t lane_stream[kRoundLanes] = {};
   cudaEvent_t lane_event[kRoundLanes] = {};
   cudaEvent_t fork_event = nullptr;
@@ -141,6 +148,10 @@ cudaError_t int_probe(const DevView& v, const LimbParams& lp, cudaStream_t s, u3
 cudaError_t export_secret(const DevView& v, const LimbParams& lp, cudaStream_t s, const u64* key, signed char* out); \
 cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain); \
 cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values); \
+cudaError_t encode_strided(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_groups, u32 group, \
+                           size_t group_stride, u32* plain); \
+cudaError_t decode_strided(const DevView& v, cudaStream_t s, const u32* plain, u32 n_groups, u32 group, \
+                           size_t group_stride, int32_t* values); \
 cudaError_t encrypt(const DevView& v, const LimbParams& lp, cudaStream_t s, const u32* parties_dev, u32 n_parties, \
                     u32 ct_first, u32 n_cts, const u32* plain, u64* ct, void* scratch, size_t scratch_bytes, \
                     u32* launches); \

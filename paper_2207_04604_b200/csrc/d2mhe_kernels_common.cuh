@@ -27,8 +27,13 @@
 
 namespace {
 
-constexpr int ntt_minb_ct(int logn) {
-  return logn == 12 ? D2MHE_MINB12 : logn == 13 ? D2MHE_MINB13 : logn == 14 ? D2MHE_MINB14 : 1;
+// Resident thread blocks per SM that the kernels of ring degree 2^logn are compiled for.  A build
+// with fewer octets per thread than the default (more threads per polynomial: the low-latency
+// variants of small calls) is compiled for two blocks per SM (64 registers at 512 threads).
+constexpr int ntt_default_g(int logn) { return logn == 12 ? D2MHE_G12 : logn == 13 ? D2MHE_G13 : logn == 14 ? D2MHE_G14 : 1; }
+constexpr int ntt_minb_ct(int logn, int g) {
+  return g != ntt_default_g(logn) ? 2
+                                  : logn == 12 ? D2MHE_MINB12 : logn == 13 ? D2MHE_MINB13 : logn == 14 ? D2MHE_MINB14 : 1;
 }
 
 // Shared-memory layout of the transform kernels: [GaussTab][polynomial].
@@ -116,7 +121,7 @@ constexpr u32 ntt_threads_ct(int logn, int g) {
 }
 
 // Thread blocks of a transform kernel that the device holds at once.
-inline u32 resident_ctas(const DevView& v) { return v.sms * (u32)ntt_minb_ct((int)v.logn); }
+inline u32 resident_ctas(const DevView& v) { return v.sms * (u32)ntt_minb_ct((int)v.logn, ntt_default_g((int)v.logn)); }
 // A call that must be cut into batches (its scratch holds `cap` of its `n_units` units, each unit
 // ctas_per_unit thread blocks) takes batches of whole waves of thread blocks when a batch is at least
 // one wave: a batch that ends part-way through a wave leaves SMs idle until its last blocks finish.
@@ -171,8 +176,11 @@ cudaError_t launch_clustered(void (*kernel)(KArgs...), u32 grid, u32 threads, si
 }
 
 // D2MHE_EXTRA_TARGS: further template arguments of the kernel (", true"), empty by default; a
-// translation unit redefines it around the launcher that needs them.
+// translation unit redefines it around the launcher that needs them.  D2MHE_DISPATCH_G12: octets per
+// thread that the dispatch below uses for N = 4096 (the default, or 1 around the launchers of the
+// low-latency variants).
 #define D2MHE_EXTRA_TARGS
+#define D2MHE_DISPATCH_G12 D2MHE_G12
 #define D2MHE_LAUNCH_ONE(KERNEL, LOGN_, G_, WIDE_, grid, stream, cs, ...)                      \
   do {                                                                                         \
     cudaError_t e_ = launch_clustered(KERNEL<LOGN_, G_, WIDE_ D2MHE_EXTRA_TARGS>, grid, ntt_threads(n_, G_), \
@@ -199,7 +207,7 @@ cudaError_t launch_clustered(void (*kernel)(KArgs...), u32 grid, u32 threads, si
     const bool wide_ = (view).wide != 0;                                                       \
     switch (logn_) {                                                                           \
       case 12:                                                                                 \
-        D2MHE_LAUNCH_W(KERNEL, 12, D2MHE_G12, wide_, grid, stream, cs, __VA_ARGS__);           \
+        D2MHE_LAUNCH_W(KERNEL, 12, D2MHE_DISPATCH_G12, wide_, grid, stream, cs, __VA_ARGS__);  \
         break;                                                                                 \
       case 13:                                                                                 \
         D2MHE_LAUNCH_W(KERNEL, 13, D2MHE_G13, wide_, grid, stream, cs, __VA_ARGS__);           \

@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(256)
 // Iterations -2 and -1 run the two forward transforms, iteration a >= 0 produces share a, so that
 // one forward and one inverse call site serve the whole kernel.
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_boot_share(DevView v, const __grid_constant__ LimbParams lp, const u64* __restrict__ agg,
                  const u32* __restrict__ recipients, const u32* __restrict__ parties, u32 n_parties,
                  u32 ct_first, u32 n_cts, u32 unit_first, const u32* __restrict__ sampled, u64* shares) {

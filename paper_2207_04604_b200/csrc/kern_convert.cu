@@ -16,7 +16,7 @@ __device__ __forceinline__ void store_octet_mont(u64* __restrict__ dst, u64 (&x)
 // pk_i = (-(sk_i p_{1,i} + e_i), p_{1,i}) with p_{1,i} uniform (BFV.PubKeyGen).  grid = n_users * L.
 // NTT(p_{1,i}) is parked in the row that finally receives p_{0,i}.
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_user_keygen(DevView v, const __grid_constant__ LimbParams lp, const u32* __restrict__ users) {
   const u32 l = blockIdx.x % v.L, user = users[blockIdx.x / v.L];
   if (!D2MHE_CHK(v.chk, user, v.K, SITE_PARTY)) return;
@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(256)
 // grid = n_units * L; units unit_first .. unit_first + n_units - 1 of the (recipient, ciphertext) grid.
 // NTT(c_1) is parked in the h_0 row of the last share, NTT(mu_k) in the h_1 row of its own share.
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_convert_share(DevView v, const __grid_constant__ LimbParams lp, const u64* __restrict__ agg,
                     const u32* __restrict__ recipients, const u32* __restrict__ parties, u32 n_parties,
                     u32 n_cts, u32 unit_first, const u32* __restrict__ sampled, u64* shares) {
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(256)
 // c_1 sk_i for BFV.Decrypt under the user's own key.  grid = n_users * n_cts * L.
 // NTT(c_1) is parked in the output row.
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_secret_product(DevView v, const __grid_constant__ LimbParams lp, const u64* __restrict__ ct,
                      const u32* __restrict__ users, u32 n_cts, u64* prod) {
   const u32 l = blockIdx.x % v.L, unit = blockIdx.x / v.L;

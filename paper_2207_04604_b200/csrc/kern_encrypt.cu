@@ -87,13 +87,13 @@ __device__ __forceinline__ void encrypt_body(const DevView& v, const LimbParams&
 }
 
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_encrypt(DevView v, const __grid_constant__ LimbParams lp, u32 unit_first, const u32* __restrict__ sampled,
               const u32* __restrict__ plain, u64* ct) {
   encrypt_body<LOGN, G, WIDE, false>(v, lp, unit_first, sampled, plain, ct);
 }
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_encrypt_split(DevView v, const __grid_constant__ LimbParams lp, u32 unit_first, const u32* __restrict__ sampled,
                     const u32* __restrict__ plain, u64* ct) {
   encrypt_body<LOGN, G, WIDE, true>(v, lp, unit_first, sampled, plain, ct);
@@ -112,14 +112,22 @@ cudaError_t sample_encrypt_noise(const DevView& v, cudaStream_t s, const u32* pa
   return cudaGetLastError();
 }
 
+// The split variant serves calls of a few thread blocks, where the latency of one block's transforms is
+// what counts: at N = 4096 it runs with one octet per thread and round (512 threads per polynomial).
+#undef D2MHE_DISPATCH_G12
+#define D2MHE_DISPATCH_G12 1
+static cudaError_t encrypt_units_split(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 unit_first,
+                                       u32 n_units, const u32* sampled, const u32* plain, u64* ct) {
+  D2MHE_DISPATCH_EX(k_encrypt_split, v, n_units * v.L * 2, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain,
+                    ct);
+}
+#undef D2MHE_DISPATCH_G12
+#define D2MHE_DISPATCH_G12 D2MHE_G12
+
 static cudaError_t encrypt_units(const DevView& v, const LimbParams& lp, cudaStream_t s, u32 unit_first, u32 n_units,
                                  const u32* sampled, const u32* plain, u64* ct) {
   // a small call (at most half of the thread blocks that the GPU holds at once) uses one block per component
-  const u32 resident = resident_ctas(v);
-  if (n_units * v.L * 2 <= resident) {
-    D2MHE_DISPATCH_EX(k_encrypt_split, v, n_units * v.L * 2, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain,
-                      ct);
-  }
+  if (n_units * v.L * 2 <= resident_ctas(v)) return encrypt_units_split(v, lp, s, unit_first, n_units, sampled, plain, ct);
   D2MHE_DISPATCH_EX(k_encrypt, v, n_units * v.L, s, 3 * (size_t)v.n, 1, v, lp, unit_first, sampled, plain, ct);
 }
 

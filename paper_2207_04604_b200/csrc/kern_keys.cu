@@ -5,7 +5,7 @@ namespace {
 
 // s_k from R_3, kept as NTT(s_k) * N^-1 in Montgomery form.   grid = n_parties * L
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_keygen(DevView v, const __grid_constant__ LimbParams lp, const u32* __restrict__ parties) {
   const u32 l = blockIdx.x % v.L, party = parties[blockIdx.x / v.L];
   if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY)) return;
@@ -24,7 +24,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 // p_1 uniform; p_{0,k} = -(p_1 s_k + e_k); p_0 = sum_k p_{0,k}.
 // grid = L: one CTA per limb walks over the parties.
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_collective_pk(DevView v, const __grid_constant__ LimbParams lp, const u32* __restrict__ parties, u32 n_parties,
                     u64* __restrict__ shares_out) {
   const u32 l = blockIdx.x;
@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 // the coefficient domain; out[l][j] = the coefficient as -1, 0 or 1, or 127 if the residue of limb l
 // is none of these.   grid = L
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_export_secret(DevView v, const __grid_constant__ LimbParams lp, const u64* key, signed char* __restrict__ out) {
   const u32 l = blockIdx.x;
   const LimbTab& lt = lp.limbs[l];

@@ -4,7 +4,7 @@
 namespace {
 
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_ntt_fwd(DevView v, const __grid_constant__ LimbParams lp, u64* __restrict__ polys) {
   const u32 l = blockIdx.x % v.L;
   const LimbTab& lt = lp.limbs[l];
@@ -19,7 +19,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 }
 
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_ntt_inv(DevView v, const __grid_constant__ LimbParams lp, u64* __restrict__ polys) {
   const u32 l = blockIdx.x % v.L;
   const LimbTab& lt = lp.limbs[l];
@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(256)
 
 // Pass B: block b of polynomial-limb r; grid = batch * L * 2^soff.
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_ntt_fwd_blk(DevView v, const __grid_constant__ LimbParams lp, u64* __restrict__ polys, u32 soff) {
   const u32 b = blockIdx.x & ((1u << soff) - 1), r = blockIdx.x >> soff;
   const LimbTab& lt = lp.limbs[r % v.L];
@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
       soff, b);
 }
 template <int LOGN, int G, bool WIDE>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_ntt_inv_blk(DevView v, const __grid_constant__ LimbParams lp, u64* __restrict__ polys, u32 soff) {
   const u32 b = blockIdx.x & ((1u << soff) - 1), r = blockIdx.x >> soff;
   const LimbTab& lt = lp.limbs[r % v.L];

@@ -35,7 +35,7 @@ __device__ __forceinline__ void load_octet_pair(const u32* a, const u32* b, u64 
 }
 
 template <int LOGN, int G>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_ntt32_fwd(DevView v, const __grid_constant__ LimbParams lp, u32* __restrict__ polys, u32 batch) {
   const LimbTab& lt = lp.limbs[blockIdx.x % v.L];
   const Rows32 r = rows_of(v, polys, batch);
@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 }
 
 template <int LOGN, int G>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_ntt32_inv(DevView v, const __grid_constant__ LimbParams lp, u32* __restrict__ polys, u32 batch) {
   const LimbTab& lt = lp.limbs[blockIdx.x % v.L];
   const Rows32 r = rows_of(v, polys, batch);

@@ -80,7 +80,7 @@ __device__ __forceinline__ u32 add_small_canon32(u32 v, int e, u32 p) {
 // sampled: [u | e_0 | e_1] bytes per unit of this launch (as for the 64-bit kernel).
 // NTT(u) of both units is parked in their c_1 rows.
 template <int LOGN, int G>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_encrypt32(DevView v, const __grid_constant__ LimbParams lp, u32 unit_first, u32 n_units,
                 const u32* __restrict__ sampled, const u32* __restrict__ plain, u32* ct) {
   const u32 l = blockIdx.x % v.L;
@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
 // noise[(u * n_parties + a) * N + j] for local unit u, as for the 64-bit kernel.
 // NTT(c_1) of both units is parked in the rows of their last shares.
 template <int LOGN, int G>
-__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN))
+__global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     k_partial_decrypt32(DevView v, const __grid_constant__ LimbParams lp, const u32* __restrict__ agg,
                         const u32* __restrict__ parties, u32 n_parties, u32 n_cts, u32 unit_first, u32 n_units,
                         const signed char* __restrict__ noise, u32* shares) {

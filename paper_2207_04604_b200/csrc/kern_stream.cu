@@ -166,11 +166,13 @@ __device__ __forceinline__ void ct32(u32& X, u32& Y, uint2 w, u32 t, u32 twot) {
 // values and plain may be the same storage (every CTA reads its whole row into shared memory before
 // it writes the row back), so neither pointer is declared __restrict__
 __global__ void __launch_bounds__(1024)
-    k_encode(DevView v, const int32_t* values, u32* plain) {
+    k_encode(DevView v, const int32_t* values, u32* plain, u32 group, size_t group_stride) {
   u32* sm = reinterpret_cast<u32*>(smem_raw);
   const PlainTab pt = v.plain;
   const u32 n = v.n, logn = v.logn, t = pt.t, twot = pt.twot;
-  const int32_t* in = values + (size_t)blockIdx.x * n;
+  // the values of block b = (g, c), c < group, start at g * group_stride + c * N: contiguous rows when
+  // group_stride = group * N, a slice of a larger [.., n_cts, N] array otherwise
+  const int32_t* in = values + (size_t)(blockIdx.x / group) * group_stride + (size_t)(blockIdx.x % group) * n;
   u32* out = plain + (size_t)blockIdx.x * n;
   bool bad = false;
   for (u32 j = threadIdx.x; j < n; j += blockDim.x) {
@@ -221,12 +223,12 @@ __global__ void __launch_bounds__(1024)
 // decode: forward transform (two stages per barrier), slots read back from bit-reversed positions
 // plain and values may be the same storage (see k_encode)
 __global__ void __launch_bounds__(1024)
-    k_decode(DevView v, const u32* plain, int32_t* values) {
+    k_decode(DevView v, const u32* plain, int32_t* values, u32 group, size_t group_stride) {
   u32* sm = reinterpret_cast<u32*>(smem_raw);
   const PlainTab pt = v.plain;
   const u32 n = v.n, logn = v.logn, t = pt.t, twot = pt.twot;
   const u32* in = plain + (size_t)blockIdx.x * n;
-  int32_t* out = values + (size_t)blockIdx.x * n;
+  int32_t* out = values + (size_t)(blockIdx.x / group) * group_stride + (size_t)(blockIdx.x % group) * n;  // as in k_encode
   for (u32 j = threadIdx.x; j < n; j += blockDim.x) sm[j] = in[j];
   __syncthreads();
   int lt = (int)logn - 1;  // log2 span of the next stage (m = n >> (lt + 1) groups)
@@ -314,22 +316,32 @@ cudaError_t combine32(const DevView& v, cudaStream_t s, const u32* agg, const u3
   return combine_words<u32>(v, s, agg, shares, n_rec, n_shares, 1, n_cts, plain);
 }
 
-cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain) {
+// values: n_groups groups of `group` rows of N values, group g starting at values + g * group_stride
+// (elements); plain: [n_groups * group, N] contiguous
+cudaError_t encode_strided(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_groups, u32 group,
+                           size_t group_stride, u32* plain) {
   const size_t smem = (size_t)v.n * 4;
   cudaError_t e = set_smem(k_encode, smem);
   if (e != cudaSuccess) return e;
   u32 threads = v.n / 4 < 1024 ? (v.n / 4 < 32 ? 32 : v.n / 4) : 1024;
-  k_encode<<<n_cts, threads, smem, s>>>(v, values, plain);
+  k_encode<<<n_groups * group, threads, smem, s>>>(v, values, plain, group, group_stride);
   return cudaGetLastError();
 }
+cudaError_t encode(const DevView& v, cudaStream_t s, const int32_t* values, u32 n_cts, u32* plain) {
+  return encode_strided(v, s, values, 1, n_cts, (size_t)n_cts * v.n, plain);
+}
 
-cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values) {
+cudaError_t decode_strided(const DevView& v, cudaStream_t s, const u32* plain, u32 n_groups, u32 group,
+                           size_t group_stride, int32_t* values) {
   const size_t smem = (size_t)v.n * 4;
   cudaError_t e = set_smem(k_decode, smem);
   if (e != cudaSuccess) return e;
   u32 threads = v.n / 4 < 1024 ? (v.n / 4 < 32 ? 32 : v.n / 4) : 1024;
-  k_decode<<<n_cts, threads, smem, s>>>(v, plain, values);
+  k_decode<<<n_groups * group, threads, smem, s>>>(v, plain, values, group, group_stride);
   return cudaGetLastError();
+}
+cudaError_t decode(const DevView& v, cudaStream_t s, const u32* plain, u32 n_cts, int32_t* values) {
+  return decode_strided(v, s, plain, 1, n_cts, (size_t)n_cts * v.n, values);
 }
 
 }  // namespace D2MHE_LAUNCH_NS

@@ -87,7 +87,7 @@ def test_round_plan_invariants():
     for n_cts in list(range(1, 40)) + [66, 683, 1000]:
         for cap in list(range(1, 12)) + [13, 23, 66, 100, 5000]:
             sizes, lanes = d2mhe.round_plan(n_cts, cap)
-            assert lanes == min(2, cap, n_cts)
+            assert lanes == min(2 if n_cts >= 4 else 1, cap, n_cts)  # fewer than four indices: one stream
             assert sum(sizes) == n_cts and min(sizes) >= 1
             assert max(sizes) - min(sizes) <= 1
             assert sizes == sorted(sizes, reverse=True)
@@ -103,4 +103,6 @@ def test_round_plan_invariants():
     assert d2mhe.round_plan(13, 13) == ([7, 6], 2)
     assert d2mhe.round_plan(13, 3) == ([2] + [1] * 11, 2)
     assert d2mhe.round_plan(13, 1) == ([1] * 13, 1)
-    assert d2mhe.round_plan(2, 100) == ([1, 1], 2)
+    assert d2mhe.round_plan(2, 100) == ([2], 1)
+    assert d2mhe.round_plan(3, 2) == ([2, 1], 1)
+    assert d2mhe.round_plan(4, 100) == ([2, 2], 2)
