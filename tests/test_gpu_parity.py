@@ -836,6 +836,37 @@ def test_round_driver_matches_stepwise_and_plain_sums(d2):
     ctx.close()
 
 
+def test_round_calls_follow_changed_index_lists(d2):
+    """The whole-round calls keep their index lists on the device between calls; a call with other
+    neighbour lists, or after another collective key, must use the new ones."""
+    cfg = wl.round_config(1)
+    K, n = cfg.num_parties, cfg.n
+    ctx = d2.Context(cfg.log2_n, cfg.moduli, K, seed=8)
+    ctx.keygen_share(list(range(K)))
+    ctx.collective_pk(list(range(K)))
+    values = wl.gradients(cfg, 8, 0, 5)
+    dv = torch.from_numpy(values).to(ctx.device)
+    ws = torch.empty(ctx.round_workspace_bytes(5), dtype=torch.uint8, device=ctx.device)
+    ring = wl.regular_graph(K, 2, 8)
+    full = (np.arange(0, K * K + 1, K, dtype=np.uint32), np.tile(np.arange(K, dtype=np.uint32), K))
+    lone = (np.arange(K + 1, dtype=np.uint32), np.arange(K, dtype=np.uint32))  # every user alone
+    for offsets, rows in (ring, full, ring, lone, full):
+        sums = torch.full((K, 5, n), -1, dtype=torch.int32, device=ctx.device)
+        ctx.round_device(dv, 2, 5, offsets, rows, sums, ws)
+        ctx.sync()
+        want = np.stack([values[rows[offsets[i]:offsets[i + 1]]].astype(np.int64).sum(axis=0) for i in range(K)])
+        assert np.array_equal(sums.cpu().numpy(), want)
+    # a collective key over fewer parties: the list of share holders changes
+    ctx.collective_pk([0, 2])
+    sums = torch.zeros((K, 5, n), dtype=torch.int32, device=ctx.device)
+    offsets, rows = ring
+    ctx.round_device(dv, 2, 5, offsets, rows, sums, ws)
+    ctx.sync()
+    want = np.stack([values[rows[offsets[i]:offsets[i + 1]]].astype(np.int64).sum(axis=0) for i in range(K)])
+    assert np.array_equal(sums.cpu().numpy(), want)
+    ctx.close()
+
+
 def test_ciphertext_index_shards_reproduce_the_whole(d2):
     """Index ranges are independent: two half-ranges equal the full range bit for bit
     (this is how several GPUs split a round without exchanging data)."""
