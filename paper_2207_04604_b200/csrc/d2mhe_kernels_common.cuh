@@ -7,7 +7,7 @@
 // Octets per thread and round (G) and resident CTAs per SM aimed at, per ring degree.
 // Threads per CTA = N / (8 G).
 #ifndef D2MHE_G12
-#define D2MHE_G12 4
+#define D2MHE_G12 2
 #endif
 #ifndef D2MHE_G13
 #define D2MHE_G13 2
