@@ -82,6 +82,38 @@ __device__ __forceinline__ void load_octet_rw(const u64* src, u64 (&x)[8]) {
   }
 }
 
+// Rows in the transform domain that only this library reads (key tables, parked transforms) are kept
+// in interleaved order: the k-th pair of values of octet q (positions 8q + 2k, 8q + 2k + 1) sits in
+// 16-byte slot k * octets + q, octets = N / 8.  The threads of a warp own consecutive octets, so each of
+// the four 16-byte accesses of an octet covers 512 consecutive bytes (four 128-byte wavefronts of the
+// load/store pipe) instead of one slot in each of sixteen lines: measured 5-6 % on the share kernel,
+// whose other limit beside the integer multiplier is that pipe.  Pointwise work is indifferent to the
+// order; rows that cross the C ABI in the transform domain keep the plain order.
+__device__ __forceinline__ void store_octet_il(u64* row, u32 q, u32 octets, const u64 (&x)[8]) {
+  ulonglong2* d = reinterpret_cast<ulonglong2*>(row) + q;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) d[(size_t)k * octets] = make_ulonglong2(x[2 * k], x[2 * k + 1]);
+}
+__device__ __forceinline__ void load_octet_il(const u64* __restrict__ row, u32 q, u32 octets, u64 (&x)[8]) {
+  const ulonglong2* s = reinterpret_cast<const ulonglong2*>(row) + q;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const ulonglong2 t = __ldg(s + (size_t)k * octets);
+    x[2 * k] = t.x;
+    x[2 * k + 1] = t.y;
+  }
+}
+// plain (coherent) load of an octet that this kernel wrote earlier
+__device__ __forceinline__ void load_octet_rw_il(const u64* row, u32 q, u32 octets, u64 (&x)[8]) {
+  const ulonglong2* s = reinterpret_cast<const ulonglong2*>(row) + q;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const ulonglong2 t = s[(size_t)k * octets];
+    x[2 * k] = t.x;
+    x[2 * k + 1] = t.y;
+  }
+}
+
 // Lambda * m for a plaintext coefficient m < 2^32: exact quotient from two widening
 // products, result in [0, 2p).
 __device__ __forceinline__ u64 shoup_u32(u32 m, u64 w, u64 ws, u64 np) {

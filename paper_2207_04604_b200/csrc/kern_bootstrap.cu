@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
       ntt_forward<LOGN, G, WIDE>(
           sm, lt, v.logn,
           [&](u32 j) { return a == -2 ? __ldg(c1 + j) : uniform_mod(sa, j, lt.p, lt.mask); },
-          [&](int, u32 q, u64(&x)[8]) { store_octet(dst + 8 * (size_t)q, x); });
+          [&](int, u32 q, u64(&x)[8]) { store_octet_il(dst, q, v.n >> 3, x); });
       continue;
     }
     const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
@@ -96,8 +96,8 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
           sm, lt, v.logn,
           [&](int, u32 q, u64(&x)[8]) {
             u64 a8[8];
-            load_octet_rw(src + 8 * (size_t)q, a8);
-            load_octet(sk + 8 * (size_t)q, x);
+            load_octet_rw_il(src, q, v.n >> 3, a8);
+            load_octet_il(sk, q, v.n >> 3, x);
 #pragma unroll
             for (int k = 0; k < 8; ++k) x[k] = mont_lazy(a8[k], x[k], lt.p, lt.pinv);
           },

@@ -6,10 +6,10 @@
 namespace {
 
 // Montgomery form (times N^-1) of the eight transform values x[k]
-__device__ __forceinline__ void store_octet_mont(u64* __restrict__ dst, u64 (&x)[8], const LimbTab& lt) {
+__device__ __forceinline__ void store_octet_mont_il(u64* row, u32 q, u32 octets, u64 (&x)[8], const LimbTab& lt) {
 #pragma unroll
   for (int k = 0; k < 8; ++k) x[k] = shoup_full(x[k], lt.mont_ninv, lt.mont_ninv_sh, lt.p);
-  store_octet(dst, x);
+  store_octet_il(row, q, octets, x);
 }
 
 // Own key pair of user i (Algorithm 2, Require): sk_i from R_3 (BFV.SecKeyGen),
@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     const Stream st(v.seed, TAG_USER_SECRET, 0, user, 0);
     ntt_forward<LOGN, G, WIDE>(
         sm, lt, v.logn, [&](u32 j) { return lift_small(st.ternary(j), lt.p); },
-        [&](int, u32 q, u64(&x)[8]) { store_octet_mont(skm + 8 * (size_t)q, x, lt); });
+        [&](int, u32 q, u64(&x)[8]) { store_octet_mont_il(skm, q, v.n >> 3, x, lt); });
   }
   {
     const Stream st(v.seed, TAG_USER_P1, l, user, 0);
@@ -46,8 +46,8 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
           return r;
         },
         [&](int, u32 q, u64(&x)[8]) {
-          store_octet(pkc0 + 8 * (size_t)q, x);  // parked, lazily reduced
-          store_octet_mont(pkm1 + 8 * (size_t)q, x, lt);
+          store_octet_il(pkc0, q, v.n >> 3, x);  // parked, lazily reduced
+          store_octet_mont_il(pkm1, q, v.n >> 3, x, lt);
         });
   }
   {
@@ -56,8 +56,8 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
         sm, lt, v.logn,
         [&](int, u32 q, u64(&x)[8]) {
           u64 a[8];
-          load_octet_rw(pkc0 + 8 * (size_t)q, a);
-          load_octet_rw(skm + 8 * (size_t)q, x);
+          load_octet_rw_il(pkc0, q, v.n >> 3, a);
+          load_octet_rw_il(skm, q, v.n >> 3, x);
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = mont_lazy(a[k], x[k], lt.p, lt.pinv);
         },
@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
   __syncthreads();
   ntt_forward<LOGN, G, WIDE>(
       sm, lt, v.logn, [&](u32 j) { return pkc0[j]; },
-      [&](int, u32 q, u64(&x)[8]) { store_octet_mont(pkm0 + 8 * (size_t)q, x, lt); });
+      [&](int, u32 q, u64(&x)[8]) { store_octet_mont_il(pkm0, q, v.n >> 3, x, lt); });
 }
 
 // mu_k, e_{0,k}, e_{1,k} of a conversion share do not depend on the limb: like the noise of the
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     ntt_forward<LOGN, G, WIDE>(
         sm, lt, v.logn,
         [&](u32 j) { return a < 0 ? __ldg(c1 + j) : lift_small((int)small[j], lt.p); },
-        [&](int, u32 q, u64(&x)[8]) { store_octet(fwd_dst + 8 * (size_t)q, x); });
+        [&](int, u32 q, u64(&x)[8]) { store_octet_il(fwd_dst, q, v.n >> 3, x); });
     if (a < 0) continue;
     const u64* sk = v.s_mont + ((size_t)party * v.L + l) * v.n;
 #pragma unroll 1
@@ -150,14 +150,14 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
           sm, lt, v.logn,
           [&](int, u32 q, u64(&x)[8]) {
             u64 a8[8];
-            load_octet_rw(h1 + 8 * (size_t)q, a8);
-            load_octet(pkc + 8 * (size_t)q, x);
+            load_octet_rw_il(h1, q, v.n >> 3, a8);
+            load_octet_il(pkc, q, v.n >> 3, x);
 #pragma unroll
             for (int k = 0; k < 8; ++k) x[k] = mont_lazy(a8[k], x[k], lt.p, lt.pinv);
             if (comp == 0) {
               u64 b8[8];
-              load_octet_rw(park + 8 * (size_t)q, a8);
-              load_octet(sk + 8 * (size_t)q, b8);
+              load_octet_rw_il(park, q, v.n >> 3, a8);
+              load_octet_il(sk, q, v.n >> 3, b8);
 #pragma unroll
               for (int k = 0; k < 8; ++k) x[k] += mont_lazy(a8[k], b8[k], lt.p, lt.pinv);  // below 4p
             }
@@ -208,13 +208,13 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
   u64* out = prod + (size_t)unit * poly + row;
   ntt_forward<LOGN, G, WIDE>(
       sm, lt, v.logn, [&](u32 j) { return __ldg(c1 + j); },
-      [&](int, u32 q, u64(&x)[8]) { store_octet(out + 8 * (size_t)q, x); });
+      [&](int, u32 q, u64(&x)[8]) { store_octet_il(out, q, v.n >> 3, x); });
   ntt_inverse<LOGN, G, WIDE>(
       sm, lt, v.logn,
       [&](int, u32 q, u64(&x)[8]) {
         u64 a8[8];
-        load_octet_rw(out + 8 * (size_t)q, a8);
-        load_octet(sk + 8 * (size_t)q, x);
+        load_octet_rw_il(out, q, v.n >> 3, a8);
+        load_octet_il(sk, q, v.n >> 3, x);
 #pragma unroll
         for (int k = 0; k < 8; ++k) x[k] = mont_lazy(a8[k], x[k], lt.p, lt.pinv);
       },

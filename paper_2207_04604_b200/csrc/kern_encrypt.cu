@@ -59,7 +59,7 @@ __device__ __forceinline__ void encrypt_body(const DevView& v, const LimbParams&
   u64* park = ct + ((size_t)unit * 2 + (split > 1 ? part : 1u)) * poly + row;
   ntt_forward<LOGN, G, WIDE>(
       sm, lt, v.logn, [&](u32 j) { return lift_small((int)small[j], lt.p); },
-      [&](int, u32 q, u64(&x)[8]) { store_octet(park + 8 * (size_t)q, x); });
+      [&](int, u32 q, u64(&x)[8]) { store_octet_il(park, q, v.n >> 3, x); });
 #pragma unroll 1
   for (u32 comp = split > 1 ? part : 0u; comp < (split > 1 ? part + 1u : 2u); ++comp) {
     const u64* pkh = v.pk_mont + comp * poly + row;
@@ -69,8 +69,8 @@ __device__ __forceinline__ void encrypt_body(const DevView& v, const LimbParams&
         sm, lt, v.logn,
         [&](int, u32 q, u64(&x)[8]) {
           u64 uh[8];
-          load_octet_rw(park + 8 * (size_t)q, uh);  // written by this same thread
-          load_octet(pkh + 8 * (size_t)q, x);
+          load_octet_rw_il(park, q, v.n >> 3, uh);  // written by this same thread
+          load_octet_il(pkh, q, v.n >> 3, x);
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = mont_lazy(uh[k], x[k], lt.p, lt.pinv);
         },

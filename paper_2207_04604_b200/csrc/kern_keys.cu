@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
       [&](int, u32 q, u64(&x)[8]) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) x[k] = shoup_full(x[k], lt.mont_ninv, lt.mont_ninv_sh, lt.p);
-        store_octet(out + 8 * (size_t)q, x);
+        store_octet_il(out, q, v.n >> 3, x);
       });
 }
 
@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
             p1h[g][k] = x[k];
             y[k] = shoup_full(x[k], lt.mont_ninv, lt.mont_ninv_sh, lt.p);
           }
-          store_octet(v.pk_mont + poly + row + 8 * (size_t)q, y);
+          store_octet_il(v.pk_mont + poly + row, q, v.n >> 3, y);
         });
   }
   for (u32 a = 0; a < n_parties; ++a) {
@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     ntt_inverse<LOGN, G, WIDE>(
         sm, lt, v.logn,
         [&](int g, u32 q, u64(&x)[8]) {
-          load_octet(sk + 8 * (size_t)q, x);
+          load_octet_il(sk, q, v.n >> 3, x);
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = mont_lazy(p1h[g][k], x[k], lt.p, lt.pinv);
         },
@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
       [&](int, u32 q, u64(&x)[8]) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) x[k] = shoup_full(x[k], lt.mont_ninv, lt.mont_ninv_sh, lt.p);
-        store_octet(v.pk_mont + row + 8 * (size_t)q, x);
+        store_octet_il(v.pk_mont + row, q, v.n >> 3, x);
       });
 }
 
@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
   ntt_inverse<LOGN, G, WIDE>(
       poly_smem(), lt, v.logn,
       [&](int, u32 q, u64(&x)[8]) {
-        load_octet_rw(row + 8 * (size_t)q, x);
+        load_octet_rw_il(row, q, v.n >> 3, x);
 #pragma unroll
         for (int k = 0; k < 8; ++k) x[k] = mont_lazy(x[k], 1, lt.p, lt.pinv);  // leaves Montgomery form; below 2p
       },

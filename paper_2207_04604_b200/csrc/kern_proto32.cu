@@ -57,13 +57,14 @@ __device__ __forceinline__ void store_octet_halves(u32* da, u32* db, bool has_b,
   if (has_b) store_octet32(db, hi);
 }
 // pointwise products of both parked transforms with one key row: halves below 2p
-__device__ __forceinline__ void product_octet_pair(const u32* pa, const u32* pb, const u64* __restrict__ key, u32 p,
-                                                   u64 (&x)[8]) {
+// (the key row is in the interleaved order of the key tables: octet q of `octets`)
+__device__ __forceinline__ void product_octet_pair(const u32* pa, const u32* pb, const u64* __restrict__ key, u32 q,
+                                                   u32 octets, u32 p, u64 (&x)[8]) {
   u32 a[8], b[8];
   u64 k[8];
   load_octet32(pa, a);
   load_octet32(pb, b);
-  load_octet(key, k);
+  load_octet_il(key, q, octets, k);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     u32 kl, kh;
@@ -121,7 +122,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     ntt_inverse<LOGN, G, MODE_PAIR>(
         sm, lt, v.logn,
         [&](int, u32 q, u64(&x)[8]) {
-          product_octet_pair(park_a + 8 * (size_t)q, park_b + 8 * (size_t)q, key + 8 * (size_t)q, p, x);
+          product_octet_pair(park_a + 8 * (size_t)q, park_b + 8 * (size_t)q, key, q, v.n >> 3, p, x);
         },
         [&](u32 j, u64 val) {
           u32 lo, hi;
@@ -184,7 +185,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     ntt_inverse<LOGN, G, MODE_PAIR>(
         sm, lt, v.logn,
         [&](int, u32 q, u64(&x)[8]) {
-          product_octet_pair(park_a + 8 * (size_t)q, park_b + 8 * (size_t)q, key + 8 * (size_t)q, p, x);
+          product_octet_pair(park_a + 8 * (size_t)q, park_b + 8 * (size_t)q, key, q, v.n >> 3, p, x);
         },
         [&](u32 j, u64 val) {
           u32 lo, hi;
