@@ -538,6 +538,9 @@ struct NttGeom {
 // s >= GB), so those rounds are separated by a named barrier of the group only and the groups drift
 // apart: one group's shared-memory phase overlaps another's arithmetic.  Rounds that span the
 // quarters keep the CTA-wide barrier.  GB = 0 turns this off.
+#ifndef D2MHE_LATE_BARRIER
+#define D2MHE_LATE_BARRIER 0
+#endif
 #ifndef D2MHE_GB14
 #define D2MHE_GB14 2
 #endif
@@ -672,7 +675,7 @@ __device__ __forceinline__ void ntt_forward(u64* __restrict__ sm, const LimbTab&
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = sm_get(sm, ad.at(k, sh), smb, md);
         }
-        if (WIDE == MODE_PAIR && last && soff == 0)  // pays only where shared-memory wavefronts bind
+        if (last && soff == 0)  // every thread has seven twiddles of its own here: consecutive entries of the regrouped copy
           fwd_octet_last<WIDE>(x, lt.WL, ge.octets, i, md);
         else
           fwd_octet<WIDE>(x, W, m << soff, (blk << s) + i, 3, md);
@@ -709,7 +712,9 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
   const u32 smb = ge.n << 3;  // bytes of the shared-memory polynomial
   const ulonglong2* __restrict__ IW = lt.IW;
   u64 x[8];
+#if !D2MHE_LATE_BARRIER
   __syncthreads();  // previous users of sm are done
+#endif
   bool from_fetch = true;
 #pragma unroll
   for (int s = (int)ge.logn - 3; s >= (int)ge.r0; s -= 3) {
@@ -735,10 +740,21 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
 #pragma unroll
           for (int k = 0; k < 8; ++k) x[k] = sm_get(sm, ad.at(k, sh), smb, md);
         }
-        if (WIDE == MODE_PAIR && from_fetch && soff == 0)
+        if (from_fetch && soff == 0)
           inv_octet_first<WIDE>(x, lt.IWL, ge.octets, i, md);
         else
           inv_octet<WIDE>(x, IW, m << soff, (blk << s) + i, 3, md);
+#if D2MHE_LATE_BARRIER
+      }
+      // Previous users of sm are done.  The first octet of a transform is fetched and taken through its
+      // first round before this barrier, which only the shared-memory stores have to wait for: the skew
+      // between the threads of the block is spent on loads and arithmetic instead of idling.
+      if (from_fetch && g == 0) __syncthreads();
+      if (LOGN || q < ge.octets) {
+        const u32 i = q >> sh, o = q & ((1u << sh) - 1);
+        const u32 base = ((i << 3) << sh) + o;
+        const OctAddr ad(base, sh);
+#endif
         if (final_round) {
           finish_octet<WIDE>(x, 3, md);
 #pragma unroll
