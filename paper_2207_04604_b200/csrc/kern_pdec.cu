@@ -2,6 +2,7 @@
 #include <algorithm>
 
 #define D2MHE_SHIFT_AS_MULTIPLY 1  // see shoup_approx_sf: measured faster in this kernel only
+#define D2MHE_LATE_BARRIER 1       // see ntt_inverse: 0.3-0.7 % here, slower in the stand-alone inverse transform
 #include "d2mhe_kernels_common.cuh"
 
 namespace {
