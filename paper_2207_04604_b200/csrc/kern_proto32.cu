@@ -40,30 +40,34 @@ __device__ __forceinline__ UnitPair unit_pair(u32 pr, u32 n_units) {
   return u;
 }
 
-__device__ __forceinline__ void load_octet32(const u32* src, u32 (&x)[8]) {  // coherent: may be this kernel's own data
-  const uint4 a = reinterpret_cast<const uint4*>(src)[0], b = reinterpret_cast<const uint4*>(src)[1];
+// Parked 32-bit rows are in interleaved octet order like the key rows: the two 16-byte halves of octet q
+// in slots q and octets + q, so that a warp's access covers 512 consecutive bytes.
+__device__ __forceinline__ void load_octet32_il(const u32* row, u32 q, u32 octets, u32 (&x)[8]) {  // coherent: this kernel's own data
+  const uint4* s = reinterpret_cast<const uint4*>(row) + q;
+  const uint4 a = s[0], b = s[octets];
   x[0] = a.x, x[1] = a.y, x[2] = a.z, x[3] = a.w, x[4] = b.x, x[5] = b.y, x[6] = b.z, x[7] = b.w;
 }
-__device__ __forceinline__ void store_octet32(u32* dst, const u32 (&x)[8]) {
-  reinterpret_cast<uint4*>(dst)[0] = make_uint4(x[0], x[1], x[2], x[3]);
-  reinterpret_cast<uint4*>(dst)[1] = make_uint4(x[4], x[5], x[6], x[7]);
+__device__ __forceinline__ void store_octet32_il(u32* row, u32 q, u32 octets, const u32 (&x)[8]) {
+  uint4* d = reinterpret_cast<uint4*>(row) + q;
+  d[0] = make_uint4(x[0], x[1], x[2], x[3]);
+  d[octets] = make_uint4(x[4], x[5], x[6], x[7]);
 }
-// halves of the eight pair words -> the two polynomials' rows
-__device__ __forceinline__ void store_octet_halves(u32* da, u32* db, bool has_b, const u64 (&x)[8]) {
+// halves of the eight pair words -> the two polynomials' parked rows
+__device__ __forceinline__ void store_octet_halves(u32* ra, u32* rb, u32 q, u32 octets, bool has_b, const u64 (&x)[8]) {
   u32 lo[8], hi[8];
 #pragma unroll
   for (int k = 0; k < 8; ++k) split64(x[k], lo[k], hi[k]);
-  store_octet32(da, lo);
-  if (has_b) store_octet32(db, hi);
+  store_octet32_il(ra, q, octets, lo);
+  if (has_b) store_octet32_il(rb, q, octets, hi);
 }
 // pointwise products of both parked transforms with one key row: halves below 2p
-// (the key row is in the interleaved order of the key tables: octet q of `octets`)
+// (the parked rows and the key row are in interleaved order: octet q of `octets`)
 __device__ __forceinline__ void product_octet_pair(const u32* pa, const u32* pb, const u64* __restrict__ key, u32 q,
                                                    u32 octets, u32 p, u64 (&x)[8]) {
   u32 a[8], b[8];
   u64 k[8];
-  load_octet32(pa, a);
-  load_octet32(pb, b);
+  load_octet32_il(pa, q, octets, a);
+  load_octet32_il(pb, q, octets, b);
   load_octet_il(key, q, octets, k);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -108,7 +112,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
         const int a = sa[j], b = sb[j];
         return join64(a < 0 ? p + (u32)a : (u32)a, b < 0 ? p + (u32)b : (u32)b);
       },
-      [&](int, u32 q, u64(&x)[8]) { store_octet_halves(park_a + 8 * (size_t)q, park_b + 8 * (size_t)q, up.has_b, x); });
+      [&](int, u32 q, u64(&x)[8]) { store_octet_halves(park_a, park_b, q, v.n >> 3, up.has_b, x); });
   const u32* ma = plain + (size_t)ua * v.n;
   const u32* mb = plain + (size_t)ub * v.n;
   const u32 delta = (u32)lt.delta, delta_sh = (u32)(lt.delta_sh >> 32);
@@ -122,7 +126,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     ntt_inverse<LOGN, G, MODE_PAIR>(
         sm, lt, v.logn,
         [&](int, u32 q, u64(&x)[8]) {
-          product_octet_pair(park_a + 8 * (size_t)q, park_b + 8 * (size_t)q, key, q, v.n >> 3, p, x);
+          product_octet_pair(park_a, park_b, key, q, v.n >> 3, p, x);
         },
         [&](u32 j, u64 val) {
           u32 lo, hi;
@@ -161,7 +165,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
   u32* park_b = shares + (((size_t)irb * n_parties + (n_parties - 1)) * n_cts + clb) * poly + row;
   ntt_forward<LOGN, G, MODE_PAIR>(
       sm, lt, v.logn, [&](u32 j) { return join64(__ldg(c1a + j), __ldg(c1b + j)); },
-      [&](int, u32 q, u64(&x)[8]) { store_octet_halves(park_a + 8 * (size_t)q, park_b + 8 * (size_t)q, up.has_b, x); });
+      [&](int, u32 q, u64(&x)[8]) { store_octet_halves(park_a, park_b, q, v.n >> 3, up.has_b, x); });
 #pragma unroll 1
   for (u32 a = 0; a < n_parties; ++a) {
     const u32 party = parties[a];
@@ -185,7 +189,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
     ntt_inverse<LOGN, G, MODE_PAIR>(
         sm, lt, v.logn,
         [&](int, u32 q, u64(&x)[8]) {
-          product_octet_pair(park_a + 8 * (size_t)q, park_b + 8 * (size_t)q, key, q, v.n >> 3, p, x);
+          product_octet_pair(park_a, park_b, key, q, v.n >> 3, p, x);
         },
         [&](u32 j, u64 val) {
           u32 lo, hi;
