@@ -1,6 +1,8 @@
 // MBFV.Bootstrap (Sec. 4.2 item 4, Eq. 4): collective noise refresh.
 #include <algorithm>
 
+#define D2MHE_SHIFT_AS_MULTIPLY 1  // as in the decryption-share kernel: measured 0.7-1 % faster here with both
+#define D2MHE_LATE_BARRIER 1
 #include "d2mhe_kernels_common.cuh"
 
 namespace {
