@@ -32,7 +32,10 @@ __device__ __forceinline__ u64 mont_lazy_sf(u64 a, u64 b, u64 p, u64 pinv, u32 d
 // kernel and spread the samples over a cluster of the limbs' CTAs was 3 % slower at N = 8192 and
 // 8 % at N = 16384, where clusters of one-CTA-per-SM blocks also leave SMs idle.)
 //
-// grid = ceil(n_units * n_parties * N / 4 / 256); one thread = four samples = one packed word.
+// grid = ceil(n_units * n_parties * N / 4 / (256 * D2MHE_SAMPLE_WORDS)); one packed word = four samples.
+#ifndef D2MHE_SAMPLE_WORDS
+#define D2MHE_SAMPLE_WORDS 4
+#endif
 // noise[(u * n_parties + a) * N + j], u = unit - unit_first, unit = irec * n_cts + cl.
 __global__ void __launch_bounds__(256)
     k_sample_share_noise(DevView v, const u32* __restrict__ recipients, const u32* __restrict__ parties,
@@ -42,18 +45,21 @@ __global__ void __launch_bounds__(256)
   load_gauss(&gt, v.gauss);
   const u32 words = v.n >> 2;
   const size_t total = (size_t)n_units * n_parties * words;
-  const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= total) return;
-  const u32 w = (u32)(e % words);
-  const size_t share = e / words;
-  const u32 a = (u32)(share % n_parties), unit = unit_first + (u32)(share / n_parties);
-  const u32 party = parties[a], recipient = recipients[unit / n_cts];
-  if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY) || !D2MHE_CHK(v.chk, recipient, v.K, SITE_PARTY)) return;
-  const Stream se(v.seed, TAG_DEC_ERR, ct_first + unit % n_cts, party, recipient);
-  u32 pack = 0;
+#pragma unroll 1
+  for (u32 it = 0; it < D2MHE_SAMPLE_WORDS; ++it) {  // several words per thread: the table load above is paid once
+    const size_t e = ((size_t)blockIdx.x * D2MHE_SAMPLE_WORDS + it) * blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const u32 w = (u32)(e % words);
+    const size_t share = e / words;
+    const u32 a = (u32)(share % n_parties), unit = unit_first + (u32)(share / n_parties);
+    const u32 party = parties[a], recipient = recipients[unit / n_cts];
+    if (!D2MHE_CHK(v.chk, party, v.K, SITE_PARTY) || !D2MHE_CHK(v.chk, recipient, v.K, SITE_PARTY)) continue;
+    const Stream se(v.seed, TAG_DEC_ERR, ct_first + unit % n_cts, party, recipient);
+    u32 pack = 0;
 #pragma unroll
-  for (u32 b = 0; b < 4; ++b) pack |= ((u32)gauss_from_r(gt, se.draw64(4 * w + b)) & 0xffu) << (8 * b);
-  noise[e] = pack;
+    for (u32 b = 0; b < 4; ++b) pack |= ((u32)gauss_from_r(gt, se.draw64(4 * w + b)) & 0xffu) << (8 * b);
+    noise[e] = pack;
+  }
 }
 
 // grid = n_units * L * split; units unit_first .. unit_first + n_units - 1 of the (recipient, ciphertext)
@@ -132,7 +138,7 @@ namespace D2MHE_LAUNCH_NS {
 cudaError_t sample_share_noise(const DevView& v, cudaStream_t s, const u32* recipients_dev, const u32* parties_dev,
                                u32 n_parties, u32 ct_first, u32 n_cts, u32 unit_first, u32 n_units, u32* out) {
   const size_t words = (size_t)n_units * n_parties * v.n / 4;
-  k_sample_share_noise<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(v, recipients_dev, parties_dev, n_parties,
+  k_sample_share_noise<<<(unsigned)((words + 256 * D2MHE_SAMPLE_WORDS - 1) / (256 * D2MHE_SAMPLE_WORDS)), 256, 0, s>>>(v, recipients_dev, parties_dev, n_parties,
                                                                       ct_first, n_cts, unit_first, n_units, out);
   return cudaGetLastError();
 }
