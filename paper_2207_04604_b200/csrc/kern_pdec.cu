@@ -1,7 +1,9 @@
 // Decryption shares: h = s_k c_1 + e for every listed share holder.
 #include <algorithm>
 
+#ifndef D2MHE_SHIFT_AS_MULTIPLY
 #define D2MHE_SHIFT_AS_MULTIPLY 1  // see shoup_approx_sf: measured faster in this kernel only
+#endif
 #define D2MHE_LATE_BARRIER 1       // see ntt_inverse: 0.3-0.7 % here, slower in the stand-alone inverse transform
 #include "d2mhe_kernels_common.cuh"
 
