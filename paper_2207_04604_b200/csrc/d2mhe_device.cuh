@@ -442,7 +442,7 @@ __device__ __forceinline__ void fwd_octet_last(u64 (&x)[8], const ulonglong2* __
 }
 template <int MODE>
 __device__ __forceinline__ void inv_octet_first(u64 (&x)[8], const ulonglong2* __restrict__ IWL, u32 oc,
-                                                u32 i, const Mod& md) {
+                                                u32 i, const Mod& md, bool reduce0 = true) {
   const u64 c16 = md.fourp << 2, c32 = md.fourp << 3, c64 = md.fourp << 4;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
@@ -461,7 +461,7 @@ __device__ __forceinline__ void inv_octet_first(u64 (&x)[8], const ulonglong2* _
 #pragma unroll
     for (int k = 0; k < 4; ++k) gs_bfly<MODE>(x[k], x[k + 4], w, md, c64);
   }
-  if (MODE == MODE_WIDE) x[0] = reduce_small(x[0], md);
+  if (MODE == MODE_WIDE && reduce0) x[0] = reduce_small(x[0], md);
 }
 
 // Inverse stages on an octet whose inputs are all below 16p (WIDE) / 4p (otherwise).
@@ -469,7 +469,7 @@ __device__ __forceinline__ void inv_octet_first(u64 (&x)[8], const ulonglong2* _
 // back below 4p here, so every output is again below 16p.
 template <int MODE>
 __device__ __forceinline__ void inv_octet(u64 (&x)[8], const ulonglong2* __restrict__ IW, u32 m,
-                                          u32 i, int nst, const Mod& md) {
+                                          u32 i, int nst, const Mod& md, bool reduce0 = true) {
   const u64 c16 = md.fourp << 2, c32 = md.fourp << 3, c64 = md.fourp << 4;
   if (nst >= 3) {
 #pragma unroll
@@ -490,7 +490,7 @@ __device__ __forceinline__ void inv_octet(u64 (&x)[8], const ulonglong2* __restr
 #pragma unroll
     for (int k = 0; k < 4; ++k) gs_bfly<MODE>(x[k], x[k + 4], w, md, c64);
   }
-  if (MODE == MODE_WIDE) x[0] = reduce_small(x[0], md);
+  if (MODE == MODE_WIDE && reduce0) x[0] = reduce_small(x[0], md);
 }
 
 // Brings the outputs of the last inverse round below 4p.  After a full round the bounds are
@@ -699,7 +699,10 @@ struct NoHook {
   __device__ __forceinline__ void operator()() const {}
 };
 // before_final() is called by every thread just before the round that calls store().
-template <int LOGN, int G, int WIDE, class Fetch, class Store, class Hook = NoHook>
+// LAZY_OUT (WIDE only): the last round skips its reductions and store() receives values below 129p
+// (the bounds listed at inv_octet, without bringing x0 back); for a caller whose store() reduces by the
+// 2^b - d fold (canon8<true>), which takes any such value in one step.
+template <int LOGN, int G, int WIDE, bool LAZY_OUT = false, class Fetch, class Store, class Hook = NoHook>
 __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab& lt, u32 logn_rt,
                                             Fetch fetch, Store store, u32 soff = 0, u32 blk = 0,
                                             Hook before_final = Hook()) {
@@ -741,9 +744,9 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
           for (int k = 0; k < 8; ++k) x[k] = sm_get(sm, ad.at(k, sh), smb, md);
         }
         if (from_fetch && soff == 0)
-          inv_octet_first<WIDE>(x, lt.IWL, ge.octets, i, md);
+          inv_octet_first<WIDE>(x, lt.IWL, ge.octets, i, md, !(LAZY_OUT && final_round));
         else
-          inv_octet<WIDE>(x, IW, m << soff, (blk << s) + i, 3, md);
+          inv_octet<WIDE>(x, IW, m << soff, (blk << s) + i, 3, md, !(LAZY_OUT && final_round));
 #if D2MHE_LATE_BARRIER
       }
       // Previous users of sm are done.  The first octet of a transform is fetched and taken through its
@@ -756,7 +759,7 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
         const OctAddr ad(base, sh);
 #endif
         if (final_round) {
-          finish_octet<WIDE>(x, 3, md);
+          if (!LAZY_OUT) finish_octet<WIDE>(x, 3, md);
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const u32 j = base + ((u32)k << sh);
@@ -782,8 +785,8 @@ __device__ __forceinline__ void ntt_inverse(u64* __restrict__ sm, const LimbTab&
         const OctAddr ad(q, sh);
 #pragma unroll
         for (int k = 0; k < 8; ++k) x[k] = sm_get(sm, ad.at(k, sh), smb, md);
-        inv_octet<WIDE>(x, IW, 1u << soff, blk, (int)ge.r0, md);
-        finish_octet<WIDE>(x, (int)ge.r0, md);
+        inv_octet<WIDE>(x, IW, 1u << soff, blk, (int)ge.r0, md, !LAZY_OUT);
+        if (!LAZY_OUT) finish_octet<WIDE>(x, (int)ge.r0, md);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const u32 j = q + ((u32)k << sh);

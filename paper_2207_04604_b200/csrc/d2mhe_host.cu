@@ -230,7 +230,7 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   // floor(q/t) mod q_l: q = Delta t + (q mod t)  =>  Delta = -(q mod t) t^-1 (mod q_l)
   const u64 q_mod_t = q_mod(t);
 
-  bool all_special = true;  // every prime is 2^b - d with b >= 32, d < 2^32 and 16 d < 2^b
+  bool all_special = true;  // every prime is 2^b - d with b >= 32, d < 2^32 and 256 d < 2^b
   for (u32 l = 0; l < L; ++l) {
     const u64 p = c->moduli[l];
     LimbTab& T = limbs[l];
@@ -263,7 +263,7 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
     T.red_shift = bits - 1;
     T.red_mul = (u32)(((u128)1 << (bits + 15)) / p);
     const u64 gap = bits >= 64 ? 0 : (((u64)1 << bits) - p);  // p = 2^bits - gap
-    const bool special = bits >= 32 && gap < ((u64)1 << 32) && (u128)16 * gap < ((u128)1 << bits);
+    const bool special = bits >= 32 && gap < ((u64)1 << 32) && (u128)256 * gap < ((u128)1 << bits);
     T.sf_d = special ? (u32)gap : 0;
     T.sf_shift = special ? bits - 32 : 0;
     if (!special) all_special = false;

@@ -128,24 +128,26 @@ __device__ __forceinline__ u64 shoup_u32(u32 m, u64 w, u64 ws, u64 np) {
   return join64(rl, rh);
 }
 
-// Canonical representative of s < 8p.  SF: the prime is 2^b - d with 16 d < 2^b (every context that
+// Canonical representative of s < 8p.  SF: the prime is 2^b - d with 256 d < 2^b (every context that
 // runs the WIDE policy); then s = k 2^b + rem is congruent to rem + k d, which is below
 // 2^b + 7d < 2p: one widening multiply-add and one conditional subtraction instead of three.
+// With SF the same holds for any s below 2^(b+7) + 2^b (k <= 129: rem + k d < p + 130 d < 2p), which is
+// what an inverse transform with LAZY_OUT hands over.
 template <bool SF = false>
 __device__ __forceinline__ u64 canon8(u64 s, const LimbTab& lt) {
   if (SF) {
     u32 s0, s1;
     split64(s, s0, s1);
-    const u32 k = s1 >> lt.sf_shift;  // s / 2^b, at most 7
+    const u32 k = s1 >> lt.sf_shift;  // s / 2^b
     return csub(madwide(k, lt.sf_d, join64(s0, s1 & ((1u << lt.sf_shift) - 1u))), lt.p);
   }
   return csub(csub(csub(s, 2 * lt.twop), lt.twop), lt.p);
 }
 
-// v (below 4p) + small signed e, canonical in [0, p)
+// v (below 4p; with SF below 129p) + small signed e, canonical in [0, p)
 template <bool SF = false>
 __device__ __forceinline__ u64 add_small_canon(u64 v, int e, const LimbTab& lt) {
-  return canon8<SF>(v + lt.p + (u64)(long long)e, lt);  // below 5p + 19
+  return canon8<SF>(v + lt.p + (u64)(long long)e, lt);  // below 5p + 19 (SF: below 130p + 19)
 }
 
 constexpr u32 ntt_threads_ct(int logn, int g) {

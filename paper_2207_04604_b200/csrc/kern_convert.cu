@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
       const u64* pkc = comp ? pk1 : pk0;
       u64* out = comp ? h1 : h0;
       const signed char* e = small + (comp + 1) * v.n;
-      ntt_inverse<LOGN, G, WIDE>(
+      ntt_inverse<LOGN, G, WIDE, true>(
           sm, lt, v.logn,
           [&](int, u32 q, u64(&x)[8]) {
             u64 a8[8];

@@ -65,7 +65,7 @@ __device__ __forceinline__ void encrypt_body(const DevView& v, const LimbParams&
     const u64* pkh = v.pk_mont + comp * poly + row;
     u64* out = ct + ((size_t)unit * 2 + comp) * poly + row;
     const signed char* e = small + (comp + 1) * v.n;
-    ntt_inverse<LOGN, G, WIDE>(
+    ntt_inverse<LOGN, G, WIDE, true>(  // lazy last round: both stores below reduce by the 2^b - d fold
         sm, lt, v.logn,
         [&](int, u32 q, u64(&x)[8]) {
           u64 uh[8];
@@ -76,9 +76,9 @@ __device__ __forceinline__ void encrypt_body(const DevView& v, const LimbParams&
         },
         [&](u32 j, u64 val) {
           if (comp == 0) {
-            // below 4p + (p + 19) + 2p
+            // below 4p + (p + 19) + 2p (WIDE: val below 129p, the fold takes it)
             u64 t = val + lt.p + (u64)(long long)e[j] + shoup_u32(m[j], lt.delta, lt.delta_sh, lt.np);
-            out[j] = canon8<WIDE>(t, lt);  // t below 7p + 19
+            out[j] = canon8<WIDE>(t, lt);  // t below 7p + 19 (WIDE: below 132p + 19)
           } else {
             out[j] = add_small_canon<WIDE>(val, (int)e[j], lt);
           }

@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(ntt_threads_ct(LOGN, G), ntt_minb_ct(LOGN, G))
       }
     }
     u64* out = shares + (((size_t)irec * n_parties + a) * n_cts + cl) * poly + row;
-    ntt_inverse<LOGN, G, WIDE>(
+    ntt_inverse<LOGN, G, WIDE, true>(  // the store below folds any value the lazy last round leaves
         sm, lt, v.logn,
         [&](int, u32 q, u64(&x)[8]) {
           u64 ch[8];
