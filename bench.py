@@ -140,7 +140,7 @@ def algorithmic_mad_slots(cfg, n_cts):
 # from the ncu captures under profiles/ (taken on a few ciphertext indices of the configuration and
 # scaled by the units of a launch: the traffic is the shares written plus c_1 and the noise bytes
 # read, all proportional to the units).  None when the kernel has changed since the capture.
-NCU_TRAFFIC_BYTES_PER_UNIT = {("resnet18-K50", "partial_decrypt"): (593737984 + 5262386000) / 100.0}
+NCU_TRAFFIC_BYTES_PER_UNIT = {("resnet18-K50", "partial_decrypt"): (589769984 + 5258257000) / 100.0}
 
 
 def measure_int_peak(ctx):
