@@ -34,22 +34,19 @@ __device__ __forceinline__ u64 mont_lazy_sf(u64 a, u64 b, u64 p, u64 pinv, u32 d
 // kernel and spread the samples over a cluster of the limbs' CTAs was 3 % slower at N = 8192 and
 // 8 % at N = 16384, where clusters of one-CTA-per-SM blocks also leave SMs idle.)
 //
-// grid = ceil(n_units * n_parties * N / 4 / (256 * D2MHE_SAMPLE_WORDS)); one packed word = four samples.
-#ifndef D2MHE_SAMPLE_WORDS
-#define D2MHE_SAMPLE_WORDS 4
-#endif
+// grid = ceil(n_units * n_parties * N / 4 / (256 * wpt)); one packed word = four samples, wpt words per thread.
 // noise[(u * n_parties + a) * N + j], u = unit - unit_first, unit = irec * n_cts + cl.
 __global__ void __launch_bounds__(256)
     k_sample_share_noise(DevView v, const u32* __restrict__ recipients, const u32* __restrict__ parties,
                          u32 n_parties, u32 ct_first, u32 n_cts, u32 unit_first, u32 n_units,
-                         u32* __restrict__ noise) {
+                         u32* __restrict__ noise, u32 wpt) {
   __shared__ GaussTab gt;
   load_gauss(&gt, v.gauss);
   const u32 words = v.n >> 2;
   const size_t total = (size_t)n_units * n_parties * words;
 #pragma unroll 1
-  for (u32 it = 0; it < D2MHE_SAMPLE_WORDS; ++it) {  // several words per thread: the table load above is paid once
-    const size_t e = ((size_t)blockIdx.x * D2MHE_SAMPLE_WORDS + it) * blockDim.x + threadIdx.x;
+  for (u32 it = 0; it < wpt; ++it) {  // several words per thread: the table load above is paid once
+    const size_t e = ((size_t)blockIdx.x * wpt + it) * blockDim.x + threadIdx.x;
     if (e >= total) return;
     const u32 w = (u32)(e % words);
     const size_t share = e / words;
@@ -140,8 +137,11 @@ namespace D2MHE_LAUNCH_NS {
 cudaError_t sample_share_noise(const DevView& v, cudaStream_t s, const u32* recipients_dev, const u32* parties_dev,
                                u32 n_parties, u32 ct_first, u32 n_cts, u32 unit_first, u32 n_units, u32* out) {
   const size_t words = (size_t)n_units * n_parties * v.n / 4;
-  k_sample_share_noise<<<(unsigned)((words + 256 * D2MHE_SAMPLE_WORDS - 1) / (256 * D2MHE_SAMPLE_WORDS)), 256, 0, s>>>(v, recipients_dev, parties_dev, n_parties,
-                                                                      ct_first, n_cts, unit_first, n_units, out);
+  // four words per thread once the grid is several waves deep (the table load and its barrier are then paid
+  // once per 4096 samples); small calls keep one word per thread: their latency is what counts
+  const u32 wpt = words >= (size_t)256 * 4 * 8 * v.sms * 2 ? 4u : 1u;
+  k_sample_share_noise<<<(unsigned)((words + 256 * (size_t)wpt - 1) / (256 * (size_t)wpt)), 256, 0, s>>>(
+      v, recipients_dev, parties_dev, n_parties, ct_first, n_cts, unit_first, n_units, out, wpt);
   return cudaGetLastError();
 }
 
