@@ -373,7 +373,7 @@ d2mhe_status d2mhe_debug_export_user_secret(d2mhe_ctx* ctx, uint32_t user, int8_
  * stream (the call synchronises).  kind 0: mad.lo.u32, 1: mad.wide.u32 with a 64-bit addend,
  * 2: mad.hi.u32 (32 lane operations per warp instruction), 3: the engine's forward butterfly on
  * eight coefficients per thread (operations = butterflies; needs a parameter set whose primes
- * are all below 2^57 and of the form 2^b - d, else D2MHE_ERR_UNSUPPORTED), 4: mul.wide.u32,
+ * are all below 2^56 and of the form 2^b - d, else D2MHE_ERR_UNSUPPORTED), 4: mul.wide.u32,
  * 5: mul.hi.u32 (both without an addend), 6: mad.wide.u32 with a loop-invariant addend.
  * 1 <= iters <= 2^24. */
 d2mhe_status d2mhe_debug_int_throughput(d2mhe_ctx* ctx, uint32_t kind, uint32_t iters,

@@ -306,7 +306,7 @@ __device__ __forceinline__ u64 shoup_approx_sf(u64 y, u64 w, u64 ws, u32 d, u32 
   return join64(rl, rh);
 }
 
-// Lazy-reduction policy.  WIDE (every prime below 2^57 and of the form above): values may grow across stages, so
+// Lazy-reduction policy.  WIDE (every prime below 2^56 and of the form above): values may grow across stages, so
 // the forward transform needs no conditional subtraction at all and the inverse reduces only
 // the one element per octet that accumulates the sums.  Otherwise (primes up to 2^61) values
 // are kept below 8p with one conditional subtraction per butterfly.
@@ -337,7 +337,7 @@ __device__ __forceinline__ u64 reduce_small(u64 x, const Mod& m) {
 }
 
 // Arithmetic mode of the engine: 0 = one residue per word, primes up to 2^61; 1 = the same with
-// the WIDE policy above (primes below 2^57); 2 = "pair": every 64-bit word carries two 32-bit
+// the WIDE policy above (primes below 2^56); 2 = "pair": every 64-bit word carries two 32-bit
 // residues of the same prime below 2^30 (two polynomials transformed side by side with the
 // same twiddles), each half with Harvey's lazy butterflies in 32-bit arithmetic: one high and
 // two low multiplies per butterfly instead of five and four.

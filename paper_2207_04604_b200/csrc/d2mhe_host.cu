@@ -432,7 +432,7 @@ d2mhe_status build_tables(d2mhe_ctx* c) {
   c->view.K = P.num_parties;
   c->view.wide = all_special ? 1 : 0;
   for (u32 l = 0; l < L; ++l)
-    if (c->moduli[l] >= ((u64)1 << 57)) c->view.wide = 0;
+    if (c->moduli[l] >= ((u64)1 << 56)) c->view.wide = 0;  // 130 p (a lazily grown value plus its additive terms) must fit 64 bits
 
   // index staging ring
   err = cudaMallocHost(reinterpret_cast<void**>(&c->idx_host), kIdxSlots * kIdxSlotWords * sizeof(u32));

@@ -43,7 +43,7 @@ struct DevView {
   u64 seed;
   u32 logn, n, L, K;
   u32 sms;       // multiprocessors of the device (launch shaping only)
-  u32 wide;      // 1 if every q_l < 2^57: lazy-reduction policy with no conditional subtractions
+  u32 wide;      // 1 if every q_l < 2^56: lazy-reduction policy with no conditional subtractions
   u64* s_mont;   // [K][L][N]  NTT(s_k) * N^-1 in Montgomery form
   u64* pk_mont;  // [2][L][N]  NTT(p_0), NTT(p_1) * N^-1 in Montgomery form
   u64* pk_coef;  // [2][L][N]  (p_0, p_1), coefficient domain

@@ -232,7 +232,7 @@ cudaError_t launch_clustered(void (*kernel)(KArgs...), u32 grid, u32 threads, si
 
 // Picks the instantiation for the ring degree: compile-time sizes for the production
 // degrees (with the octets-per-thread count G chosen per degree), the run-time-size build
-// for everything else; `wide` selects the lazy-reduction policy (all primes below 2^57).
+// for everything else; `wide` selects the lazy-reduction policy (all primes below 2^56).
 // extra = bytes of small-sample storage in front of the polynomial; cs = cluster size.
 #define D2MHE_DISPATCH_EX(KERNEL, view, grid, stream, extra, cs, ...)                          \
   do {                                                                                         \

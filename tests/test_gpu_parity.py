@@ -337,7 +337,7 @@ def _run_round(d2, ctx, o, cfg_k, parties, offsets, rows, values, ct_first, keep
     return got
 
 
-@pytest.mark.parametrize("log2_n,bits,L,K", [(3, 36, 2, 3), (4, 30, 2, 3), (5, 36, 3, 4), (6, 54, 2, 2), (8, 60, 3, 3), (10, 54, 5, 3)])
+@pytest.mark.parametrize("log2_n,bits,L,K", [(3, 36, 2, 3), (4, 30, 2, 3), (5, 36, 3, 4), (6, 54, 2, 2), (8, 60, 3, 3), (10, 54, 5, 3), (6, 56, 2, 3), (7, 57, 2, 2)])
 def test_small_rings_every_message(d2, log2_n, bits, L, K):
     moduli = small_moduli(log2_n, bits, L)
     seed = 77 + log2_n
